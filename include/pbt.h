@@ -1,0 +1,255 @@
+/*
+ * pbt.h -- C ABI of the lockstep Population Based Training library for one
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library trains a whole population of small networks concurrently on one
+ * GPU, each member with its own hyperparameter vector h, and interleaves the
+ * paper's exploit / explore step (Algorithm 1 of "Population Based Training of
+ * Neural Networks", executed in the partial-synchrony form of Appendix A.1: all
+ * members advance the same number of steps, then exploit-and-explore runs).
+ *
+ * Conventions
+ *   - Every function returns a pbt_status; none throws or aborts.
+ *     pbt_last_error() gives a human-readable reason for the last failure.
+ *   - "device" pointers are CUDA device addresses on the current device;
+ *     "host" pointers are ordinary host memory.  The library allocates no device
+ *     memory: the caller passes one workspace (size from pbt_query_workspace)
+ *     and the data pools, and keeps both alive until pbt_destroy.
+ *   - All work is enqueued on the stream given to pbt_create.  Calls that
+ *     return data to the host (pbt_get_*) synchronise that stream; the others
+ *     return as soon as the work is enqueued.
+ *   - There is no CPU fallback: without a CUDA device every call that would
+ *     launch work fails with PBT_ERR_CUDA.
+ *
+ * Canonical parameter order ("flat order") used by pbt_state_view: for stack 0
+ * then stack 1, for each layer l in order: W_l as [out][in] row-major, then
+ * b_l[out].  P = total count.  The toy model's flat vector is theta itself.
+ */
+#ifndef PBT_H_
+#define PBT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PBT_MAX_LAYERS 8   /* weight layers per stack */
+#define PBT_MAX_NH 8       /* hyperparameter slots per member */
+#define PBT_N_SCALARS 4    /* Adam running beta products: c1,c2 of stack 0; c1,c2 of stack 1 */
+
+typedef enum pbt_status {
+  PBT_OK = 0,
+  PBT_ERR_INVALID_ARG = 1,
+  PBT_ERR_UNSUPPORTED = 2, /* a combination the kernels do not implement (never a silent CPU path) */
+  PBT_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
+  PBT_ERR_CUDA = 4,        /* a CUDA call failed */
+  PBT_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (status word set by a kernel) */
+  PBT_ERR_STATE = 6        /* call not valid in the handle's current state */
+} pbt_status;
+
+typedef enum pbt_dtype {
+  PBT_FP64_TOY = 0,        /* toy quadratic, everything in double */
+  PBT_FP32 = 1,            /* fp32 weights, fp32 GEMMs */
+  PBT_BF16_FP32MASTER = 2  /* bf16 GEMM operands (weights shadow, activations, deltas), fp32 masters and optimiser state */
+} pbt_dtype;
+
+typedef enum pbt_model { PBT_TOY_QUADRATIC = 0, PBT_MLP = 1, PBT_GAN_PAIR = 2 } pbt_model;
+
+typedef enum pbt_loss {
+  PBT_LOSS_TOY = 0,
+  PBT_LOSS_MSE = 1,        /* mean_i sum_j (z_ij - y_ij)^2 */
+  PBT_LOSS_CE_HARD = 2,    /* softmax cross-entropy, int32 class labels */
+  PBT_LOSS_CE_SOFT = 3,    /* cross-entropy against a target distribution */
+  PBT_LOSS_GAN_LOGISTIC = 4 /* non-saturating logistic GAN losses */
+} pbt_loss;
+
+typedef enum pbt_optimizer { PBT_OPT_SGD_PLAIN = 0, PBT_OPT_SGDM = 1, PBT_OPT_ADAM = 2 } pbt_optimizer;
+
+/* exploit / explore switches ("PBT targets" ablation, Section 4.4) */
+#define PBT_COPY_WEIGHTS 1u  /* exploit copies weights and optimiser state */
+#define PBT_COPY_HPARAMS 2u  /* exploit copies the donor's hyperparameters */
+#define PBT_EXPLORE 4u       /* members that copied perturb their hyperparameters */
+
+/*
+ * Description of a population (plain data, copied by pbt_create).
+ *
+ * Networks: stack s has n_layers[s] weight layers; layer l maps
+ * widths[s][l] -> widths[s][l+1], ReLU after every layer but the last.
+ * PBT_MLP uses stack 0 only.  PBT_GAN_PAIR: stack 0 is the generator
+ * (noise -> sample), stack 1 the discriminator (sample -> one logit);
+ * widths[1][0] must equal the generator's output width.
+ * PBT_TOY_QUADRATIC: theta and h both have nh components, n_layers ignored.
+ *
+ * Hyperparameter slots: slot_* is the column of h that holds the quantity for
+ * each member, or -1 when the quantity is the same constant for everybody
+ * (const_*).  The toy model uses all nh columns as h itself.
+ */
+typedef struct pbt_spec {
+  int32_t n_members;
+  int32_t dtype;      /* pbt_dtype */
+  int32_t model;      /* pbt_model */
+  int32_t loss;       /* pbt_loss */
+  int32_t optimizer;  /* pbt_optimizer */
+  int32_t n_layers[2];
+  int32_t widths[2][PBT_MAX_LAYERS + 1];
+  int32_t batch;        /* training rows per member per update */
+  int32_t eval_batch;   /* rows of the held-out set (GAN: generated samples scored) */
+  int32_t pool_rows;    /* rows of every training pool */
+  int32_t gan_d_steps;  /* K discriminator updates per step (Section 4.3.1: 5) */
+  int32_t nh;
+  int32_t slot_lr;      /* learning rate (generator's for a GAN) */
+  int32_t slot_lr_d;    /* discriminator learning rate */
+  int32_t slot_momentum;
+  int32_t slot_beta1;
+  int32_t slot_wd;
+  uint32_t perturb_mask; /* bit k set: explore may perturb slot k */
+  uint32_t flags;        /* PBT_COPY_WEIGHTS | PBT_COPY_HPARAMS | PBT_EXPLORE */
+  int32_t trunc_num, trunc_den; /* truncation fraction, 1/5 in the paper */
+  int32_t reserved0;
+  double const_lr, const_momentum, const_beta1, const_beta2, const_eps, const_wd;
+  double toy_eta;                 /* toy step size */
+  double toy_theta0[PBT_MAX_NH];  /* toy initial theta (same for all members) */
+  double factor_lo, factor_hi;    /* perturbation factors, 0.8 / 1.2 */
+  double clamp_lo[PBT_MAX_NH], clamp_hi[PBT_MAX_NH]; /* applied after perturbation; +-inf = none */
+} pbt_spec;
+
+/*
+ * Caller-owned device data (kept by reference).  Element type of x/z/soft
+ * targets: float for PBT_FP32, bfloat16 (raw 16-bit) for PBT_BF16_FP32MASTER.
+ *   MLP : x_pool [pool_rows][in],  y_pool: MSE float [pool_rows][out],
+ *         CE_HARD int32 [pool_rows], CE_SOFT x-type [pool_rows][out];
+ *         x_eval / y_eval the same with eval_batch rows.
+ *   GAN : x_pool real samples [pool_rows][d], z_pool noise [pool_rows][zdim],
+ *         x_eval fixed evaluation noise [eval_batch][zdim]; y_* unused (NULL).
+ *   TOY : all NULL.
+ * Each (member, step) trains on the contiguous rows [off, off + batch) of the
+ * pools, off a multiple of 128 drawn from the batch stream of the counter-based
+ * generator, so the rows are reproducible from (seed, member, step).
+ */
+typedef struct pbt_data {
+  const void* x_pool;
+  const void* y_pool;
+  const void* z_pool;
+  const void* x_eval;
+  const void* y_eval;
+} pbt_data;
+
+/*
+ * Host-side view of one member's record (theta, h, p, t) plus optimiser state.
+ * Every pointer is caller-owned host memory and may be NULL to skip that part.
+ * w/opt1/opt2/grad hold P elements in flat order: float (double for the toy).
+ * `grad` (last gradient applied) is filled by pbt_get_state, ignored by set.
+ * step and round are population-wide (lockstep); setting them through any
+ * member sets them for the population.
+ */
+typedef struct pbt_state_view {
+  void* w;
+  void* opt1;       /* SGD momentum buffer, or Adam first moment */
+  void* opt2;       /* Adam second moment */
+  void* grad;
+  double* scalars;  /* [PBT_N_SCALARS] */
+  double* hparams;  /* [nh] */
+  double* fitness;  /* [1] */
+  int64_t* step;
+  int64_t* round;
+} pbt_state_view;
+
+typedef struct pbt_handle pbt_t;
+
+/* Bytes of device workspace pbt_create needs for this spec (256-byte aligned base). */
+int pbt_query_workspace(const pbt_spec* spec, size_t* bytes);
+
+/* Number of parameters P of one member in flat order. */
+int pbt_param_count(const pbt_spec* spec, int64_t* count);
+
+/*
+ * Build the initial population P (Algorithm 1, input): member-major slabs in
+ * the workspace; weights U(-a, a), a = sqrt(6 / fan_in), drawn on the device from
+ * the init stream of Philox4x32-10 keyed by `seed`; biases and optimiser state
+ * zero; h from init_hparams (host, [n_members][nh] doubles, row-major).
+ * `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ * On failure *out is NULL.
+ */
+int pbt_create(pbt_t** out, const pbt_spec* spec, const double* init_hparams, uint64_t seed,
+               const pbt_data* data, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Release the handle (host memory only; the workspace stays the caller's). */
+int pbt_destroy(pbt_t* p);
+
+/*
+ * theta <- step(theta | h) for every member, k times in lockstep (Eq. 2, chained
+ * as in Eq. 3).  MLP: forward, loss, backward, optimiser update with the member's
+ * own h.  GAN: K discriminator updates then one generator update per step
+ * (Section 4.3.1).  Toy: one gradient-ascent step on the surrogate objective.
+ */
+int pbt_step(pbt_t* p, int k);
+
+/*
+ * p <- eval(theta) for every member (Eq. 1): minus the held-out loss, the toy's
+ * true objective Q(theta), or minus the energy distance between eval_batch
+ * generated samples and the eight-mode ring.  Result stays on the device
+ * (read it with pbt_get_fitness).
+ */
+int pbt_eval(pbt_t* p);
+
+/*
+ * One ready point for the whole population (Algorithm 1: exploit, the
+ * theta != theta' guard, explore, population update): truncation selection on
+ * the current fitness vector (Section 4.1.1 (b)), slab copy donor -> recipient of
+ * weights, optimiser state and (flag) hyperparameters, perturbation of the
+ * recipients' h by factor_lo / factor_hi (Section 4.1.1 (a)), p[b] <- p[src[b]],
+ * round <- round + 1.
+ */
+int pbt_exploit_explore(pbt_t* p);
+
+/* Read / overwrite one member's record.  get synchronises the stream. */
+int pbt_get_state(pbt_t* p, int member, pbt_state_view* out_host);
+int pbt_set_state(pbt_t* p, int member, const pbt_state_view* in_host);
+
+/* fitness vector p[n_members] as doubles (host).  set allows a test to inject a
+ * fitness vector so that selection can be compared bit for bit. */
+int pbt_get_fitness(pbt_t* p, double* out_host);
+int pbt_set_fitness(pbt_t* p, const double* in_host);
+
+/* h[n_members][nh] as doubles (host). */
+int pbt_get_hparams(pbt_t* p, double* out_host);
+int pbt_set_hparams(pbt_t* p, const double* in_host);
+
+/* copy map of the last ready point: src[i] == i for members that kept their state. */
+int pbt_get_copy_map(pbt_t* p, int32_t* src_out_host);
+
+/* argmax_i p[i], lowest index on ties (Algorithm 1, return value). */
+int pbt_get_best(pbt_t* p, int32_t* member_out_host);
+
+/* per-member training loss of the last step: [n_members][2] doubles
+ * (column 0: MLP loss or generator loss; column 1: discriminator loss). */
+int pbt_get_last_loss(pbt_t* p, double* out_host);
+
+/*
+ * Use the caller's rows for the next step instead of a pool window: x is
+ * [n_members][batch][in], y the matching targets, both device pointers in the
+ * pools' element types; copied before the call returns to the stream.  MLP only.
+ */
+int pbt_set_batch(pbt_t* p, const void* x_device, const void* y_device);
+
+/* Kernel launches issued by the last pbt_step / pbt_eval / pbt_exploit_explore call. */
+int pbt_get_launch_count(const pbt_t* p, int64_t* count);
+
+/*
+ * Elapsed device time, in milliseconds, of one named kernel class accumulated
+ * since pbt_profile_begin: "gemm", "optimizer", "loss", "copy", "select".
+ * Profiling brackets each launch with events on the handle's stream and
+ * therefore slows the step down; it is off unless begun.
+ */
+int pbt_profile_begin(pbt_t* p);
+int pbt_profile_end(pbt_t* p);
+int pbt_profile_get(pbt_t* p, const char* kernel_class, double* ms_total, int64_t* launches);
+
+const char* pbt_last_error(const pbt_t* p); /* p may be NULL: error of the last failed create/query */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PBT_H_ */

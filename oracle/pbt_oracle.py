@@ -1,0 +1,559 @@
+"""Plain CPU oracle for lockstep Population Based Training -- TEST INFRASTRUCTURE.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may use
+this module; the GPU library never imports, links or calls it, and it shares
+no code with the GPU path.  It is slow on purpose: one member at a time,
+float64 arithmetic, NumPy matmul as the only library primitive, no blocking
+or fusion, so each function can be read against the passage it cites.
+
+What it follows
+---------------
+* Algorithm 1 (Section 3) in the partial-synchrony form of Appendix A.1: all
+  members take the same number of `step`s, then `eval`, then exploit/explore.
+* `step` (Eq. 2): one gradient update of the member's weights conditioned on
+  its own hyperparameters h (SGD, SGD with momentum, or Adam; Sections 4.1.1,
+  4.2.1, 4.3.1 name the optimisers, Appendix A.4 gives Adam's constants).
+* `eval` (Eq. 1): a function of the weights only -- held-out loss (negated so
+  that larger is better), the toy's true objective Q (Figure 2), or the
+  negative energy distance of generated samples to the target mixture.
+* `exploit`: truncation selection (Section 4.1.1 (b)): rank all members; each
+  member in the bottom 20 % copies a member drawn uniformly from the top 20 %.
+* `explore`: perturb (Section 4.1.1 (a)): every hyperparameter of a member
+  that copied is multiplied by 0.8 or 1.2 independently (0.5 / 2.0 in Section
+  4.3.1 are the same operator with other factors).
+* The guard of Algorithm 1 (explore and re-evaluate only when the weights
+  changed) and the population update.
+
+Readings taken where the paper is silent (each one is listed in the design
+notes of the repository): total order (fitness descending, member index
+ascending; NaN ranks last; -0 equals +0); n_cut = max(1, floor(N * 1/5));
+donor index by multiply-shift of one Philox word; one Philox bit per
+perturbed slot with probability 1/2; clamp after perturbation; optimiser state
+travels with the weights; Adam's bias correction uses running products of the
+betas actually used; bf16 populations round GEMM operands (weights shadow,
+activations, back-propagated deltas) to bfloat16 and keep masters in float32.
+
+Pins (tests/test_oracle_*.py): toy closed form and the paper's printed Q ~ 0.4
+(Figure 2 caption); brute-force enumeration of truncation selection for
+N = 2..5; donor uniformity; copy / explore / lineage invariants; member
+isolation with exploit off; finite-difference gradients; least-squares special
+case; hand-computed optimiser trajectories; energy-distance special cases;
+Philox known-answer vectors.  `Population.run` over a whole neural-network
+config has no external truth to compare with: parity unpinned beyond the pins
+of its parts.
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Optional
+
+import numpy as np
+
+from . import philox as px
+
+# flag bits and tags are re-declared here on purpose (no shared constants with
+# the GPU library)
+COPY_WEIGHTS, COPY_HPARAMS, EXPLORE = 1, 2, 4
+N_SCALARS = 4  # c1, c2 of stack 0; c1, c2 of stack 1 (Adam bias-correction products)
+MAX_LAYERS = 8
+WINDOW_ALIGN = 128
+
+
+# --------------------------------------------------------------------------
+# rounding helpers
+# --------------------------------------------------------------------------
+def round_bf16(a: np.ndarray) -> np.ndarray:
+    """float -> nearest bfloat16 (ties to even), returned as float64 values."""
+    f = np.asarray(a, dtype=np.float64).astype(np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    u = (u + np.uint64(0x7FFF) + ((u >> np.uint64(16)) & np.uint64(1))) & np.uint64(0xFFFF0000)
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(f.shape)
+
+
+def _f32(a):
+    return np.asarray(a, dtype=np.float64).astype(np.float32)
+
+
+# --------------------------------------------------------------------------
+# exploit / explore: pure functions on small arrays (Section 4.1.1)
+# --------------------------------------------------------------------------
+def n_cut_of(n: int, num: int = 1, den: int = 5) -> int:
+    """Size of the bottom and of the top set: 20 % of N, at least one, never overlapping."""
+    if n < 2:
+        return 0
+    c = max(1, (n * num) // den)
+    return min(c, n // 2)
+
+
+def rank_members(fitness) -> List[int]:
+    """Members from best to worst: fitness descending, index ascending on ties; NaN last."""
+    keyed = []
+    for i, f in enumerate(fitness):
+        f = float(f)
+        if math.isnan(f):
+            f = -math.inf
+        keyed.append((-f if f != 0.0 else 0.0, i))
+    keyed.sort()
+    return [i for _, i in keyed]
+
+
+def donor_index(word: int, n_cut: int) -> int:
+    """Uniform index in [0, n_cut) from a 32-bit word by multiply-shift."""
+    return (int(word) * int(n_cut)) >> 32
+
+
+def truncation_select(fitness, seed: int, rnd: int, num: int = 1, den: int = 5) -> np.ndarray:
+    """Copy map src[N]: src[i] == i for members that keep their state; a bottom
+    member b gets src[b] = a top member drawn uniformly (Section 4.1.1 (b))."""
+    n = len(fitness)
+    src = np.arange(n, dtype=np.int32)
+    c = n_cut_of(n, num, den)
+    if c == 0:
+        return src
+    order = rank_members(fitness)
+    top, bottom = order[:c], order[n - c:]
+    for b in bottom:
+        word = px.draw(seed, b, rnd, px.STREAM_EXPLOIT, 0)[0]
+        src[b] = top[donor_index(word, c)]
+    return src
+
+
+def explore_bits(seed: int, member: int, rnd: int, nh: int) -> List[int]:
+    """One bit per hyperparameter slot: 1 -> multiply by the high factor, 0 -> low."""
+    bits = []
+    for k in range(nh):
+        words = px.draw(seed, member, rnd, px.STREAM_EXPLORE, k >> 2)
+        bits.append((words[k & 3] >> 31) & 1)
+    return bits
+
+
+def perturb(h_row: np.ndarray, bits, mask, factor_lo, factor_hi, lo, hi) -> np.ndarray:
+    """Section 4.1.1 (a): each perturbable slot times factor_lo or factor_hi (one
+    rounding, in h's own dtype), then clamped to [lo, hi]."""
+    dt = h_row.dtype.type
+    out = h_row.copy()
+    for k in range(len(out)):
+        if not mask[k]:
+            continue
+        f = dt(factor_hi) if bits[k] else dt(factor_lo)
+        v = dt(out[k] * f)
+        v = max(v, dt(lo[k]))
+        v = min(v, dt(hi[k]))
+        out[k] = v
+    return out
+
+
+# --------------------------------------------------------------------------
+# losses (batch means) and their derivative with respect to the logits
+# --------------------------------------------------------------------------
+def softplus(x):
+    return np.maximum(x, 0.0) + np.log1p(np.exp(-np.abs(x)))
+
+
+def sigmoid(x):
+    return np.where(x >= 0, 1.0 / (1.0 + np.exp(-np.abs(x))), np.exp(-np.abs(x)) / (1.0 + np.exp(-np.abs(x))))
+
+
+def loss_mse(z, y):
+    """mean over the batch of sum_j (z_j - y_j)^2;  dL/dz = 2 (z - y) / B."""
+    b = z.shape[0]
+    d = z - y.reshape(z.shape)
+    return float((d * d).sum() / b), 2.0 * d / b
+
+
+def loss_ce_hard(z, labels):
+    """mean_i [ logsumexp(z_i) - z_i[label_i] ];  dL/dz = (softmax(z) - onehot) / B."""
+    b = z.shape[0]
+    zm = z - z.max(axis=1, keepdims=True)
+    e = np.exp(zm)
+    s = e.sum(axis=1, keepdims=True)
+    logp = zm - np.log(s)
+    idx = np.arange(b)
+    loss = float(-logp[idx, labels].sum() / b)
+    d = e / s
+    d[idx, labels] -= 1.0
+    return loss, d / b
+
+
+def loss_ce_soft(z, t):
+    """mean_i [ -sum_j t_ij log softmax(z_i)_j ];  dL/dz = (softmax(z) * sum_j t_ij - t) / B."""
+    b = z.shape[0]
+    zm = z - z.max(axis=1, keepdims=True)
+    e = np.exp(zm)
+    s = e.sum(axis=1, keepdims=True)
+    logp = zm - np.log(s)
+    loss = float(-(t * logp).sum() / b)
+    d = (e / s) * t.sum(axis=1, keepdims=True) - t
+    return loss, d / b
+
+
+def energy_distance_to_ring(x: np.ndarray, n_modes: int = 8) -> float:
+    """V-statistic energy distance between the sample x[n,2] and the equally
+    weighted modes mu_k = (cos 2 pi k/8, sin 2 pi k/8):
+        E = 2/(n K) sum_i sum_k |x_i - mu_k| - 1/n^2 sum_i sum_j |x_i - x_j|
+            - 1/K^2 sum_k sum_l |mu_k - mu_l|."""
+    x = np.asarray(x, dtype=np.float64)
+    n = x.shape[0]
+    k = np.arange(n_modes)
+    mu = np.stack([np.cos(2 * np.pi * k / n_modes), np.sin(2 * np.pi * k / n_modes)], axis=1)
+    cross = 0.0
+    for i in range(n):
+        cross += np.sqrt(((x[i] - mu) ** 2).sum(axis=1)).sum()
+    within = 0.0
+    for i in range(n):
+        within += np.sqrt(((x[i] - x) ** 2).sum(axis=1)).sum()
+    modes = 0.0
+    for a in range(n_modes):
+        modes += np.sqrt(((mu[a] - mu) ** 2).sum(axis=1)).sum()
+    return 2.0 * cross / (n * n_modes) - within / (n * n) - modes / (n_modes * n_modes)
+
+
+# --------------------------------------------------------------------------
+# optimiser updates on one tensor (float64 arithmetic; caller stores in master precision)
+# --------------------------------------------------------------------------
+def sgdm_update(theta, vel, g, lr, mu):
+    """v <- mu v + g;  theta <- theta - lr v  (no dampening, no Nesterov)."""
+    vel = mu * vel + g
+    return theta - lr * vel, vel
+
+
+def adam_update(theta, m, v, g, lr, b1, b2, eps, wd, c1, c2):
+    """m <- b1 m + (1-b1) g; v <- b2 v + (1-b2) g^2;
+    theta <- theta - lr (m/(1-c1)) / (sqrt(v/(1-c2)) + eps) - lr wd theta,
+    where c1, c2 are the running products of the betas used so far (including
+    this step); with constant betas c1 = b1^t, the textbook bias correction."""
+    m = b1 * m + (1.0 - b1) * g
+    v = b2 * v + (1.0 - b2) * g * g
+    mhat = m / (1.0 - c1)
+    vhat = v / (1.0 - c2)
+    theta = theta - lr * mhat / (np.sqrt(vhat) + eps) - lr * wd * theta
+    return theta, m, v
+
+
+# --------------------------------------------------------------------------
+# the population
+# --------------------------------------------------------------------------
+class Population:
+    """State (theta, h, p, t) of every member (Algorithm 1) plus optimiser state."""
+
+    def __init__(self, cfg, inputs, seed: Optional[int] = None):
+        self.cfg = cfg
+        self.inp = inputs
+        self.seed = int(cfg.seed if seed is None else seed)
+        self.N = cfg.n_members
+        self.toy = cfg.model == "toy_quadratic"
+        self.gan = cfg.model == "gan_pair"
+        self.bf16 = cfg.dtype == "bf16_fp32master"
+        self.master = np.float64 if self.toy else np.float32
+        self.q = round_bf16 if self.bf16 else (lambda a: np.asarray(a, dtype=np.float64))
+        self.step_count = 0
+        self.round = 0
+        self.H = np.array(inputs.init_hparams, dtype=np.float64).astype(self.master)
+        self.fitness = np.zeros(self.N, dtype=self.master)
+        self.src = np.arange(self.N, dtype=np.int32)
+        self.last_loss = np.zeros((self.N, 2), dtype=np.float64)
+        self.scalars = np.ones((self.N, N_SCALARS), dtype=np.float32)
+        # tensors[m] = list over (stack, layer) of dicts W, b
+        self.shapes = []  # (stack, layer, out, in)
+        if self.toy:
+            d = cfg.nh
+            self.theta = np.tile(np.asarray(cfg.toy_theta0, dtype=np.float64), (self.N, 1))
+            assert self.theta.shape == (self.N, d)
+        else:
+            for s, ws in enumerate(cfg.widths):
+                for l in range(len(ws) - 1):
+                    self.shapes.append((s, l, ws[l + 1], ws[l]))
+            self.W = [[None] * len(self.shapes) for _ in range(self.N)]
+            self.b = [[None] * len(self.shapes) for _ in range(self.N)]
+            for m in range(self.N):
+                for t, (s, l, fo, fi) in enumerate(self.shapes):
+                    self.W[m][t] = self._init_weight(m, s, l, fo, fi)
+                    self.b[m][t] = np.zeros(fo, dtype=np.float32)
+            z = lambda: [[np.zeros_like(x) for x in row] for row in self.W]
+            zb = lambda: [[np.zeros_like(x) for x in row] for row in self.b]
+            self.o1W, self.o1b = z(), zb()      # momentum / Adam m
+            self.o2W, self.o2b = z(), zb()      # Adam v
+            self.gW, self.gb = z(), zb()        # last gradient (for inspection)
+
+    # ----- initial weights: U(-a, a), a = sqrt(6 / fan_in), biases zero ------
+    def _init_weight(self, m, s, l, fo, fi):
+        n = fo * fi
+        blocks = np.arange((n + 3) // 4, dtype=np.uint64)
+        words = px.philox4x32_10_np(np.uint64(m), blocks, np.uint64(px.STREAM_INIT),
+                                    np.uint64(s * MAX_LAYERS + l), self.seed)
+        x = np.stack(words, axis=1).reshape(-1)[:n]
+        u = (x >> np.uint32(8)).astype(np.float32) * np.float32(2.0 ** -23) - np.float32(1.0)
+        a = np.float32(math.sqrt(6.0 / fi))
+        return (u * a).astype(np.float32).reshape(fo, fi)
+
+    # ----- helpers -----------------------------------------------------------
+    def _tensors_of_stack(self, s):
+        return [t for t, sh in enumerate(self.shapes) if sh[0] == s]
+
+    def _hp(self, m, name, default):
+        k = self.cfg.slot(name)
+        return float(self.H[m, k]) if k >= 0 else float(default)
+
+    def _window(self, m, block, word_index, pool_rows, batch):
+        """Start row of this (member, step) window: a multiple of 128 drawn from
+        the batch stream, so both sides read identical rows of the pool."""
+        n_win = (pool_rows - batch) // WINDOW_ALIGN + 1
+        w = px.draw(self.seed, m, self.step_count, px.STREAM_BATCH, block)[word_index]
+        return WINDOW_ALIGN * ((int(w) * n_win) >> 32)
+
+    # ----- network forward / backward for one member -------------------------
+    def forward(self, m, s, a0):
+        """z_l = a_{l-1} W_l^T + b_l, a_l = ReLU(z_l) on hidden layers, last layer
+        linear.  Returns (activations a_0..a_{L-1} as fed to the next GEMM, z_L)."""
+        ts = self._tensors_of_stack(s)
+        acts = [np.asarray(a0, dtype=np.float64)]
+        z = None
+        for i, t in enumerate(ts):
+            w = self.q(self.W[m][t])
+            z = acts[-1] @ w.T + self.b[m][t].astype(np.float64)
+            if i + 1 < len(ts):
+                acts.append(self.q(np.maximum(z, 0.0)))
+        return acts, z
+
+    def backward(self, m, s, acts, dz_last, need_wgrad=True, need_input_grad=False):
+        """dW_l = dZ_l^T a_{l-1};  db_l = column sums of dZ_l;
+        dZ_{l-1} = (dZ_l W_l) * [a_{l-1} > 0].  dz_last is already rounded."""
+        ts = self._tensors_of_stack(s)
+        dz = dz_last
+        gW, gb = {}, {}
+        dinput = None
+        for i in range(len(ts) - 1, -1, -1):
+            t = ts[i]
+            if need_wgrad:
+                gW[t] = dz.T @ acts[i]
+                gb[t] = dz.sum(axis=0)
+            if i > 0:
+                da = dz @ self.q(self.W[m][t])
+                dz = self.q(da * (acts[i] > 0.0))
+            elif need_input_grad:
+                dinput = self.q(dz @ self.q(self.W[m][t]))
+        return gW, gb, dinput
+
+    # ----- optimiser over the tensors of one stack ---------------------------
+    def _apply(self, m, s, gW, gb, lr):
+        cfg = self.cfg
+        ts = self._tensors_of_stack(s)
+        for t in ts:
+            self.gW[m][t] = _f32(gW[t])
+            self.gb[m][t] = _f32(gb[t])
+        if cfg.optimizer == "sgdm":
+            mu = self._hp(m, "momentum", cfg.momentum)
+            for t in ts:
+                for P, O, g in ((self.W, self.o1W, gW[t]), (self.b, self.o1b, gb[t])):
+                    # the gradient is consumed at master precision (it is stored as float32)
+                    th, vel = sgdm_update(P[m][t].astype(np.float64), O[m][t].astype(np.float64),
+                                          _f32(g).astype(np.float64), lr, mu)
+                    P[m][t], O[m][t] = _f32(th), _f32(vel)
+        elif cfg.optimizer == "adam":
+            b1 = self._hp(m, "beta1", cfg.beta1)
+            b2 = float(np.float32(cfg.beta2))
+            wd = float(np.float32(self._hp(m, "wd", cfg.weight_decay)))
+            eps = float(np.float32(cfg.eps))
+            # running products kept in float32 (they are part of the copied state)
+            c1 = np.float32(self.scalars[m, 2 * s] * np.float32(b1))
+            c2 = np.float32(self.scalars[m, 2 * s + 1] * np.float32(cfg.beta2))
+            self.scalars[m, 2 * s], self.scalars[m, 2 * s + 1] = c1, c2
+            b1 = float(np.float32(b1))
+            for t in ts:
+                for P, O1, O2, g in ((self.W, self.o1W, self.o2W, gW[t]),
+                                     (self.b, self.o1b, self.o2b, gb[t])):
+                    th, mm, vv = adam_update(P[m][t].astype(np.float64), O1[m][t].astype(np.float64),
+                                             O2[m][t].astype(np.float64), _f32(g).astype(np.float64),
+                                             lr, b1, b2, eps, wd, float(c1), float(c2))
+                    P[m][t], O1[m][t], O2[m][t] = _f32(th), _f32(mm), _f32(vv)
+        else:
+            raise ValueError(cfg.optimizer)
+
+    # ----- one `step` (Eq. 2) for one member ----------------------------------
+    def _loss_and_dz(self, z, y):
+        cfg = self.cfg
+        if cfg.loss == "mse":
+            return loss_mse(z, y.astype(np.float64))
+        if cfg.loss == "ce_hard":
+            return loss_ce_hard(z, y)
+        if cfg.loss == "ce_soft":
+            return loss_ce_soft(z, y.astype(np.float64))
+        raise ValueError(cfg.loss)
+
+    def _step_toy(self, m):
+        # ascend the surrogate 1.2 - sum_i h_i theta_i^2 (Figure 2):
+        # theta_i <- theta_i + eta * (-2 h_i theta_i), three roundings per element
+        eta = np.float64(self.cfg.toy_eta)
+        g = (np.float64(-2.0) * self.H[m]) * self.theta[m]
+        self.theta[m] = self.theta[m] + eta * g
+
+    def _step_mlp(self, m, batch=None):
+        cfg = self.cfg
+        if batch is None:
+            off = self._window(m, 0, 0, cfg.pool_rows, cfg.batch)
+            x = self.inp.x_pool[off:off + cfg.batch]
+            y = self.inp.y_pool[off:off + cfg.batch]
+        else:
+            x, y = batch
+        acts, z = self.forward(m, 0, self.q(x))
+        loss, dz = self._loss_and_dz(z, y)
+        self.last_loss[m, 0] = loss
+        gW, gb, _ = self.backward(m, 0, acts, self.q(dz))
+        self._apply(m, 0, gW, gb, self._hp(m, "lr", 0.0))
+
+    def _step_gan(self, m):
+        """Section 4.3.1: K discriminator updates, then one generator update.
+        Non-saturating logistic losses: L_D = mean softplus(-D(x)) + mean
+        softplus(D(G(z))), L_G = mean softplus(-D(G(z)))."""
+        cfg = self.cfg
+        B = cfg.batch
+        for j in range(cfg.gan_d_steps):
+            offr = self._window(m, j, 0, cfg.pool_rows, B)
+            offz = self._window(m, j, 1, cfg.pool_rows, B)
+            real = self.q(self.inp.x_pool[offr:offr + B])
+            zz = self.q(self.inp.z_pool[offz:offz + B])
+            _, gout = self.forward(m, 0, zz)
+            fake = self.q(gout)
+            acts, d = self.forward(m, 1, np.concatenate([real, fake], axis=0))
+            d = d.reshape(-1)
+            self.last_loss[m, 1] = softplus(-d[:B]).mean() + softplus(d[B:]).mean()
+            dl = np.concatenate([-sigmoid(-d[:B]), sigmoid(d[B:])]) / B
+            gW, gb, _ = self.backward(m, 1, acts, self.q(dl.reshape(-1, 1)))
+            self._apply(m, 1, gW, gb, self._hp(m, "lr_d", 0.0))
+        offz = self._window(m, cfg.gan_d_steps, 1, cfg.pool_rows, B)
+        zz = self.q(self.inp.z_pool[offz:offz + B])
+        gacts, gout = self.forward(m, 0, zz)
+        fake = self.q(gout)
+        dacts, d = self.forward(m, 1, fake)
+        d = d.reshape(-1)
+        self.last_loss[m, 0] = softplus(-d).mean()
+        dl = -sigmoid(-d) / B
+        _, _, dfake = self.backward(m, 1, dacts, self.q(dl.reshape(-1, 1)),
+                                    need_wgrad=False, need_input_grad=True)
+        gW, gb, _ = self.backward(m, 0, gacts, dfake)
+        self._apply(m, 0, gW, gb, self._hp(m, "lr", 0.0))
+
+    def step(self, k: int = 1, members=None, batch=None):
+        """k lockstep steps for all (or the given) members (Algorithm 1, line `step`)."""
+        members = range(self.N) if members is None else members
+        for _ in range(k):
+            for m in members:
+                if self.toy:
+                    self._step_toy(m)
+                elif self.gan:
+                    self._step_gan(m)
+                else:
+                    self._step_mlp(m, batch)
+            self.step_count += 1
+
+    # ----- `eval` (Eq. 1): a function of the weights only ---------------------
+    def eval_member(self, m) -> float:
+        cfg = self.cfg
+        if self.toy:
+            s = np.float64(0.0)
+            for i in range(self.theta.shape[1]):
+                s = s + self.theta[m, i] * self.theta[m, i]
+            return float(np.float64(1.2) - s)
+        if self.gan:
+            _, x = self.forward(m, 0, self.q(self.inp.x_eval))
+            return -energy_distance_to_ring(_f32(x))
+        _, z = self.forward(m, 0, self.q(self.inp.x_eval))
+        loss, _ = self._loss_and_dz(z, self.inp.y_eval)
+        return -loss
+
+    def eval(self, members=None):
+        members = range(self.N) if members is None else members
+        for m in members:
+            self.fitness[m] = self.master(self.eval_member(m))
+        return self.fitness.copy()
+
+    # ----- exploit + explore at a ready point ---------------------------------
+    def exploit_explore(self):
+        cfg = self.cfg
+        src = truncation_select(self.fitness, self.seed, self.round, cfg.trunc_num, cfg.trunc_den)
+        copied = [b for b in range(self.N) if src[b] != b]
+        for b in copied:
+            d = int(src[b])
+            if cfg.flags & COPY_WEIGHTS:
+                self._copy_member(b, d)
+            if cfg.flags & COPY_HPARAMS:
+                self.H[b] = self.H[d]
+        if cfg.flags & EXPLORE:
+            for b in copied:
+                bits = explore_bits(self.seed, b, self.round, cfg.nh)
+                self.H[b] = perturb(self.H[b], bits, cfg.perturb, cfg.factor_lo, cfg.factor_hi,
+                                    cfg.clamp_lo, cfg.clamp_hi)
+        if cfg.flags & COPY_WEIGHTS:
+            for b in copied:
+                # eval depends on the weights only, so the copy's performance is the donor's
+                self.fitness[b] = self.fitness[int(src[b])]
+        self.src = src
+        self.round += 1
+        return src
+
+    def _copy_member(self, dst, src):
+        if self.toy:
+            self.theta[dst] = self.theta[src]
+            return
+        for A in (self.W, self.b, self.o1W, self.o1b, self.o2W, self.o2b):
+            A[dst] = [x.copy() for x in A[src]]
+        self.scalars[dst] = self.scalars[src]
+
+    def best(self) -> int:
+        """Member with the highest p; the lowest index wins ties (Algorithm 1, return)."""
+        return rank_members(self.fitness)[0]
+
+    # ----- whole run in partial synchrony (Appendix A.1) ----------------------
+    def run(self, total_steps=None, on_ready=None):
+        cfg = self.cfg
+        total = cfg.total_steps if total_steps is None else total_steps
+        for _ in range(total):
+            self.step(1)
+            if self.step_count % cfg.ready_interval == 0:
+                self.eval()
+                if on_ready is not None:
+                    on_ready(self, "pre")
+                self.exploit_explore()
+                if on_ready is not None:
+                    on_ready(self, "post")
+        return self.best()
+
+    # ----- flat views in the interface order ----------------------------------
+    # Per stack, per layer: W[out][in] row-major, then b[out]; stacks in order.
+    def _flat(self, Ws, bs, m):
+        parts = []
+        for t in range(len(self.shapes)):
+            parts.append(np.asarray(Ws[m][t]).reshape(-1))
+            parts.append(np.asarray(bs[m][t]).reshape(-1))
+        return np.concatenate(parts)
+
+    def get_flat(self, m) -> Dict[str, np.ndarray]:
+        if self.toy:
+            return {"w": self.theta[m].copy()}
+        return {"w": self._flat(self.W, self.b, m), "opt1": self._flat(self.o1W, self.o1b, m),
+                "opt2": self._flat(self.o2W, self.o2b, m), "grad": self._flat(self.gW, self.gb, m),
+                "scalars": self.scalars[m].astype(np.float64)}
+
+    def set_flat(self, m, w=None, opt1=None, opt2=None, scalars=None):
+        if self.toy:
+            if w is not None:
+                self.theta[m] = np.asarray(w, dtype=np.float64)
+            return
+        for vec, Ws, bs in ((w, self.W, self.b), (opt1, self.o1W, self.o1b), (opt2, self.o2W, self.o2b)):
+            if vec is None:
+                continue
+            vec = np.asarray(vec, dtype=np.float32)
+            o = 0
+            for t, (s, l, fo, fi) in enumerate(self.shapes):
+                Ws[m][t] = vec[o:o + fo * fi].reshape(fo, fi).copy()
+                o += fo * fi
+                bs[m][t] = vec[o:o + fo].copy()
+                o += fo
+        if scalars is not None:
+            self.scalars[m] = np.asarray(scalars, dtype=np.float32)
+
+    @property
+    def n_params(self) -> int:
+        if self.toy:
+            return self.theta.shape[1]
+        return sum(fo * fi + fo for (_, _, fo, fi) in self.shapes)
