@@ -1,0 +1,384 @@
+"""ctypes binding of libpbt_b200.so: argument marshalling only.
+
+Every step of the hot path runs inside the library's CUDA kernels.  PyTorch is
+used here for device memory (the workspace and the data pools) and for the
+stream; nothing in this module computes any part of the method, and there is no
+fallback: if the shared library or a CUDA device is missing, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import math
+import os
+from typing import Dict, Optional
+
+import numpy as np
+
+PBT_MAX_LAYERS = 8
+PBT_MAX_NH = 8
+PBT_N_SCALARS = 4
+
+_DTYPE = {"fp64_toy": 0, "fp32": 1, "bf16_fp32master": 2}
+_MODEL = {"toy_quadratic": 0, "mlp": 1, "gan_pair": 2}
+_LOSS = {"toy": 0, "mse": 1, "ce_hard": 2, "ce_soft": 3, "gan_logistic": 4}
+_OPT = {"sgd_plain": 0, "sgdm": 1, "adam": 2}
+
+STATUS = {0: "PBT_OK", 1: "PBT_ERR_INVALID_ARG", 2: "PBT_ERR_UNSUPPORTED", 3: "PBT_ERR_WORKSPACE",
+          4: "PBT_ERR_CUDA", 5: "PBT_ERR_TIMEOUT", 6: "PBT_ERR_STATE"}
+
+
+class PbtSpec(C.Structure):
+    _fields_ = [
+        ("n_members", C.c_int32), ("dtype", C.c_int32), ("model", C.c_int32), ("loss", C.c_int32),
+        ("optimizer", C.c_int32), ("n_layers", C.c_int32 * 2),
+        ("widths", (C.c_int32 * (PBT_MAX_LAYERS + 1)) * 2),
+        ("batch", C.c_int32), ("eval_batch", C.c_int32), ("pool_rows", C.c_int32),
+        ("gan_d_steps", C.c_int32), ("nh", C.c_int32),
+        ("slot_lr", C.c_int32), ("slot_lr_d", C.c_int32), ("slot_momentum", C.c_int32),
+        ("slot_beta1", C.c_int32), ("slot_wd", C.c_int32),
+        ("perturb_mask", C.c_uint32), ("flags", C.c_uint32),
+        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("reserved0", C.c_int32),
+        ("const_lr", C.c_double), ("const_momentum", C.c_double), ("const_beta1", C.c_double),
+        ("const_beta2", C.c_double), ("const_eps", C.c_double), ("const_wd", C.c_double),
+        ("toy_eta", C.c_double), ("toy_theta0", C.c_double * PBT_MAX_NH),
+        ("factor_lo", C.c_double), ("factor_hi", C.c_double),
+        ("clamp_lo", C.c_double * PBT_MAX_NH), ("clamp_hi", C.c_double * PBT_MAX_NH),
+    ]
+
+
+class PbtData(C.Structure):
+    _fields_ = [("x_pool", C.c_void_p), ("y_pool", C.c_void_p), ("z_pool", C.c_void_p),
+                ("x_eval", C.c_void_p), ("y_eval", C.c_void_p)]
+
+
+class PbtStateView(C.Structure):
+    _fields_ = [("w", C.c_void_p), ("opt1", C.c_void_p), ("opt2", C.c_void_p), ("grad", C.c_void_p),
+                ("scalars", C.POINTER(C.c_double)), ("hparams", C.POINTER(C.c_double)),
+                ("fitness", C.POINTER(C.c_double)), ("step", C.POINTER(C.c_int64)),
+                ("round", C.POINTER(C.c_int64))]
+
+
+EXPORTS = [
+    "pbt_query_workspace", "pbt_param_count", "pbt_create", "pbt_destroy", "pbt_step", "pbt_eval",
+    "pbt_exploit_explore", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
+    "pbt_get_hparams", "pbt_set_hparams", "pbt_get_copy_map", "pbt_get_best", "pbt_get_last_loss",
+    "pbt_set_batch", "pbt_get_launch_count", "pbt_profile_begin", "pbt_profile_end", "pbt_profile_get",
+    "pbt_last_error",
+]
+
+_LIB = None
+
+
+def library_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libpbt_b200.so")
+
+
+def load_library() -> C.CDLL:
+    """dlopen the CUDA library; raises if it has not been built (no fallback exists)."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = library_path()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: run paper_1711_09846_b200/build.py (nvcc, sm_100a); "
+                           "there is no CPU or PyTorch fallback")
+    lib = C.CDLL(path)
+    vp = C.c_void_p
+    lib.pbt_query_workspace.argtypes = [C.POINTER(PbtSpec), C.POINTER(C.c_size_t)]
+    lib.pbt_param_count.argtypes = [C.POINTER(PbtSpec), C.POINTER(C.c_int64)]
+    lib.pbt_create.argtypes = [C.POINTER(vp), C.POINTER(PbtSpec), C.POINTER(C.c_double), C.c_uint64,
+                               C.POINTER(PbtData), vp, C.c_size_t, vp]
+    lib.pbt_destroy.argtypes = [vp]
+    lib.pbt_step.argtypes = [vp, C.c_int]
+    lib.pbt_eval.argtypes = [vp]
+    lib.pbt_exploit_explore.argtypes = [vp]
+    lib.pbt_get_state.argtypes = [vp, C.c_int, C.POINTER(PbtStateView)]
+    lib.pbt_set_state.argtypes = [vp, C.c_int, C.POINTER(PbtStateView)]
+    lib.pbt_get_fitness.argtypes = [vp, C.POINTER(C.c_double)]
+    lib.pbt_set_fitness.argtypes = [vp, C.POINTER(C.c_double)]
+    lib.pbt_get_hparams.argtypes = [vp, C.POINTER(C.c_double)]
+    lib.pbt_set_hparams.argtypes = [vp, C.POINTER(C.c_double)]
+    lib.pbt_get_copy_map.argtypes = [vp, C.POINTER(C.c_int32)]
+    lib.pbt_get_best.argtypes = [vp, C.POINTER(C.c_int32)]
+    lib.pbt_get_last_loss.argtypes = [vp, C.POINTER(C.c_double)]
+    lib.pbt_set_batch.argtypes = [vp, vp, vp]
+    lib.pbt_get_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
+    lib.pbt_profile_begin.argtypes = [vp]
+    lib.pbt_profile_end.argtypes = [vp]
+    lib.pbt_profile_get.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    lib.pbt_last_error.argtypes = [vp]
+    lib.pbt_last_error.restype = C.c_char_p
+    for name in EXPORTS:
+        if name != "pbt_last_error":
+            getattr(lib, name).restype = C.c_int
+    _LIB = lib
+    return lib
+
+
+class PbtError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"{STATUS.get(code, code)}: {msg}")
+        self.code = code
+
+
+def spec_from_config(cfg) -> PbtSpec:
+    """Translate a declarative population description (see workloads.configs.PBTConfig) into pbt_spec."""
+    s = PbtSpec()
+    s.n_members = cfg.n_members
+    s.dtype = _DTYPE[cfg.dtype]
+    s.model = _MODEL[cfg.model]
+    s.loss = _LOSS[cfg.loss]
+    s.optimizer = _OPT[cfg.optimizer]
+    if cfg.model != "toy_quadratic":
+        for k, ws in enumerate(cfg.widths):
+            s.n_layers[k] = len(ws) - 1
+            for l, w in enumerate(ws):
+                s.widths[k][l] = w
+    s.batch, s.eval_batch, s.pool_rows = cfg.batch, cfg.eval_batch, cfg.pool_rows
+    s.gan_d_steps = cfg.gan_d_steps
+    s.nh = cfg.nh
+    s.slot_lr = cfg.slot("lr")
+    s.slot_lr_d = cfg.slot("lr_d")
+    s.slot_momentum = cfg.slot("momentum")
+    s.slot_beta1 = cfg.slot("beta1")
+    s.slot_wd = cfg.slot("wd")
+    mask = 0
+    for k, on in enumerate(cfg.perturb):
+        mask |= (1 << k) if on else 0
+    s.perturb_mask = mask
+    s.flags = cfg.flags
+    s.trunc_num, s.trunc_den = cfg.trunc_num, cfg.trunc_den
+    s.const_lr = 0.0
+    s.const_momentum = cfg.momentum
+    s.const_beta1, s.const_beta2, s.const_eps, s.const_wd = cfg.beta1, cfg.beta2, cfg.eps, cfg.weight_decay
+    s.toy_eta = cfg.toy_eta
+    for k, v in enumerate(cfg.toy_theta0):
+        s.toy_theta0[k] = v
+    s.factor_lo, s.factor_hi = cfg.factor_lo, cfg.factor_hi
+    for k in range(PBT_MAX_NH):
+        s.clamp_lo[k] = cfg.clamp_lo[k] if k < len(cfg.clamp_lo) else -math.inf
+        s.clamp_hi[k] = cfg.clamp_hi[k] if k < len(cfg.clamp_hi) else math.inf
+    return s
+
+
+def param_count(cfg) -> int:
+    lib = load_library()
+    n = C.c_int64(0)
+    spec = spec_from_config(cfg)
+    rc = lib.pbt_param_count(C.byref(spec), C.byref(n))
+    if rc:
+        raise PbtError(rc, lib.pbt_last_error(None).decode())
+    return n.value
+
+
+class Population:
+    """One population living on one GPU.  Thin wrapper over the pbt_* calls."""
+
+    def __init__(self, cfg, inputs, seed: Optional[int] = None, device: str = "cuda:0"):
+        import torch
+        self._torch = torch
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: this library has no CPU path")
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.seed = int(cfg.seed if seed is None else seed)
+        self.spec = spec_from_config(cfg)
+        self.N, self.nh = cfg.n_members, cfg.nh
+        self.toy = cfg.model == "toy_quadratic"
+        torch.cuda.set_device(self.device)
+        self.stream = torch.cuda.Stream(device=self.device)
+        self._keep = []
+        data = PbtData()
+        if not self.toy:
+            op_dtype = torch.bfloat16 if cfg.dtype == "bf16_fp32master" else torch.float32
+
+            def dev(a, dtype):
+                if a is None:
+                    return None
+                t = torch.from_numpy(np.ascontiguousarray(a)).to(self.device).to(dtype).contiguous()
+                self._keep.append(t)
+                return t
+
+            ydt = {"mse": torch.float32, "ce_hard": torch.int32, "ce_soft": op_dtype}.get(cfg.loss, op_dtype)
+            self.x_pool = dev(inputs.x_pool, op_dtype)
+            self.y_pool = dev(inputs.y_pool, ydt)
+            self.z_pool = dev(inputs.z_pool, op_dtype)
+            self.x_eval = dev(inputs.x_eval, op_dtype)
+            self.y_eval = dev(inputs.y_eval, ydt)
+            for name in ("x_pool", "y_pool", "z_pool", "x_eval", "y_eval"):
+                t = getattr(self, name)
+                setattr(data, name, t.data_ptr() if t is not None else None)
+        nbytes = C.c_size_t(0)
+        self._check(self.lib.pbt_query_workspace(C.byref(self.spec), C.byref(nbytes)), None)
+        self.workspace_bytes = nbytes.value
+        self.workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        h0 = np.ascontiguousarray(inputs.init_hparams, dtype=np.float64)
+        assert h0.shape == (self.N, self.nh)
+        self.handle = C.c_void_p(None)
+        torch.cuda.synchronize(self.device)
+        rc = self.lib.pbt_create(C.byref(self.handle), C.byref(self.spec),
+                                 h0.ctypes.data_as(C.POINTER(C.c_double)), C.c_uint64(self.seed),
+                                 C.byref(data), C.c_void_p(base), C.c_size_t(nbytes.value),
+                                 C.c_void_p(self.stream.cuda_stream))
+        self._check(rc, None)
+        n = C.c_int64(0)
+        self._check(self.lib.pbt_param_count(C.byref(self.spec), C.byref(n)), None)
+        self.n_params = n.value
+
+    # ------------------------------------------------------------------
+    def _check(self, rc, handle=True):
+        if rc != 0:
+            h = self.handle if (handle and getattr(self, "handle", None)) else None
+            raise PbtError(rc, self.lib.pbt_last_error(h).decode())
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.synchronize()
+            self.lib.pbt_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def synchronize(self):
+        self.stream.synchronize()
+
+    # ----- the hot path ---------------------------------------------------
+    def step(self, k: int = 1):
+        self._check(self.lib.pbt_step(self.handle, int(k)))
+
+    def eval(self):
+        self._check(self.lib.pbt_eval(self.handle))
+
+    def exploit_explore(self):
+        self._check(self.lib.pbt_exploit_explore(self.handle))
+
+    # ----- state access ---------------------------------------------------
+    def get_state(self, m: int) -> Dict[str, np.ndarray]:
+        dt = np.float64 if self.toy else np.float32
+        P = self.n_params
+        out = {k: np.zeros(P, dtype=dt) for k in (("w",) if self.toy else ("w", "opt1", "opt2", "grad"))}
+        sc = np.zeros(PBT_N_SCALARS, dtype=np.float64)
+        hp = np.zeros(max(self.nh, 1), dtype=np.float64)
+        fit = C.c_double(0)
+        step, rnd = C.c_int64(0), C.c_int64(0)
+        v = PbtStateView()
+        for k, a in out.items():
+            setattr(v, k, a.ctypes.data)
+        v.scalars = sc.ctypes.data_as(C.POINTER(C.c_double))
+        v.hparams = hp.ctypes.data_as(C.POINTER(C.c_double))
+        v.fitness = C.pointer(fit)
+        v.step = C.pointer(step)
+        v.round = C.pointer(rnd)
+        self._check(self.lib.pbt_get_state(self.handle, int(m), C.byref(v)))
+        out.update(scalars=sc, hparams=hp[:self.nh], fitness=fit.value, step=step.value, round=rnd.value)
+        return out
+
+    def set_state(self, m: int, w=None, opt1=None, opt2=None, scalars=None, hparams=None, fitness=None,
+                  step=None, round=None):
+        dt = np.float64 if self.toy else np.float32
+        keep = []
+        v = PbtStateView()
+        for name, a in (("w", w), ("opt1", opt1), ("opt2", opt2)):
+            if a is not None:
+                a = np.ascontiguousarray(a, dtype=dt)
+                assert a.size == self.n_params
+                keep.append(a)
+                setattr(v, name, a.ctypes.data)
+        if scalars is not None:
+            a = np.ascontiguousarray(scalars, dtype=np.float64)
+            keep.append(a)
+            v.scalars = a.ctypes.data_as(C.POINTER(C.c_double))
+        if hparams is not None:
+            a = np.ascontiguousarray(hparams, dtype=np.float64)
+            keep.append(a)
+            v.hparams = a.ctypes.data_as(C.POINTER(C.c_double))
+        if fitness is not None:
+            f = C.c_double(float(fitness))
+            keep.append(f)
+            v.fitness = C.pointer(f)
+        if step is not None:
+            s_ = C.c_int64(int(step))
+            keep.append(s_)
+            v.step = C.pointer(s_)
+        if round is not None:
+            r_ = C.c_int64(int(round))
+            keep.append(r_)
+            v.round = C.pointer(r_)
+        self._check(self.lib.pbt_set_state(self.handle, int(m), C.byref(v)))
+
+    def fitness(self) -> np.ndarray:
+        f = np.zeros(self.N, dtype=np.float64)
+        self._check(self.lib.pbt_get_fitness(self.handle, f.ctypes.data_as(C.POINTER(C.c_double))))
+        return f
+
+    def set_fitness(self, f):
+        f = np.ascontiguousarray(f, dtype=np.float64)
+        assert f.shape == (self.N,)
+        self._check(self.lib.pbt_set_fitness(self.handle, f.ctypes.data_as(C.POINTER(C.c_double))))
+
+    def hparams(self) -> np.ndarray:
+        h = np.zeros((self.N, self.nh), dtype=np.float64)
+        self._check(self.lib.pbt_get_hparams(self.handle, h.ctypes.data_as(C.POINTER(C.c_double))))
+        return h
+
+    def set_hparams(self, h):
+        h = np.ascontiguousarray(h, dtype=np.float64)
+        assert h.shape == (self.N, self.nh)
+        self._check(self.lib.pbt_set_hparams(self.handle, h.ctypes.data_as(C.POINTER(C.c_double))))
+
+    def copy_map(self) -> np.ndarray:
+        s = np.zeros(self.N, dtype=np.int32)
+        self._check(self.lib.pbt_get_copy_map(self.handle, s.ctypes.data_as(C.POINTER(C.c_int32))))
+        return s
+
+    def best(self) -> int:
+        b = C.c_int32(0)
+        self._check(self.lib.pbt_get_best(self.handle, C.byref(b)))
+        return b.value
+
+    def last_loss(self) -> np.ndarray:
+        l = np.zeros((self.N, 2), dtype=np.float64)
+        self._check(self.lib.pbt_get_last_loss(self.handle, l.ctypes.data_as(C.POINTER(C.c_double))))
+        return l
+
+    def set_batch(self, x_dev, y_dev):
+        """x_dev [N, batch, in], y_dev matching targets: device tensors in the pools' dtypes."""
+        assert x_dev.is_cuda and y_dev.is_cuda and x_dev.is_contiguous() and y_dev.is_contiguous()
+        self._check(self.lib.pbt_set_batch(self.handle, C.c_void_p(x_dev.data_ptr()), C.c_void_p(y_dev.data_ptr())))
+
+    def launch_count(self) -> int:
+        n = C.c_int64(0)
+        self._check(self.lib.pbt_get_launch_count(self.handle, C.byref(n)))
+        return n.value
+
+    def profile_begin(self):
+        self._check(self.lib.pbt_profile_begin(self.handle))
+
+    def profile_end(self) -> Dict[str, Dict[str, float]]:
+        self._check(self.lib.pbt_profile_end(self.handle))
+        out = {}
+        for cls in ("gemm", "optimizer", "loss", "copy", "select", "other"):
+            ms, n = C.c_double(0), C.c_int64(0)
+            self._check(self.lib.pbt_profile_get(self.handle, cls.encode(), C.byref(ms), C.byref(n)))
+            out[cls] = {"ms": ms.value, "launches": n.value}
+        return out
+
+    # ----- Algorithm 1 in partial synchrony ---------------------------------
+    def run(self, total_steps: Optional[int] = None) -> int:
+        cfg = self.cfg
+        total = cfg.total_steps if total_steps is None else total_steps
+        done = 0
+        while done < total:
+            k = min(cfg.ready_interval, total - done)
+            self.step(k)
+            done += k
+            if done % cfg.ready_interval == 0:
+                self.eval()
+                self.exploit_explore()
+        return self.best()

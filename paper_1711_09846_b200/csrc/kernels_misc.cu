@@ -1,0 +1,411 @@
+// Small kernels of the training step: weight initialisation, batch windows,
+// losses with their logit derivatives, bias gradients, evaluation reductions,
+// the toy model.  All reductions run in a fixed order (no floating atomics), so
+// a run is bit-reproducible.
+#include "pbt_common.cuh"
+
+namespace pbt {
+
+// ---------------------------------------------------------------------------
+// Initial weights: U(-a, a) from the init stream, one Philox call per 4 elements.
+// Element idx of tensor `tensor_id` of member m uses
+// philox(seed; m, idx >> 2, init stream, tensor_id).x[idx & 3].
+// ---------------------------------------------------------------------------
+__global__ void k_init_weights(float* __restrict__ w32, long long p_pad, long long w_off, long long count,
+                               int tensor_id, float bound, uint64_t seed) {
+  const int m = blockIdx.y;
+  const long long blk = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (blk * 4 >= count) return;
+  const U4 r = philox4x32_10((uint32_t)m, (uint32_t)blk, kStreamInit, (uint32_t)tensor_id, seed);
+  float* dst = w32 + (long long)m * p_pad + w_off;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const long long idx = blk * 4 + j;
+    if (idx < count) {
+      const float u = __fsub_rn(__fmul_rn((float)(r.x[j] >> 8), 1.1920928955078125e-07f), 1.0f);
+      dst[idx] = __fmul_rn(u, bound);
+    }
+  }
+}
+
+cudaError_t launch_init_weights(float* w32, long long p_pad, int n_members, long long w_off, int fan_out,
+                                int fan_in, int tensor_id, float bound, uint64_t seed, cudaStream_t s) {
+  const long long count = (long long)fan_out * fan_in;
+  const long long blocks4 = (count + 3) / 4;
+  dim3 grid((unsigned)((blocks4 + 255) / 256), n_members);
+  k_init_weights<<<grid, 256, 0, s>>>(w32, p_pad, w_off, count, tensor_id, bound, seed);
+  return cudaGetLastError();
+}
+
+__global__ void k_f32_to_bf16(const float* __restrict__ in, bf16* __restrict__ out, long long n) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (; i < n; i += stride) out[i] = __float2bfloat16_rn(in[i]);
+}
+
+cudaError_t launch_f32_to_bf16(const float* in, bf16* out, long long n, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  long long blocks = (n + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  k_f32_to_bf16<<<(unsigned)blocks, 256, 0, s>>>(in, out, n);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// Training-batch window: rows [off, off + rows) of the pool, contiguous, so the
+// copy is a flat byte range per member.
+// ---------------------------------------------------------------------------
+__global__ void k_gather_window(char* __restrict__ dst, long long dst_stride_bytes, long long dst_offset_bytes,
+                                const char* __restrict__ pool, int row_bytes, int rows, int pool_rows, int block,
+                                int word_index, uint64_t seed, const Counters* __restrict__ counters) {
+  if (counters->use_supplied_batch) return;
+  const int m = blockIdx.y;
+  const U4 r = philox4x32_10((uint32_t)m, (uint32_t)counters->step, kStreamBatch, (uint32_t)block, seed);
+  const uint32_t n_win = (uint32_t)((pool_rows - rows) / 128 + 1);
+  const long long off = 128ll * (long long)(((uint64_t)r.x[word_index] * n_win) >> 32);
+  const long long bytes = (long long)rows * row_bytes;
+  const char* src = pool + off * row_bytes;
+  char* d = dst + (long long)m * dst_stride_bytes + dst_offset_bytes;
+  const long long n16 = bytes / 16;
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long nthreads = (long long)gridDim.x * blockDim.x;
+  if ((((uintptr_t)src | (uintptr_t)d) & 15) == 0) {
+    const int4* s4 = reinterpret_cast<const int4*>(src);
+    int4* d4 = reinterpret_cast<int4*>(d);
+    for (long long i = tid; i < n16; i += nthreads) d4[i] = __ldg(s4 + i);
+    for (long long i = n16 * 16 + tid; i < bytes; i += nthreads) d[i] = src[i];
+  } else {
+    for (long long i = tid; i < bytes; i += nthreads) d[i] = src[i];
+  }
+}
+
+cudaError_t launch_gather_window(char* dst, long long dst_stride_bytes, long long dst_offset_bytes,
+                                 const char* pool, int row_bytes, int rows, int pool_rows, int n_members,
+                                 int block, int word_index, uint64_t seed, const Counters* counters,
+                                 cudaStream_t s) {
+  const long long bytes = (long long)rows * row_bytes;
+  long long blocks = (bytes / 16 + 255) / 256;
+  if (blocks < 1) blocks = 1;
+  if (blocks > 64) blocks = 64;
+  dim3 grid((unsigned)blocks, n_members);
+  k_gather_window<<<grid, 256, 0, s>>>(dst, dst_stride_bytes, dst_offset_bytes, pool, row_bytes, rows, pool_rows,
+                                       block, word_index, seed, counters);
+  return cudaGetLastError();
+}
+
+template <typename TD>
+__global__ void k_copy_rows(TD* __restrict__ dst, long long dst_ld, long long dst_stride,
+                            const float* __restrict__ src, long long src_ld, long long src_stride, int rows,
+                            int cols) {
+  const int m = blockIdx.y;
+  const long long total = (long long)rows * cols;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / cols, c = i % cols;
+    const float v = src[m * src_stride + r * src_ld + c];
+    if constexpr (sizeof(TD) == 2) dst[m * dst_stride + r * dst_ld + c] = __float2bfloat16_rn(v);
+    else dst[m * dst_stride + r * dst_ld + c] = v;
+  }
+}
+
+cudaError_t launch_copy_rows(void* dst, int dst_dtype, long long dst_ld, long long dst_stride, const float* src,
+                             long long src_ld, long long src_stride, int rows, int cols, int n_members,
+                             cudaStream_t s) {
+  const long long total = (long long)rows * cols;
+  long long blocks = (total + 255) / 256;
+  if (blocks > 32) blocks = 32;
+  dim3 grid((unsigned)blocks, n_members);
+  if (dst_dtype == kBF16)
+    k_copy_rows<bf16><<<grid, 256, 0, s>>>((bf16*)dst, dst_ld, dst_stride, src, src_ld, src_stride, rows, cols);
+  else
+    k_copy_rows<float><<<grid, 256, 0, s>>>((float*)dst, dst_ld, dst_stride, src, src_ld, src_stride, rows, cols);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// Losses: one warp per (member, row).  Writes the row's loss and, when asked,
+// dL/dz of the batch-mean loss in the operand type.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float load_as_float(const void* p, int dtype, long long i) {
+  return dtype == kBF16 ? __bfloat162float(reinterpret_cast<const bf16*>(p)[i])
+                        : reinterpret_cast<const float*>(p)[i];
+}
+__device__ __forceinline__ void store_from_float(void* p, int dtype, long long i, float v) {
+  if (dtype == kBF16) reinterpret_cast<bf16*>(p)[i] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float*>(p)[i] = v;
+}
+__device__ __forceinline__ float softplus_f(float x) { return fmaxf(x, 0.f) + log1pf(expf(-fabsf(x))); }
+__device__ __forceinline__ float sigmoid_f(float x) {
+  const float e = expf(-fabsf(x));
+  return x >= 0.f ? 1.f / (1.f + e) : e / (1.f + e);
+}
+
+__global__ void k_loss_rows(LossArgs a) {
+  const int warps_per_block = blockDim.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int m = blockIdx.y;
+  const int row = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
+  if (row >= a.rows) return;
+  const float* z = a.logits + m * a.stride_logits + (long long)row * a.ld_logits;
+  const long long dz_base = m * a.stride_dz + (long long)row * a.ld_dz;
+  float loss = 0.f;
+  if (a.kind == PBT_LOSS_MSE) {
+    const float* y = reinterpret_cast<const float*>(a.target) + m * a.stride_target + (long long)row * a.cols;
+    float acc = 0.f;
+    for (int c = lane; c < a.cols; c += 32) {
+      const float d = z[c] - y[c];
+      acc += d * d;
+      if (a.dz) store_from_float(a.dz, a.dz_dtype, dz_base + c, 2.f * d * a.inv_batch);
+    }
+    loss = warp_sum(acc);
+  } else if (a.kind == PBT_LOSS_CE_HARD || a.kind == PBT_LOSS_CE_SOFT) {
+    float mx = -INFINITY;
+    for (int c = lane; c < a.cols; c += 32) mx = fmaxf(mx, z[c]);
+    mx = warp_max(mx);
+    float se = 0.f;
+    for (int c = lane; c < a.cols; c += 32) se += expf(z[c] - mx);
+    se = warp_sum(se);
+    const float lse = logf(se);
+    const float inv_se = 1.f / se;
+    if (a.kind == PBT_LOSS_CE_HARD) {
+      const int label = reinterpret_cast<const int*>(a.target)[m * a.stride_target + row];
+      loss = lse - (z[label] - mx);
+      if (a.dz)
+        for (int c = lane; c < a.cols; c += 32) {
+          const float p = expf(z[c] - mx) * inv_se;
+          store_from_float(a.dz, a.dz_dtype, dz_base + c, (p - (c == label ? 1.f : 0.f)) * a.inv_batch);
+        }
+    } else {
+      const long long tb = m * a.stride_target + (long long)row * a.cols;
+      float tsum = 0.f, tl = 0.f;
+      for (int c = lane; c < a.cols; c += 32) {
+        const float t = load_as_float(a.target, a.target_dtype, tb + c);
+        tsum += t;
+        tl += t * ((z[c] - mx) - lse);
+      }
+      tsum = warp_sum(tsum);
+      loss = -warp_sum(tl);
+      if (a.dz)
+        for (int c = lane; c < a.cols; c += 32) {
+          const float t = load_as_float(a.target, a.target_dtype, tb + c);
+          const float p = expf(z[c] - mx) * inv_se;
+          store_from_float(a.dz, a.dz_dtype, dz_base + c, (p * tsum - t) * a.inv_batch);
+        }
+    }
+  } else {  // PBT_LOSS_GAN_LOGISTIC: one logit per row
+    const float d = z[0];
+    const bool real = row < a.n_real_rows;
+    loss = real ? softplus_f(-d) : softplus_f(d);
+    if (a.dz && lane == 0)
+      store_from_float(a.dz, a.dz_dtype, dz_base, (real ? -sigmoid_f(-d) : sigmoid_f(d)) * a.inv_batch);
+  }
+  if (lane == 0) a.row_loss[(long long)m * a.rows + row] = loss;
+}
+
+cudaError_t launch_loss_rows(const LossArgs& a, cudaStream_t s) {
+  const int warps = 8;
+  dim3 grid((a.rows + warps - 1) / warps, a.n_members);
+  k_loss_rows<<<grid, warps * 32, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+// block-wide sum in a fixed order: thread t adds elements t, t+256, ...; then a tree over shared memory
+template <typename T>
+__device__ __forceinline__ T block_sum_256(T v, T* sh) {
+  sh[threadIdx.x] = v;
+  __syncthreads();
+#pragma unroll
+  for (int o = 128; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+    __syncthreads();
+  }
+  const T r = sh[0];
+  __syncthreads();
+  return r;
+}
+
+__global__ void k_reduce_rows(const float* __restrict__ row_loss, int rows, float scale, void* out,
+                              int out_is_double, int out_stride) {
+  __shared__ double sh[256];
+  const int m = blockIdx.x;
+  double acc = 0.0;
+  for (int r = threadIdx.x; r < rows; r += 256) acc += (double)row_loss[(long long)m * rows + r];
+  const double total = block_sum_256<double>(acc, sh);
+  if (threadIdx.x == 0) {
+    const float v = (float)total * scale;
+    if (out_is_double) reinterpret_cast<double*>(out)[(long long)m * out_stride] = (double)v;
+    else reinterpret_cast<float*>(out)[(long long)m * out_stride] = v;
+  }
+}
+
+cudaError_t launch_reduce_rows(const float* row_loss, int rows, int n_members, float scale, void* out,
+                               int out_is_double, int out_stride, cudaStream_t s) {
+  k_reduce_rows<<<n_members, 256, 0, s>>>(row_loss, rows, scale, out, out_is_double, out_stride);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// Bias gradient: column sums of dZ.  Block = 32 columns x 8 row-lanes.
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void k_bias_grad(const T* __restrict__ dz, long long ld, long long stride, int rows, int cols,
+                            float* __restrict__ out, long long out_stride) {
+  __shared__ float sh[8][33];
+  const int m = blockIdx.y;
+  const int c = blockIdx.x * 32 + threadIdx.x;
+  float acc = 0.f;
+  if (c < cols) {
+    const T* p = dz + m * stride + c;
+    for (int r = threadIdx.y; r < rows; r += 8) {
+      if constexpr (sizeof(T) == 2) acc += __bfloat162float(p[(long long)r * ld]);
+      else acc += p[(long long)r * ld];
+    }
+  }
+  sh[threadIdx.y][threadIdx.x] = acc;
+  __syncthreads();
+  if (threadIdx.y == 0 && c < cols) {
+    float t = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) t += sh[j][threadIdx.x];
+    out[m * out_stride + c] = t;
+  }
+}
+
+cudaError_t launch_bias_grad(const void* dz, int dz_dtype, long long ld, long long stride, int rows, int cols,
+                             float* out, long long out_stride, int n_members, cudaStream_t s) {
+  dim3 grid((cols + 31) / 32, n_members), block(32, 8);
+  if (dz_dtype == kBF16)
+    k_bias_grad<bf16><<<grid, block, 0, s>>>((const bf16*)dz, ld, stride, rows, cols, out, out_stride);
+  else
+    k_bias_grad<float><<<grid, block, 0, s>>>((const float*)dz, ld, stride, rows, cols, out, out_stride);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// Toy model (Figure 2): ascend 1.2 - sum_i h_i theta_i^2; evaluate 1.2 - sum_i theta_i^2.
+// Explicitly rounded operations (no fused multiply-add) so the CPU reproduces every bit.
+// ---------------------------------------------------------------------------
+__global__ void k_toy_step(double* theta, const double* __restrict__ H, int n_members, int dim, double eta) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_members * dim) return;
+  const int m = i / dim, k = i % dim;
+  const double h = H[m * PBT_MAX_NH + k];
+  const double g = __dmul_rn(__dmul_rn(-2.0, h), theta[i]);
+  theta[i] = __dadd_rn(theta[i], __dmul_rn(eta, g));
+}
+
+__global__ void k_toy_eval(const double* __restrict__ theta, double* fitness, int n_members, int dim) {
+  const int m = blockIdx.x * blockDim.x + threadIdx.x;
+  if (m >= n_members) return;
+  double s = 0.0;
+  for (int k = 0; k < dim; ++k) s = __dadd_rn(s, __dmul_rn(theta[m * dim + k], theta[m * dim + k]));
+  fitness[m] = __dsub_rn(1.2, s);
+}
+
+cudaError_t launch_toy_step(double* theta, const double* H, int n_members, int dim, double eta, cudaStream_t s) {
+  const int n = n_members * dim;
+  k_toy_step<<<(n + 127) / 128, 128, 0, s>>>(theta, H, n_members, dim, eta);
+  return cudaGetLastError();
+}
+cudaError_t launch_toy_eval(const double* theta, double* fitness, int n_members, int dim, cudaStream_t s) {
+  k_toy_eval<<<(n_members + 127) / 128, 128, 0, s>>>(theta, fitness, n_members, dim);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// Energy distance of n generated 2-D points to the eight-mode unit ring.
+// Block b of member m handles points i in [b*256, b*256+256) against all j.
+// ---------------------------------------------------------------------------
+constexpr int kEdBlock = 256;
+int energy_partial_count(int n) { return 2 * ((n + kEdBlock - 1) / kEdBlock); }
+
+__global__ void k_energy_partial(const float* __restrict__ x, long long stride, int n, double* __restrict__ partial) {
+  __shared__ float2 tile[kEdBlock];
+  __shared__ double sh[256];
+  const int m = blockIdx.y;
+  const float2* xm = reinterpret_cast<const float2*>(x + m * stride);
+  const int i = blockIdx.x * kEdBlock + threadIdx.x;
+  const bool valid = i < n;
+  const float2 xi = valid ? xm[i] : make_float2(0.f, 0.f);
+  double within = 0.0;
+  for (int j0 = 0; j0 < n; j0 += kEdBlock) {
+    const int j = j0 + threadIdx.x;
+    tile[threadIdx.x] = j < n ? xm[j] : make_float2(0.f, 0.f);
+    __syncthreads();
+    const int cnt = min(kEdBlock, n - j0);
+    float acc = 0.f;
+    for (int t = 0; t < cnt; ++t) {
+      const float dx = xi.x - tile[t].x, dy = xi.y - tile[t].y;
+      acc += sqrtf(dx * dx + dy * dy);
+    }
+    within += (double)acc;
+    __syncthreads();
+  }
+  double cross = 0.0;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    double sn, cs;
+    sincospi(k * 0.25, &sn, &cs);
+    const double dx = (double)xi.x - cs, dy = (double)xi.y - sn;
+    cross += sqrt(dx * dx + dy * dy);
+  }
+  if (!valid) { within = 0.0; cross = 0.0; }
+  const double w = block_sum_256<double>(within, sh);
+  const double c = block_sum_256<double>(cross, sh);
+  if (threadIdx.x == 0) {
+    partial[((long long)m * gridDim.x + blockIdx.x) * 2 + 0] = w;
+    partial[((long long)m * gridDim.x + blockIdx.x) * 2 + 1] = c;
+  }
+}
+
+__global__ void k_energy_final(const double* __restrict__ partial, int nblocks, int n, float* fitness) {
+  const int m = blockIdx.x * blockDim.x + threadIdx.x;
+  if (m >= (int)gridDim.x * (int)blockDim.x) return;
+  double within = 0.0, cross = 0.0;
+  for (int b = 0; b < nblocks; ++b) {
+    within += partial[((long long)m * nblocks + b) * 2 + 0];
+    cross += partial[((long long)m * nblocks + b) * 2 + 1];
+  }
+  double modes = 0.0;
+  for (int a = 0; a < 8; ++a)
+    for (int b = 0; b < 8; ++b) {
+      double sa, ca, sb, cb;
+      sincospi(a * 0.25, &sa, &ca);
+      sincospi(b * 0.25, &sb, &cb);
+      modes += sqrt((ca - cb) * (ca - cb) + (sa - sb) * (sa - sb));
+    }
+  const double e = 2.0 * cross / ((double)n * 8.0) - within / ((double)n * (double)n) - modes / 64.0;
+  fitness[m] = (float)(-e);
+}
+
+cudaError_t launch_energy_distance(const float* x, long long stride, int n, int n_members, double* partial,
+                                   float* fitness, cudaStream_t s) {
+  const int nblocks = (n + kEdBlock - 1) / kEdBlock;
+  dim3 grid(nblocks, n_members);
+  k_energy_partial<<<grid, kEdBlock, 0, s>>>(x, stride, n, partial);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  k_energy_final<<<n_members, 1, 0, s>>>(partial, nblocks, n, fitness);
+  return cudaGetLastError();
+}
+
+__global__ void k_advance_step(Counters* c) {
+  c->step += 1;
+  c->use_supplied_batch = 0;
+}
+cudaError_t launch_advance_step(Counters* c, cudaStream_t s) {
+  k_advance_step<<<1, 1, 0, s>>>(c);
+  return cudaGetLastError();
+}
+
+}  // namespace pbt

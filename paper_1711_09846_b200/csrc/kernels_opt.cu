@@ -1,0 +1,166 @@
+// Fused per-member optimiser kernels: theta <- step(theta | h) (Eq. 2), the
+// update part.  One pass over the member-major slabs; every member reads its own
+// learning rate / momentum / beta1 / weight decay from its row of H.
+//
+// HBM-bound by construction.  Adam moves, per parameter, 16 B in (master, m, v,
+// gradient) and 14 B out (master, m, v, bf16 shadow); SGD-momentum 12 B in and
+// 8 B out (+2 B shadow for bf16 populations).  All streams are accessed as
+// 16-byte vectors, two per thread per stream, fully coalesced.
+#include "pbt_common.cuh"
+
+namespace pbt {
+
+__device__ __forceinline__ float hp(const float* __restrict__ Hrow, int slot, float fallback) {
+  return slot >= 0 ? Hrow[slot] : fallback;
+}
+
+__device__ __forceinline__ float4 ld_stream(const float* p) {
+  // read-once data: bypass L1 allocation
+  float4 v;
+  asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_stream(float* p, float4 v) {
+  asm volatile("st.global.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_bf16x4(bf16* p, float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+  __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u;
+  u.x = *reinterpret_cast<uint32_t*>(&lo);
+  u.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+
+constexpr int kOptThreads = 256;
+constexpr int kOptVecPerThread = 2;                              // float4 per stream per thread per iteration
+constexpr int kOptTile = kOptThreads * kOptVecPerThread * 4;     // elements per block iteration
+
+// v <- mu v + g ; theta <- theta - lr v
+__global__ void __launch_bounds__(kOptThreads) k_sgdm(OptArgs a) {
+  const int m = blockIdx.y;
+  const float* Hrow = a.H + (long long)m * a.nh_stride;
+  const float lr = hp(Hrow, a.slot_lr, a.const_lr);
+  const float mu = hp(Hrow, a.slot_momentum, a.const_momentum);
+  const long long base = (long long)m * a.p_pad + a.begin;
+  float* w = a.w32 + base;
+  float* v = a.opt1 + base;
+  const float* g = a.grad + base;
+  bf16* w16 = a.w16 ? a.w16 + base : nullptr;
+  for (long long t0 = (long long)blockIdx.x * kOptTile; t0 < a.count; t0 += (long long)gridDim.x * kOptTile) {
+#pragma unroll
+    for (int j = 0; j < kOptVecPerThread; ++j) {
+      const long long i = t0 + ((long long)j * kOptThreads + threadIdx.x) * 4;
+      if (i < a.count) {
+        const float4 gw = ld_stream(g + i), ww = ld_stream(w + i), vv = ld_stream(v + i);
+        float4 nv, nw;
+        nv.x = __fmaf_rn(mu, vv.x, gw.x); nv.y = __fmaf_rn(mu, vv.y, gw.y);
+        nv.z = __fmaf_rn(mu, vv.z, gw.z); nv.w = __fmaf_rn(mu, vv.w, gw.w);
+        nw.x = __fmaf_rn(-lr, nv.x, ww.x); nw.y = __fmaf_rn(-lr, nv.y, ww.y);
+        nw.z = __fmaf_rn(-lr, nv.z, ww.z); nw.w = __fmaf_rn(-lr, nv.w, ww.w);
+        st_stream(v + i, nv);
+        st_stream(w + i, nw);
+        if (w16) st_bf16x4(w16 + i, nw);
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ float adam_one(float w, float& m1, float& m2, float g, float b1, float omb1, float b2,
+                                          float omb2, float inv_bc1, float inv_bc2, float lr, float eps,
+                                          float lrwd) {
+  m1 = __fmaf_rn(b1, m1, omb1 * g);
+  m2 = __fmaf_rn(b2, m2, omb2 * g * g);
+  const float mhat = m1 * inv_bc1;
+  const float vhat = m2 * inv_bc2;
+  const float upd = __fdividef(mhat, sqrtf(vhat) + eps);
+  return w - lr * upd - lrwd * w;
+}
+
+// m <- b1 m + (1-b1) g ; v <- b2 v + (1-b2) g^2 ;
+// theta <- theta - lr (m / (1-c1)) / (sqrt(v / (1-c2)) + eps) - lr wd theta,
+// c1, c2 = running products of the betas including this step.
+__global__ void __launch_bounds__(kOptThreads) k_adam(OptArgs a) {
+  const int m = blockIdx.y;
+  const float* Hrow = a.H + (long long)m * a.nh_stride;
+  const float lr = hp(Hrow, a.slot_lr, a.const_lr);
+  const float b1 = hp(Hrow, a.slot_beta1, a.const_beta1);
+  const float wd = hp(Hrow, a.slot_wd, a.const_wd);
+  const float b2 = a.const_beta2, eps = a.const_eps;
+  const float c1 = __fmul_rn(a.scalars[m * PBT_N_SCALARS + a.scalar_base + 0], b1);
+  const float c2 = __fmul_rn(a.scalars[m * PBT_N_SCALARS + a.scalar_base + 1], b2);
+  const float inv_bc1 = 1.f / (1.f - c1), inv_bc2 = 1.f / (1.f - c2);
+  const float omb1 = 1.f - b1, omb2 = 1.f - b2, lrwd = lr * wd;
+  const long long base = (long long)m * a.p_pad + a.begin;
+  float* w = a.w32 + base;
+  float* m1 = a.opt1 + base;
+  float* m2 = a.opt2 + base;
+  const float* g = a.grad + base;
+  bf16* w16 = a.w16 ? a.w16 + base : nullptr;
+  for (long long t0 = (long long)blockIdx.x * kOptTile; t0 < a.count; t0 += (long long)gridDim.x * kOptTile) {
+    float4 gw[kOptVecPerThread], ww[kOptVecPerThread], aa[kOptVecPerThread], bb[kOptVecPerThread];
+#pragma unroll
+    for (int j = 0; j < kOptVecPerThread; ++j) {
+      const long long i = t0 + ((long long)j * kOptThreads + threadIdx.x) * 4;
+      if (i < a.count) {
+        gw[j] = ld_stream(g + i); ww[j] = ld_stream(w + i);
+        aa[j] = ld_stream(m1 + i); bb[j] = ld_stream(m2 + i);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kOptVecPerThread; ++j) {
+      const long long i = t0 + ((long long)j * kOptThreads + threadIdx.x) * 4;
+      if (i < a.count) {
+        float4 nw;
+        nw.x = adam_one(ww[j].x, aa[j].x, bb[j].x, gw[j].x, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
+        nw.y = adam_one(ww[j].y, aa[j].y, bb[j].y, gw[j].y, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
+        nw.z = adam_one(ww[j].z, aa[j].z, bb[j].z, gw[j].z, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
+        nw.w = adam_one(ww[j].w, aa[j].w, bb[j].w, gw[j].w, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
+        st_stream(m1 + i, aa[j]);
+        st_stream(m2 + i, bb[j]);
+        st_stream(w + i, nw);
+        if (w16) st_bf16x4(w16 + i, nw);
+      }
+    }
+  }
+}
+
+// after the Adam pass of a stack: store the advanced beta products
+__global__ void k_adam_advance(OptArgs a) {
+  const int m = blockIdx.x * blockDim.x + threadIdx.x;
+  if (m >= a.n_members) return;
+  const float* Hrow = a.H + (long long)m * a.nh_stride;
+  const float b1 = hp(Hrow, a.slot_beta1, a.const_beta1);
+  float* sc = a.scalars + m * PBT_N_SCALARS + a.scalar_base;
+  sc[0] = __fmul_rn(sc[0], b1);
+  sc[1] = __fmul_rn(sc[1], a.const_beta2);
+}
+
+static unsigned opt_grid_x(const OptArgs& a) {
+  long long tiles = (a.count + kOptTile - 1) / kOptTile;
+  // enough blocks to fill 148 SMs several times over, but let big slabs loop
+  long long per_member = (148ll * 8 + a.n_members - 1) / a.n_members;
+  if (per_member < 1) per_member = 1;
+  if (tiles > per_member) tiles = per_member;
+  if (tiles < 1) tiles = 1;
+  return (unsigned)tiles;
+}
+
+cudaError_t launch_sgdm(const OptArgs& a, cudaStream_t s) {
+  dim3 grid(opt_grid_x(a), a.n_members);
+  k_sgdm<<<grid, kOptThreads, 0, s>>>(a);
+  return cudaGetLastError();
+}
+cudaError_t launch_adam(const OptArgs& a, cudaStream_t s) {
+  dim3 grid(opt_grid_x(a), a.n_members);
+  k_adam<<<grid, kOptThreads, 0, s>>>(a);
+  return cudaGetLastError();
+}
+cudaError_t launch_adam_advance(const OptArgs& a, cudaStream_t s) {
+  k_adam_advance<<<(a.n_members + 127) / 128, 128, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace pbt

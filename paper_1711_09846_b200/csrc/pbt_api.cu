@@ -1,0 +1,1002 @@
+// Host side of the library: the C ABI of pbt.h, the member-major layout of the
+// population in the caller's workspace, and the lockstep schedule of one
+// training step / evaluation / ready point as a sequence of kernel launches.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "pbt_common.cuh"
+
+using namespace pbt;
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+struct Layer {
+  int in, out;
+  long long w_off, b_off;  // element offsets inside a member's padded slab
+};
+struct Stack {
+  int nl;
+  Layer L[PBT_MAX_LAYERS];
+  long long begin, count;  // padded element range of the stack inside the slab
+  int rows_cap;            // rows the activation buffers can hold
+};
+
+enum KClass { kGemm = 0, kOpt, kLoss, kCopy, kSelect, kOther, kNumClasses };
+const char* const kClassNames[kNumClasses] = {"gemm", "optimizer", "loss", "copy", "select", "other"};
+
+struct ProfRec {
+  int cls;
+  cudaEvent_t a, b;
+};
+
+}  // namespace
+
+struct pbt_handle {
+  pbt_spec spec;
+  pbt_data data;
+  cudaStream_t stream;
+  uint64_t seed;
+  int N, ns, nh;
+  bool toy, gan, is_bf16;
+  int cdt;      // DType of GEMM operands
+  int esz;      // bytes of one operand element
+  long long P, P_pad;
+  Stack st[2];
+  int max_width, dz_rows_cap, rowloss_cap;
+  // device state (all inside the caller's workspace)
+  float *W32, *O1, *O2, *G;
+  bf16* W16;
+  float* scalars;
+  void* H;        // [N][PBT_MAX_NH] float (double for the toy)
+  void* fitness;  // [N] float (double for the toy)
+  int* src;
+  Counters* counters;
+  float* last_loss;  // [N][2]
+  double* theta;     // toy: [N][nh]
+  void* act[2][PBT_MAX_LAYERS];  // input of layer l of stack s: [N][rows_cap][in_l]
+  float* logits[2];              // [N][rows_cap][out_last]
+  void* dz[2];                   // ping-pong deltas [N][dz_rows_cap][max_width]
+  void* ybatch;
+  long long ybatch_stride;  // elements of the target type per member
+  float* row_loss;
+  double* ed_partial;
+  size_t workspace_bytes;
+  // bookkeeping
+  int64_t launches;
+  bool profiling;
+  std::vector<ProfRec> prof;
+  std::vector<cudaEvent_t> event_pool;
+  double prof_ms[kNumClasses];
+  int64_t prof_n[kNumClasses];
+  cudaGraphExec_t step_graph;
+  int64_t graph_nodes;  // kernels in one captured step
+  bool graph_failed;
+  char err[512];
+};
+
+namespace {
+
+int fail(pbt_t* p, int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof(buf), fmt, ap);
+  va_end(ap);
+  snprintf(g_err, sizeof(g_err), "%s", buf);
+  if (p) snprintf(p->err, sizeof(p->err), "%s", buf);
+  return code;
+}
+
+#define CU(p, expr)                                                                                   \
+  do {                                                                                                \
+    cudaError_t e_ = (expr);                                                                          \
+    if (e_ != cudaSuccess) return fail(p, PBT_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_));     \
+  } while (0)
+
+long long pad32(long long n) { return (n + 31) / 32 * 32; }
+size_t align256(size_t n) { return (n + 255) / 256 * 256; }
+
+int validate(const pbt_spec* s) {
+  if (!s) return fail(nullptr, PBT_ERR_INVALID_ARG, "spec is NULL");
+  if (s->n_members < 1 || s->n_members > 1024) return fail(nullptr, PBT_ERR_INVALID_ARG, "n_members must be in [1, 1024]");
+  if (s->nh < 0 || s->nh > PBT_MAX_NH) return fail(nullptr, PBT_ERR_INVALID_ARG, "nh must be in [0, %d]", PBT_MAX_NH);
+  if (s->trunc_num < 0 || s->trunc_den < 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "bad truncation fraction");
+  const int slots[5] = {s->slot_lr, s->slot_lr_d, s->slot_momentum, s->slot_beta1, s->slot_wd};
+  for (int i = 0; i < 5; ++i)
+    if (slots[i] < -1 || slots[i] >= s->nh) return fail(nullptr, PBT_ERR_INVALID_ARG, "hyperparameter slot out of range");
+  if (s->model == PBT_TOY_QUADRATIC) {
+    if (s->dtype != PBT_FP64_TOY) return fail(nullptr, PBT_ERR_UNSUPPORTED, "the toy model runs in fp64 only");
+    if (s->nh < 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "toy model needs nh >= 1");
+    return PBT_OK;
+  }
+  if (s->model != PBT_MLP && s->model != PBT_GAN_PAIR) return fail(nullptr, PBT_ERR_INVALID_ARG, "unknown model");
+  if (s->dtype != PBT_FP32 && s->dtype != PBT_BF16_FP32MASTER)
+    return fail(nullptr, PBT_ERR_UNSUPPORTED, "networks run in fp32 or bf16 with fp32 masters");
+  if (s->optimizer != PBT_OPT_SGDM && s->optimizer != PBT_OPT_ADAM)
+    return fail(nullptr, PBT_ERR_UNSUPPORTED, "network optimiser must be SGD-momentum or Adam");
+  const int ns = s->model == PBT_GAN_PAIR ? 2 : 1;
+  for (int k = 0; k < ns; ++k) {
+    if (s->n_layers[k] < 1 || s->n_layers[k] > PBT_MAX_LAYERS) return fail(nullptr, PBT_ERR_INVALID_ARG, "n_layers out of range");
+    for (int l = 0; l <= s->n_layers[k]; ++l)
+      if (s->widths[k][l] < 1 || s->widths[k][l] > 65536) return fail(nullptr, PBT_ERR_INVALID_ARG, "layer width out of range");
+  }
+  if (s->batch < 1 || s->eval_batch < 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "batch sizes must be positive");
+  if (s->pool_rows < s->batch) return fail(nullptr, PBT_ERR_INVALID_ARG, "pool smaller than one batch");
+  if (s->model == PBT_GAN_PAIR) {
+    if (s->loss != PBT_LOSS_GAN_LOGISTIC) return fail(nullptr, PBT_ERR_UNSUPPORTED, "GAN pairs use the logistic loss");
+    if (s->widths[1][0] != s->widths[0][s->n_layers[0]]) return fail(nullptr, PBT_ERR_INVALID_ARG, "discriminator input != generator output");
+    if (s->widths[1][s->n_layers[1]] != 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "discriminator must end in one logit");
+    if (s->widths[0][s->n_layers[0]] != 2) return fail(nullptr, PBT_ERR_UNSUPPORTED, "GAN evaluation (energy distance to the ring) is two-dimensional");
+    if (s->gan_d_steps < 1 || s->gan_d_steps > 64) return fail(nullptr, PBT_ERR_INVALID_ARG, "gan_d_steps out of range");
+    if (s->optimizer != PBT_OPT_ADAM) return fail(nullptr, PBT_ERR_UNSUPPORTED, "GAN pairs use Adam");
+  } else {
+    if (s->loss != PBT_LOSS_MSE && s->loss != PBT_LOSS_CE_HARD && s->loss != PBT_LOSS_CE_SOFT)
+      return fail(nullptr, PBT_ERR_UNSUPPORTED, "MLP loss must be MSE or cross-entropy");
+  }
+  return PBT_OK;
+}
+
+// Fills the layout-dependent fields of h and assigns workspace pointers starting at base
+// (base may be NULL: sizes only).  Returns the bytes needed.
+size_t plan(pbt_handle* h, char* base) {
+  const pbt_spec& s = h->spec;
+  h->N = s.n_members;
+  h->nh = s.nh;
+  h->toy = s.model == PBT_TOY_QUADRATIC;
+  h->gan = s.model == PBT_GAN_PAIR;
+  h->is_bf16 = s.dtype == PBT_BF16_FP32MASTER;
+  h->cdt = h->is_bf16 ? kBF16 : kF32;
+  h->esz = h->is_bf16 ? 2 : 4;
+  h->ns = h->toy ? 0 : (h->gan ? 2 : 1);
+  size_t off = 0;
+  auto take = [&](size_t bytes) -> char* {
+    char* p = base ? base + off : nullptr;
+    off += align256(bytes);
+    return p;
+  };
+  const size_t N = h->N;
+  h->counters = (Counters*)take(sizeof(Counters));
+  h->src = (int*)take(N * sizeof(int));
+  h->H = take(N * PBT_MAX_NH * sizeof(double));
+  h->fitness = take(N * sizeof(double));
+  h->last_loss = (float*)take(N * 2 * sizeof(float));
+  h->scalars = (float*)take(N * PBT_N_SCALARS * sizeof(float));
+  if (h->toy) {
+    h->P = s.nh;
+    h->P_pad = s.nh;
+    h->theta = (double*)take(N * s.nh * sizeof(double));
+    h->workspace_bytes = off;
+    return off;
+  }
+  long long p = 0, flat = 0;
+  h->max_width = 1;
+  for (int k = 0; k < h->ns; ++k) {
+    Stack& st = h->st[k];
+    st.nl = s.n_layers[k];
+    st.begin = p;
+    for (int l = 0; l < st.nl; ++l) {
+      Layer& L = st.L[l];
+      L.in = s.widths[k][l];
+      L.out = s.widths[k][l + 1];
+      L.w_off = p;
+      p += pad32((long long)L.in * L.out);
+      L.b_off = p;
+      p += pad32(L.out);
+      flat += (long long)L.in * L.out + L.out;
+      if (L.in > h->max_width) h->max_width = L.in;
+      if (L.out > h->max_width) h->max_width = L.out;
+    }
+    st.count = p - st.begin;
+  }
+  h->P = flat;
+  h->P_pad = p;
+  if (h->gan) {
+    h->st[0].rows_cap = s.batch > s.eval_batch ? s.batch : s.eval_batch;
+    h->st[1].rows_cap = 2 * s.batch;
+    h->dz_rows_cap = 2 * s.batch;
+  } else {
+    h->st[0].rows_cap = s.batch > s.eval_batch ? s.batch : s.eval_batch;
+    h->dz_rows_cap = s.batch;
+  }
+  h->rowloss_cap = h->dz_rows_cap > s.eval_batch ? h->dz_rows_cap : s.eval_batch;
+  const size_t slab = (size_t)h->P_pad * sizeof(float);
+  h->W32 = (float*)take(N * slab);
+  h->O1 = (float*)take(N * slab);
+  h->O2 = s.optimizer == PBT_OPT_ADAM ? (float*)take(N * slab) : nullptr;
+  h->G = (float*)take(N * slab);
+  h->W16 = h->is_bf16 ? (bf16*)take(N * (size_t)h->P_pad * 2) : nullptr;
+  for (int k = 0; k < h->ns; ++k) {
+    Stack& st = h->st[k];
+    for (int l = 0; l < st.nl; ++l) {
+      // layer 0 of an MLP / generator only ever holds training rows (evaluation reads the held-out set in place)
+      const int rows = (l == 0 && k == 0) ? s.batch : st.rows_cap;
+      h->act[k][l] = take(N * (size_t)rows * st.L[l].in * h->esz);
+    }
+    h->logits[k] = (float*)take(N * (size_t)st.rows_cap * st.L[st.nl - 1].out * sizeof(float));
+  }
+  for (int i = 0; i < 2; ++i) h->dz[i] = take(N * (size_t)h->dz_rows_cap * h->max_width * h->esz);
+  if (!h->gan) {
+    const int out = h->st[0].L[h->st[0].nl - 1].out;
+    if (s.loss == PBT_LOSS_MSE) h->ybatch_stride = (long long)s.batch * out;
+    else if (s.loss == PBT_LOSS_CE_HARD) h->ybatch_stride = s.batch;
+    else h->ybatch_stride = (long long)s.batch * out;
+    const size_t tsz = s.loss == PBT_LOSS_CE_SOFT ? h->esz : 4;
+    h->ybatch_stride = (h->ybatch_stride * tsz + 15) / 16 * 16 / tsz;
+    h->ybatch = take(N * (size_t)h->ybatch_stride * tsz);
+  } else {
+    h->ybatch = nullptr;
+    h->ybatch_stride = 0;
+  }
+  h->row_loss = (float*)take(N * (size_t)h->rowloss_cap * sizeof(float));
+  h->ed_partial = h->gan ? (double*)take(N * (size_t)energy_partial_count(s.eval_batch) * sizeof(double)) : nullptr;
+  h->workspace_bytes = off;
+  return off;
+}
+
+long long act_stride(const pbt_handle* h, int k, int l) {
+  const Stack& st = h->st[k];
+  const int rows = (l == 0 && k == 0) ? h->spec.batch : st.rows_cap;
+  return (long long)rows * st.L[l].in;
+}
+long long logits_stride(const pbt_handle* h, int k) {
+  const Stack& st = h->st[k];
+  return (long long)st.rows_cap * st.L[st.nl - 1].out;
+}
+long long dz_stride(const pbt_handle* h) { return (long long)h->dz_rows_cap * h->max_width; }
+
+// ----- launch bookkeeping -----------------------------------------------------
+cudaEvent_t get_event(pbt_handle* h) {
+  if (!h->event_pool.empty()) {
+    cudaEvent_t e = h->event_pool.back();
+    h->event_pool.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+struct LaunchScope {
+  pbt_handle* h;
+  int cls;
+  cudaEvent_t a, b;
+  LaunchScope(pbt_handle* h_, int cls_) : h(h_), cls(cls_), a(nullptr), b(nullptr) {
+    h->launches++;
+    if (h->profiling) {
+      a = get_event(h);
+      b = get_event(h);
+      cudaEventRecord(a, h->stream);
+    }
+  }
+  ~LaunchScope() {
+    if (h->profiling) {
+      cudaEventRecord(b, h->stream);
+      h->prof.push_back(ProfRec{cls, a, b});
+    }
+  }
+};
+
+#define LAUNCH(h, cls, expr)                                                                        \
+  do {                                                                                              \
+    cudaError_t e_;                                                                                 \
+    {                                                                                               \
+      LaunchScope scope_(h, cls);                                                                   \
+      e_ = (expr);                                                                                  \
+    }                                                                                               \
+    if (e_ != cudaSuccess) return fail(h, PBT_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_));   \
+  } while (0)
+
+int gemm(pbt_handle* h, const GemmArgs& g) {
+  if (gemm_tc_supported(g)) {
+    LAUNCH(h, kGemm, launch_gemm_tc(g, h->counters, h->stream));
+  } else {
+    LAUNCH(h, kGemm, launch_gemm_simt(g, h->stream));
+  }
+  return PBT_OK;
+}
+
+const void* weights(const pbt_handle* h, long long off) {
+  return h->is_bf16 ? (const void*)(h->W16 + off) : (const void*)(h->W32 + off);
+}
+
+// z_l = a_{l-1} W_l^T + b_l, ReLU on hidden layers; the last layer's output goes to logits[k] in fp32
+int forward(pbt_handle* h, int k, int rows, const void* in, long long in_stride) {
+  const Stack& st = h->st[k];
+  for (int l = 0; l < st.nl; ++l) {
+    const Layer& L = st.L[l];
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.M = rows; g.N = L.out; g.K = L.in; g.batch = h->N;
+    g.in_dtype = h->cdt;
+    g.A = l == 0 ? in : h->act[k][l];
+    g.lda = L.in;
+    g.strideA = l == 0 ? in_stride : act_stride(h, k, l);
+    g.B = weights(h, L.w_off); g.ldb = L.in; g.strideB = h->P_pad;
+    g.bias = h->W32 + L.b_off; g.strideBias = h->P_pad;
+    if (l + 1 < st.nl) {
+      g.C = h->act[k][l + 1]; g.ldc = L.out; g.strideC = act_stride(h, k, l + 1);
+      g.out_dtype = h->cdt; g.relu = 1;
+    } else {
+      g.C = h->logits[k]; g.ldc = L.out; g.strideC = logits_stride(h, k);
+      g.out_dtype = kF32; g.relu = 0;
+    }
+    int rc = gemm(h, g);
+    if (rc) return rc;
+  }
+  return PBT_OK;
+}
+
+// dW_l = dZ_l^T a_{l-1}, db_l = column sums of dZ_l, dZ_{l-1} = (dZ_l W_l) * [a_{l-1} > 0].
+// dZ of the last layer is in h->dz[*cur]; on return *cur names the buffer written last.
+int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride, bool need_wgrad,
+             bool need_input_grad, int* cur) {
+  const Stack& st = h->st[k];
+  const long long dzs = dz_stride(h);
+  for (int l = st.nl - 1; l >= 0; --l) {
+    const Layer& L = st.L[l];
+    const void* dz = h->dz[*cur];
+    if (need_wgrad) {
+      GemmArgs g;
+      memset(&g, 0, sizeof(g));
+      g.M = L.out; g.N = L.in; g.K = rows; g.batch = h->N;
+      g.in_dtype = h->cdt; g.out_dtype = kF32;
+      g.A = dz; g.lda = L.out; g.strideA = dzs; g.a_mn = 1;
+      g.B = l == 0 ? in : h->act[k][l]; g.ldb = L.in; g.strideB = l == 0 ? in_stride : act_stride(h, k, l); g.b_mn = 1;
+      g.C = h->G + L.w_off; g.ldc = L.in; g.strideC = h->P_pad;
+      int rc = gemm(h, g);
+      if (rc) return rc;
+      LAUNCH(h, kLoss, launch_bias_grad(dz, h->cdt, L.out, dzs, rows, L.out, h->G + L.b_off, h->P_pad, h->N, h->stream));
+    }
+    if (l > 0 || need_input_grad) {
+      GemmArgs g;
+      memset(&g, 0, sizeof(g));
+      g.M = rows; g.N = L.in; g.K = L.out; g.batch = h->N;
+      g.in_dtype = h->cdt; g.out_dtype = h->cdt;
+      g.A = dz; g.lda = L.out; g.strideA = dzs;
+      g.B = weights(h, L.w_off); g.ldb = L.in; g.strideB = h->P_pad; g.b_mn = 1;
+      g.C = h->dz[1 - *cur]; g.ldc = L.in; g.strideC = dzs;
+      if (l > 0) { g.mask = h->act[k][l]; g.ldmask = L.in; g.strideMask = act_stride(h, k, l); }
+      int rc = gemm(h, g);
+      if (rc) return rc;
+      *cur = 1 - *cur;
+    }
+  }
+  return PBT_OK;
+}
+
+int optimizer(pbt_handle* h, int k, int slot_lr, int scalar_base) {
+  const pbt_spec& s = h->spec;
+  OptArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n_members = h->N; a.p_pad = h->P_pad; a.begin = h->st[k].begin; a.count = h->st[k].count;
+  a.w32 = h->W32; a.opt1 = h->O1; a.opt2 = h->O2; a.grad = h->G; a.w16 = h->W16;
+  a.H = (const float*)h->H; a.nh_stride = PBT_MAX_NH;
+  a.slot_lr = slot_lr; a.slot_momentum = s.slot_momentum; a.slot_beta1 = s.slot_beta1; a.slot_wd = s.slot_wd;
+  a.const_lr = (float)s.const_lr; a.const_momentum = (float)s.const_momentum; a.const_beta1 = (float)s.const_beta1;
+  a.const_beta2 = (float)s.const_beta2; a.const_eps = (float)s.const_eps; a.const_wd = (float)s.const_wd;
+  a.scalars = h->scalars; a.scalar_base = scalar_base;
+  if (s.optimizer == PBT_OPT_SGDM) {
+    LAUNCH(h, kOpt, launch_sgdm(a, h->stream));
+  } else {
+    LAUNCH(h, kOpt, launch_adam(a, h->stream));
+    LAUNCH(h, kOther, launch_adam_advance(a, h->stream));
+  }
+  return PBT_OK;
+}
+
+int loss_and_dz(pbt_handle* h, int k, int rows, int n_real, const void* target, long long target_stride,
+                bool want_dz, int dz_buf, float scale, void* out, int out_stride) {
+  const pbt_spec& s = h->spec;
+  const Stack& st = h->st[k];
+  LossArgs a;
+  memset(&a, 0, sizeof(a));
+  a.kind = s.loss; a.n_members = h->N; a.rows = rows; a.cols = st.L[st.nl - 1].out;
+  a.n_real_rows = n_real; a.inv_batch = 1.0f / (float)s.batch;
+  a.logits = h->logits[k]; a.ld_logits = a.cols; a.stride_logits = logits_stride(h, k);
+  a.target = target; a.stride_target = target_stride;
+  a.target_dtype = s.loss == PBT_LOSS_CE_SOFT ? h->cdt : kF32;
+  a.dz = want_dz ? h->dz[dz_buf] : nullptr; a.dz_dtype = h->cdt; a.ld_dz = a.cols; a.stride_dz = dz_stride(h);
+  a.row_loss = h->row_loss;
+  LAUNCH(h, kLoss, launch_loss_rows(a, h->stream));
+  LAUNCH(h, kLoss, launch_reduce_rows(h->row_loss, rows, h->N, scale, out, 0, out_stride, h->stream));
+  return PBT_OK;
+}
+
+size_t target_row_bytes(const pbt_handle* h) {
+  const pbt_spec& s = h->spec;
+  const int out = h->st[0].L[h->st[0].nl - 1].out;
+  if (s.loss == PBT_LOSS_MSE) return (size_t)out * 4;
+  if (s.loss == PBT_LOSS_CE_HARD) return 4;
+  return (size_t)out * h->esz;
+}
+
+int step_mlp(pbt_handle* h) {
+  const pbt_spec& s = h->spec;
+  const Stack& st = h->st[0];
+  const int in = st.L[0].in;
+  LAUNCH(h, kCopy, launch_gather_window((char*)h->act[0][0], act_stride(h, 0, 0) * h->esz, 0, (const char*)h->data.x_pool,
+                                        in * h->esz, s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, h->stream));
+  const size_t trb = target_row_bytes(h);
+  const size_t tsz = s.loss == PBT_LOSS_CE_SOFT ? h->esz : 4;
+  LAUNCH(h, kCopy, launch_gather_window((char*)h->ybatch, h->ybatch_stride * tsz, 0, (const char*)h->data.y_pool, (int)trb,
+                                        s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, h->stream));
+  int rc = forward(h, 0, s.batch, h->act[0][0], act_stride(h, 0, 0));
+  if (rc) return rc;
+  rc = loss_and_dz(h, 0, s.batch, s.batch, h->ybatch, h->ybatch_stride, true, 0, 1.0f / s.batch, h->last_loss, 2);
+  if (rc) return rc;
+  int cur = 0;
+  rc = backward(h, 0, s.batch, h->act[0][0], act_stride(h, 0, 0), true, false, &cur);
+  if (rc) return rc;
+  return optimizer(h, 0, s.slot_lr, 0);
+}
+
+// Section 4.3.1: K discriminator updates, then one generator update.
+int step_gan(pbt_handle* h) {
+  const pbt_spec& s = h->spec;
+  const int B = s.batch;
+  const int zdim = h->st[0].L[0].in, xdim = h->st[1].L[0].in;
+  const long long d_in_stride = act_stride(h, 1, 0);
+  int rc;
+  for (int j = 0; j <= s.gan_d_steps; ++j) {
+    const bool d_phase = j < s.gan_d_steps;
+    if (d_phase)
+      LAUNCH(h, kCopy, launch_gather_window((char*)h->act[1][0], d_in_stride * h->esz, 0, (const char*)h->data.x_pool,
+                                            xdim * h->esz, B, s.pool_rows, h->N, j, 0, h->seed, h->counters, h->stream));
+    LAUNCH(h, kCopy, launch_gather_window((char*)h->act[0][0], act_stride(h, 0, 0) * h->esz, 0, (const char*)h->data.z_pool,
+                                          zdim * h->esz, B, s.pool_rows, h->N, j, 1, h->seed, h->counters, h->stream));
+    rc = forward(h, 0, B, h->act[0][0], act_stride(h, 0, 0));
+    if (rc) return rc;
+    // generated samples become discriminator input rows (after the real rows in a discriminator update)
+    char* fake_dst = (char*)h->act[1][0] + (d_phase ? (size_t)B * xdim * h->esz : 0);
+    LAUNCH(h, kCopy, launch_copy_rows(fake_dst, h->cdt, xdim, d_in_stride, h->logits[0], xdim, logits_stride(h, 0), B, xdim,
+                                      h->N, h->stream));
+    const int rows = d_phase ? 2 * B : B;
+    rc = forward(h, 1, rows, h->act[1][0], d_in_stride);
+    if (rc) return rc;
+    rc = loss_and_dz(h, 1, rows, B, nullptr, 0, true, 0, 1.0f / B, h->last_loss + (d_phase ? 1 : 0), 2);
+    if (rc) return rc;
+    int cur = 0;
+    if (d_phase) {
+      rc = backward(h, 1, rows, h->act[1][0], d_in_stride, true, false, &cur);
+      if (rc) return rc;
+      rc = optimizer(h, 1, s.slot_lr_d, 2);
+      if (rc) return rc;
+    } else {
+      rc = backward(h, 1, rows, h->act[1][0], d_in_stride, false, true, &cur);
+      if (rc) return rc;
+      rc = backward(h, 0, B, h->act[0][0], act_stride(h, 0, 0), true, false, &cur);
+      if (rc) return rc;
+      rc = optimizer(h, 0, s.slot_lr, 0);
+      if (rc) return rc;
+    }
+  }
+  return PBT_OK;
+}
+
+int one_step(pbt_handle* h) {
+  int rc;
+  if (h->toy) {
+    LAUNCH(h, kOpt, launch_toy_step(h->theta, (const double*)h->H, h->N, h->nh, h->spec.toy_eta, h->stream));
+  } else if (h->gan) {
+    rc = step_gan(h);
+    if (rc) return rc;
+  } else {
+    rc = step_mlp(h);
+    if (rc) return rc;
+  }
+  LAUNCH(h, kOther, launch_advance_step(h->counters, h->stream));
+  return PBT_OK;
+}
+
+int check_device_status(pbt_handle* h) {
+  Counters c;
+  CU(h, cudaMemcpyAsync(&c, h->counters, sizeof(c), cudaMemcpyDeviceToHost, h->stream));
+  CU(h, cudaStreamSynchronize(h->stream));
+  if (c.status != 0) return fail(h, c.status, "a kernel reported status %d (site %d)", c.status, c.status_info);
+  return PBT_OK;
+}
+
+int refresh_shadow(pbt_handle* h, int member) {
+  if (!h->is_bf16) return PBT_OK;
+  const long long off = (long long)member * h->P_pad;
+  LAUNCH(h, kOther, launch_f32_to_bf16(h->W32 + off, h->W16 + off, h->P_pad, h->stream));
+  return PBT_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------
+// C ABI
+// ------------------------------------------------------------------------------
+extern "C" {
+
+const char* pbt_last_error(const pbt_t* p) { return p ? p->err : g_err; }
+
+int pbt_query_workspace(const pbt_spec* spec, size_t* bytes) {
+  if (!bytes) return fail(nullptr, PBT_ERR_INVALID_ARG, "bytes is NULL");
+  int rc = validate(spec);
+  if (rc) return rc;
+  pbt_handle* h = new pbt_handle();
+  h->spec = *spec;
+  *bytes = plan(h, nullptr);
+  delete h;
+  return PBT_OK;
+}
+
+int pbt_param_count(const pbt_spec* spec, int64_t* count) {
+  if (!count) return fail(nullptr, PBT_ERR_INVALID_ARG, "count is NULL");
+  int rc = validate(spec);
+  if (rc) return rc;
+  pbt_handle* h = new pbt_handle();
+  h->spec = *spec;
+  plan(h, nullptr);
+  *count = h->P;
+  delete h;
+  return PBT_OK;
+}
+
+int pbt_create(pbt_t** out, const pbt_spec* spec, const double* init_hparams, uint64_t seed, const pbt_data* data,
+               void* workspace, size_t workspace_bytes, void* stream) {
+  if (!out) return fail(nullptr, PBT_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  int rc = validate(spec);
+  if (rc) return rc;
+  if (spec->nh > 0 && !init_hparams) return fail(nullptr, PBT_ERR_INVALID_ARG, "init_hparams is NULL");
+  if (spec->model != PBT_TOY_QUADRATIC) {
+    if (!data) return fail(nullptr, PBT_ERR_INVALID_ARG, "data is NULL");
+    if (!data->x_pool || !data->x_eval) return fail(nullptr, PBT_ERR_INVALID_ARG, "x_pool / x_eval missing");
+    if (spec->model == PBT_MLP && (!data->y_pool || !data->y_eval)) return fail(nullptr, PBT_ERR_INVALID_ARG, "y_pool / y_eval missing");
+    if (spec->model == PBT_GAN_PAIR && !data->z_pool) return fail(nullptr, PBT_ERR_INVALID_ARG, "z_pool missing");
+  }
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+    cudaGetLastError();
+    return fail(nullptr, PBT_ERR_CUDA, "no CUDA device: this library has no CPU path");
+  }
+  pbt_handle* h = new pbt_handle();
+  h->spec = *spec;
+  if (data) h->data = *data;
+  h->stream = (cudaStream_t)stream;
+  h->seed = seed;
+  h->step_graph = nullptr;
+  const size_t need = plan(h, nullptr);
+  if (!workspace || ((uintptr_t)workspace & 255) != 0 || workspace_bytes < need) {
+    delete h;
+    return fail(nullptr, PBT_ERR_WORKSPACE, "workspace must be 256-byte aligned and hold %zu bytes (got %zu)", need, workspace_bytes);
+  }
+  plan(h, (char*)workspace);
+  auto bail = [&](int code) {
+    snprintf(g_err, sizeof(g_err), "%s", h->err);
+    delete h;
+    return code;
+  };
+#define CREATE_CU(expr)                                                                              \
+  do {                                                                                               \
+    cudaError_t e_ = (expr);                                                                         \
+    if (e_ != cudaSuccess) { fail(h, PBT_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); return bail(PBT_ERR_CUDA); } \
+  } while (0)
+  // zero the persistent state (everything up to and including the gradient slabs); activations need no clearing
+  const size_t state_bytes = h->toy ? need : (size_t)((char*)(h->is_bf16 ? (void*)(h->W16 + (size_t)h->N * h->P_pad) : (void*)(h->G + (size_t)h->N * h->P_pad)) - (char*)workspace);
+  CREATE_CU(cudaMemsetAsync(workspace, 0, state_bytes, h->stream));
+  // hyperparameters and scalars
+  {
+    std::vector<double> Hd((size_t)h->N * PBT_MAX_NH, 0.0);
+    std::vector<float> Hf((size_t)h->N * PBT_MAX_NH, 0.f);
+    for (int m = 0; m < h->N; ++m)
+      for (int k = 0; k < h->nh; ++k) {
+        Hd[(size_t)m * PBT_MAX_NH + k] = init_hparams[(size_t)m * h->nh + k];
+        Hf[(size_t)m * PBT_MAX_NH + k] = (float)init_hparams[(size_t)m * h->nh + k];
+      }
+    if (h->toy) CREATE_CU(cudaMemcpyAsync(h->H, Hd.data(), Hd.size() * 8, cudaMemcpyHostToDevice, h->stream));
+    else CREATE_CU(cudaMemcpyAsync(h->H, Hf.data(), Hf.size() * 4, cudaMemcpyHostToDevice, h->stream));
+    std::vector<float> ones((size_t)h->N * PBT_N_SCALARS, 1.f);
+    CREATE_CU(cudaMemcpyAsync(h->scalars, ones.data(), ones.size() * 4, cudaMemcpyHostToDevice, h->stream));
+    std::vector<int> ident(h->N);
+    for (int m = 0; m < h->N; ++m) ident[m] = m;
+    CREATE_CU(cudaMemcpyAsync(h->src, ident.data(), ident.size() * 4, cudaMemcpyHostToDevice, h->stream));
+    if (h->toy) {
+      std::vector<double> th((size_t)h->N * h->nh);
+      for (int m = 0; m < h->N; ++m)
+        for (int k = 0; k < h->nh; ++k) th[(size_t)m * h->nh + k] = spec->toy_theta0[k];
+      CREATE_CU(cudaMemcpyAsync(h->theta, th.data(), th.size() * 8, cudaMemcpyHostToDevice, h->stream));
+    }
+    CREATE_CU(cudaStreamSynchronize(h->stream));  // the host vectors above go out of scope
+  }
+  if (!h->toy) {
+    for (int k = 0; k < h->ns; ++k)
+      for (int l = 0; l < h->st[k].nl; ++l) {
+        const Layer& L = h->st[k].L[l];
+        const float bound = (float)sqrt(6.0 / (double)L.in);
+        CREATE_CU(launch_init_weights(h->W32, h->P_pad, h->N, L.w_off, L.out, L.in, k * PBT_MAX_LAYERS + l, bound, seed, h->stream));
+      }
+    if (h->is_bf16) CREATE_CU(launch_f32_to_bf16(h->W32, h->W16, (long long)h->N * h->P_pad, h->stream));
+  }
+#undef CREATE_CU
+  h->err[0] = 0;
+  *out = h;
+  return PBT_OK;
+}
+
+int pbt_destroy(pbt_t* p) {
+  if (!p) return PBT_OK;
+  if (p->step_graph) cudaGraphExecDestroy(p->step_graph);
+  for (auto& r : p->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  for (auto e : p->event_pool) cudaEventDestroy(e);
+  delete p;
+  return PBT_OK;
+}
+
+int pbt_step(pbt_t* p, int k) {
+  if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  if (k < 0) return fail(p, PBT_ERR_INVALID_ARG, "k must be >= 0");
+  p->launches = 0;
+  // Small populations are launch-bound: replay one captured step as a CUDA graph.  Capture needs a
+  // non-default stream and no per-launch event records.
+  const bool want_graph = !p->profiling && !p->graph_failed && p->stream != nullptr && k > 0;
+  if (want_graph && !p->step_graph) {
+    cudaGraph_t graph = nullptr;
+    if (cudaStreamBeginCapture(p->stream, cudaStreamCaptureModeRelaxed) == cudaSuccess) {
+      const int64_t before = p->launches;
+      int rc = one_step(p);
+      cudaError_t e = cudaStreamEndCapture(p->stream, &graph);
+      p->graph_nodes = p->launches - before;
+      p->launches = before;
+      if (rc == PBT_OK && e == cudaSuccess && graph &&
+          cudaGraphInstantiate(&p->step_graph, graph, 0) == cudaSuccess) {
+        // ready
+      } else {
+        p->step_graph = nullptr;
+        p->graph_failed = true;
+        cudaGetLastError();
+      }
+      if (graph) cudaGraphDestroy(graph);
+    } else {
+      p->graph_failed = true;
+      cudaGetLastError();
+    }
+  }
+  if (want_graph && p->step_graph) {
+    for (int i = 0; i < k; ++i) CU(p, cudaGraphLaunch(p->step_graph, p->stream));
+    p->launches = (int64_t)k * p->graph_nodes;
+    return PBT_OK;
+  }
+  for (int i = 0; i < k; ++i) {
+    int rc = one_step(p);
+    if (rc) return rc;
+  }
+  return PBT_OK;
+}
+
+int pbt_eval(pbt_t* p) {
+  if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  p->launches = 0;
+  const pbt_spec& s = p->spec;
+  if (p->toy) {
+    LAUNCH(p, kLoss, launch_toy_eval(p->theta, (double*)p->fitness, p->N, p->nh, p->stream));
+    return PBT_OK;
+  }
+  int rc = forward(p, 0, s.eval_batch, p->data.x_eval, 0);
+  if (rc) return rc;
+  if (p->gan) {
+    LAUNCH(p, kLoss, launch_energy_distance(p->logits[0], logits_stride(p, 0), s.eval_batch, p->N, p->ed_partial,
+                                            (float*)p->fitness, p->stream));
+    p->launches++;  // the launcher issues two kernels
+    return PBT_OK;
+  }
+  LossArgs a;
+  memset(&a, 0, sizeof(a));
+  const Stack& st = p->st[0];
+  a.kind = s.loss; a.n_members = p->N; a.rows = s.eval_batch; a.cols = st.L[st.nl - 1].out;
+  a.n_real_rows = s.eval_batch; a.inv_batch = 1.0f / (float)s.eval_batch;
+  a.logits = p->logits[0]; a.ld_logits = a.cols; a.stride_logits = logits_stride(p, 0);
+  a.target = p->data.y_eval; a.stride_target = 0;
+  a.target_dtype = s.loss == PBT_LOSS_CE_SOFT ? p->cdt : kF32;
+  a.dz = nullptr; a.row_loss = p->row_loss;
+  LAUNCH(p, kLoss, launch_loss_rows(a, p->stream));
+  LAUNCH(p, kLoss, launch_reduce_rows(p->row_loss, s.eval_batch, p->N, -1.0f / (float)s.eval_batch, p->fitness, 0, 1, p->stream));
+  return PBT_OK;
+}
+
+int pbt_exploit_explore(pbt_t* p) {
+  if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  p->launches = 0;
+  const pbt_spec& s = p->spec;
+  SelectArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n = p->N; a.nh = p->nh;
+  int n_cut = 0;
+  if (p->N >= 2) {
+    long long c = ((long long)p->N * s.trunc_num) / s.trunc_den;
+    if (c < 1) c = 1;
+    if (c > p->N / 2) c = p->N / 2;
+    n_cut = (int)c;
+  }
+  a.n_cut = n_cut;
+  a.h_is_double = p->toy ? 1 : 0;
+  a.H = p->H; a.fitness = p->fitness; a.src = p->src; a.counters = p->counters; a.seed = p->seed;
+  a.perturb_mask = s.perturb_mask; a.flags = s.flags;
+  a.factor_lo = s.factor_lo; a.factor_hi = s.factor_hi;
+  for (int k = 0; k < PBT_MAX_NH; ++k) { a.clamp_lo[k] = s.clamp_lo[k]; a.clamp_hi[k] = s.clamp_hi[k]; }
+  LAUNCH(p, kSelect, launch_select_explore(a, p->stream));
+  if (!(s.flags & PBT_COPY_WEIGHTS) || n_cut == 0) return PBT_OK;
+  CopyArgs c;
+  memset(&c, 0, sizeof(c));
+  c.n = p->N; c.src = p->src;
+  auto add = [&](void* base, long long stride, long long bytes) {
+    if (!base) return;
+    c.base[c.n_arrays] = (char*)base; c.stride_bytes[c.n_arrays] = stride; c.copy_bytes[c.n_arrays] = bytes;
+    c.n_arrays++;
+  };
+  if (p->toy) {
+    // nh doubles per member: tiny, and not a multiple of 16 bytes in general -> dedicated path below
+    LAUNCH(p, kCopy, launch_copy_small((char*)p->theta, (long long)p->nh * 8, p->src, p->N, p->stream));
+    return PBT_OK;
+  }
+  const long long slab = p->P_pad * 4;
+  add(p->W32, slab, slab);
+  add(p->O1, slab, slab);
+  add(p->O2, slab, slab);
+  add(p->W16, p->P_pad * 2, p->P_pad * 2);
+  add(p->scalars, PBT_N_SCALARS * 4, PBT_N_SCALARS * 4);
+  LAUNCH(p, kCopy, launch_slab_copy(c, p->stream));
+  return PBT_OK;
+}
+
+int pbt_get_state(pbt_t* p, int member, pbt_state_view* v) {
+  if (!p || !v) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  if (member < 0 || member >= p->N) return fail(p, PBT_ERR_INVALID_ARG, "member out of range");
+  std::vector<float> sc(PBT_N_SCALARS);
+  Counters c;
+  if (p->toy) {
+    if (v->w) CU(p, cudaMemcpyAsync(v->w, p->theta + (size_t)member * p->nh, p->nh * 8, cudaMemcpyDeviceToHost, p->stream));
+  } else {
+    struct { void* host; const float* dev; } parts[4] = {{v->w, p->W32}, {v->opt1, p->O1}, {v->opt2, p->O2}, {v->grad, p->G}};
+    for (auto& part : parts) {
+      if (!part.host) continue;
+      float* dst = (float*)part.host;
+      if (!part.dev) {  // no second moment for SGD-momentum: report zeros
+        memset(dst, 0, (size_t)p->P * 4);
+        continue;
+      }
+      const float* slab = part.dev + (size_t)member * p->P_pad;
+      for (int k = 0; k < p->ns; ++k)
+        for (int l = 0; l < p->st[k].nl; ++l) {
+          const Layer& L = p->st[k].L[l];
+          const size_t nw = (size_t)L.in * L.out;
+          CU(p, cudaMemcpyAsync(dst, slab + L.w_off, nw * 4, cudaMemcpyDeviceToHost, p->stream));
+          dst += nw;
+          CU(p, cudaMemcpyAsync(dst, slab + L.b_off, (size_t)L.out * 4, cudaMemcpyDeviceToHost, p->stream));
+          dst += L.out;
+        }
+    }
+  }
+  CU(p, cudaMemcpyAsync(sc.data(), p->scalars + (size_t)member * PBT_N_SCALARS, PBT_N_SCALARS * 4, cudaMemcpyDeviceToHost, p->stream));
+  CU(p, cudaMemcpyAsync(&c, p->counters, sizeof(c), cudaMemcpyDeviceToHost, p->stream));
+  double hd[PBT_MAX_NH];
+  float hf[PBT_MAX_NH];
+  double fd = 0;
+  float ff = 0;
+  if (p->toy) {
+    CU(p, cudaMemcpyAsync(hd, (double*)p->H + (size_t)member * PBT_MAX_NH, sizeof(hd), cudaMemcpyDeviceToHost, p->stream));
+    CU(p, cudaMemcpyAsync(&fd, (double*)p->fitness + member, 8, cudaMemcpyDeviceToHost, p->stream));
+  } else {
+    CU(p, cudaMemcpyAsync(hf, (float*)p->H + (size_t)member * PBT_MAX_NH, sizeof(hf), cudaMemcpyDeviceToHost, p->stream));
+    CU(p, cudaMemcpyAsync(&ff, (float*)p->fitness + member, 4, cudaMemcpyDeviceToHost, p->stream));
+  }
+  CU(p, cudaStreamSynchronize(p->stream));
+  if (c.status != 0) return fail(p, c.status, "a kernel reported status %d (site %d)", c.status, c.status_info);
+  if (v->scalars) for (int i = 0; i < PBT_N_SCALARS; ++i) v->scalars[i] = sc[i];
+  if (v->hparams) for (int k = 0; k < p->nh; ++k) v->hparams[k] = p->toy ? hd[k] : (double)hf[k];
+  if (v->fitness) *v->fitness = p->toy ? fd : (double)ff;
+  if (v->step) *v->step = c.step;
+  if (v->round) *v->round = c.round;
+  return PBT_OK;
+}
+
+int pbt_set_state(pbt_t* p, int member, const pbt_state_view* v) {
+  if (!p || !v) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  if (member < 0 || member >= p->N) return fail(p, PBT_ERR_INVALID_ARG, "member out of range");
+  if (p->toy) {
+    if (v->w) CU(p, cudaMemcpyAsync(p->theta + (size_t)member * p->nh, v->w, p->nh * 8, cudaMemcpyHostToDevice, p->stream));
+  } else {
+    struct { const void* host; float* dev; } parts[3] = {{v->w, p->W32}, {v->opt1, p->O1}, {v->opt2, p->O2}};
+    for (auto& part : parts) {
+      if (!part.host || !part.dev) continue;
+      const float* srcp = (const float*)part.host;
+      float* slab = part.dev + (size_t)member * p->P_pad;
+      for (int k = 0; k < p->ns; ++k)
+        for (int l = 0; l < p->st[k].nl; ++l) {
+          const Layer& L = p->st[k].L[l];
+          const size_t nw = (size_t)L.in * L.out;
+          CU(p, cudaMemcpyAsync(slab + L.w_off, srcp, nw * 4, cudaMemcpyHostToDevice, p->stream));
+          srcp += nw;
+          CU(p, cudaMemcpyAsync(slab + L.b_off, srcp, (size_t)L.out * 4, cudaMemcpyHostToDevice, p->stream));
+          srcp += L.out;
+        }
+    }
+    if (v->w) {
+      int rc = refresh_shadow(p, member);
+      if (rc) return rc;
+    }
+  }
+  float sc[PBT_N_SCALARS];
+  if (v->scalars) {
+    for (int i = 0; i < PBT_N_SCALARS; ++i) sc[i] = (float)v->scalars[i];
+    CU(p, cudaMemcpyAsync(p->scalars + (size_t)member * PBT_N_SCALARS, sc, sizeof(sc), cudaMemcpyHostToDevice, p->stream));
+  }
+  double hd[PBT_MAX_NH] = {0};
+  float hf[PBT_MAX_NH] = {0};
+  if (v->hparams) {
+    for (int k = 0; k < p->nh; ++k) { hd[k] = v->hparams[k]; hf[k] = (float)v->hparams[k]; }
+    if (p->toy) CU(p, cudaMemcpyAsync((double*)p->H + (size_t)member * PBT_MAX_NH, hd, sizeof(hd), cudaMemcpyHostToDevice, p->stream));
+    else CU(p, cudaMemcpyAsync((float*)p->H + (size_t)member * PBT_MAX_NH, hf, sizeof(hf), cudaMemcpyHostToDevice, p->stream));
+  }
+  double fd = 0;
+  float ff = 0;
+  if (v->fitness) {
+    fd = *v->fitness; ff = (float)fd;
+    if (p->toy) CU(p, cudaMemcpyAsync((double*)p->fitness + member, &fd, 8, cudaMemcpyHostToDevice, p->stream));
+    else CU(p, cudaMemcpyAsync((float*)p->fitness + member, &ff, 4, cudaMemcpyHostToDevice, p->stream));
+  }
+  long long st = 0, rd = 0;
+  if (v->step) { st = *v->step; CU(p, cudaMemcpyAsync(&p->counters->step, &st, 8, cudaMemcpyHostToDevice, p->stream)); }
+  if (v->round) { rd = *v->round; CU(p, cudaMemcpyAsync(&p->counters->round, &rd, 8, cudaMemcpyHostToDevice, p->stream)); }
+  CU(p, cudaStreamSynchronize(p->stream));  // host staging above lives on this frame
+  return PBT_OK;
+}
+
+int pbt_get_fitness(pbt_t* p, double* out) {
+  if (!p || !out) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  if (p->toy) {
+    CU(p, cudaMemcpyAsync(out, p->fitness, (size_t)p->N * 8, cudaMemcpyDeviceToHost, p->stream));
+    CU(p, cudaStreamSynchronize(p->stream));
+  } else {
+    std::vector<float> f(p->N);
+    CU(p, cudaMemcpyAsync(f.data(), p->fitness, (size_t)p->N * 4, cudaMemcpyDeviceToHost, p->stream));
+    CU(p, cudaStreamSynchronize(p->stream));
+    for (int i = 0; i < p->N; ++i) out[i] = f[i];
+  }
+  return check_device_status(p);
+}
+
+int pbt_set_fitness(pbt_t* p, const double* in) {
+  if (!p || !in) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  if (p->toy) {
+    CU(p, cudaMemcpyAsync(p->fitness, in, (size_t)p->N * 8, cudaMemcpyHostToDevice, p->stream));
+    CU(p, cudaStreamSynchronize(p->stream));
+  } else {
+    std::vector<float> f(p->N);
+    for (int i = 0; i < p->N; ++i) f[i] = (float)in[i];
+    CU(p, cudaMemcpyAsync(p->fitness, f.data(), (size_t)p->N * 4, cudaMemcpyHostToDevice, p->stream));
+    CU(p, cudaStreamSynchronize(p->stream));
+  }
+  return PBT_OK;
+}
+
+int pbt_get_hparams(pbt_t* p, double* out) {
+  if (!p || !out) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  const size_t n = (size_t)p->N * PBT_MAX_NH;
+  if (p->toy) {
+    std::vector<double> hbuf(n);
+    CU(p, cudaMemcpyAsync(hbuf.data(), p->H, n * 8, cudaMemcpyDeviceToHost, p->stream));
+    CU(p, cudaStreamSynchronize(p->stream));
+    for (int m = 0; m < p->N; ++m) for (int k = 0; k < p->nh; ++k) out[(size_t)m * p->nh + k] = hbuf[(size_t)m * PBT_MAX_NH + k];
+  } else {
+    std::vector<float> hbuf(n);
+    CU(p, cudaMemcpyAsync(hbuf.data(), p->H, n * 4, cudaMemcpyDeviceToHost, p->stream));
+    CU(p, cudaStreamSynchronize(p->stream));
+    for (int m = 0; m < p->N; ++m) for (int k = 0; k < p->nh; ++k) out[(size_t)m * p->nh + k] = hbuf[(size_t)m * PBT_MAX_NH + k];
+  }
+  return PBT_OK;
+}
+
+int pbt_set_hparams(pbt_t* p, const double* in) {
+  if (!p || !in) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  const size_t n = (size_t)p->N * PBT_MAX_NH;
+  std::vector<double> hd(n, 0.0);
+  std::vector<float> hf(n, 0.f);
+  for (int m = 0; m < p->N; ++m)
+    for (int k = 0; k < p->nh; ++k) {
+      hd[(size_t)m * PBT_MAX_NH + k] = in[(size_t)m * p->nh + k];
+      hf[(size_t)m * PBT_MAX_NH + k] = (float)in[(size_t)m * p->nh + k];
+    }
+  if (p->toy) CU(p, cudaMemcpyAsync(p->H, hd.data(), n * 8, cudaMemcpyHostToDevice, p->stream));
+  else CU(p, cudaMemcpyAsync(p->H, hf.data(), n * 4, cudaMemcpyHostToDevice, p->stream));
+  CU(p, cudaStreamSynchronize(p->stream));
+  return PBT_OK;
+}
+
+int pbt_get_copy_map(pbt_t* p, int32_t* out) {
+  if (!p || !out) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  CU(p, cudaMemcpyAsync(out, p->src, (size_t)p->N * 4, cudaMemcpyDeviceToHost, p->stream));
+  CU(p, cudaStreamSynchronize(p->stream));
+  return PBT_OK;
+}
+
+int pbt_get_best(pbt_t* p, int32_t* member) {
+  if (!p || !member) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  std::vector<double> f(p->N);
+  int rc = pbt_get_fitness(p, f.data());
+  if (rc) return rc;
+  int best = 0;
+  double bf = f[0] != f[0] ? -INFINITY : f[0];
+  for (int i = 1; i < p->N; ++i) {
+    const double v = f[i] != f[i] ? -INFINITY : f[i];
+    if (v > bf) { bf = v; best = i; }
+  }
+  *member = best;
+  return PBT_OK;
+}
+
+int pbt_get_last_loss(pbt_t* p, double* out) {
+  if (!p || !out) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  std::vector<float> f((size_t)p->N * 2);
+  CU(p, cudaMemcpyAsync(f.data(), p->last_loss, f.size() * 4, cudaMemcpyDeviceToHost, p->stream));
+  CU(p, cudaStreamSynchronize(p->stream));
+  for (size_t i = 0; i < f.size(); ++i) out[i] = f[i];
+  return PBT_OK;
+}
+
+int pbt_set_batch(pbt_t* p, const void* x, const void* y) {
+  if (!p || !x || !y) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  if (p->toy || p->gan) return fail(p, PBT_ERR_UNSUPPORTED, "caller-supplied batches are for MLP populations");
+  const pbt_spec& s = p->spec;
+  const size_t xb = (size_t)p->N * s.batch * p->st[0].L[0].in * p->esz;
+  CU(p, cudaMemcpyAsync(p->act[0][0], x, xb, cudaMemcpyDeviceToDevice, p->stream));
+  const size_t trb = target_row_bytes(p) * s.batch;
+  const size_t tsz = s.loss == PBT_LOSS_CE_SOFT ? p->esz : 4;
+  CU(p, cudaMemcpy2DAsync(p->ybatch, p->ybatch_stride * tsz, y, trb, trb, p->N, cudaMemcpyDeviceToDevice, p->stream));
+  const int one = 1;
+  CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &one, 4, cudaMemcpyHostToDevice, p->stream));
+  CU(p, cudaStreamSynchronize(p->stream));
+  return PBT_OK;
+}
+
+int pbt_get_launch_count(const pbt_t* p, int64_t* count) {
+  if (!p || !count) return fail(nullptr, PBT_ERR_INVALID_ARG, "NULL argument");
+  *count = p->launches;
+  return PBT_OK;
+}
+
+int pbt_profile_begin(pbt_t* p) {
+  if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  for (auto& r : p->prof) { p->event_pool.push_back(r.a); p->event_pool.push_back(r.b); }
+  p->prof.clear();
+  for (int i = 0; i < kNumClasses; ++i) { p->prof_ms[i] = 0; p->prof_n[i] = 0; }
+  p->profiling = true;
+  return PBT_OK;
+}
+
+int pbt_profile_end(pbt_t* p) {
+  if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  p->profiling = false;
+  CU(p, cudaStreamSynchronize(p->stream));
+  for (auto& r : p->prof) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) { p->prof_ms[r.cls] += ms; p->prof_n[r.cls] += 1; }
+    p->event_pool.push_back(r.a);
+    p->event_pool.push_back(r.b);
+  }
+  p->prof.clear();
+  return PBT_OK;
+}
+
+int pbt_profile_get(pbt_t* p, const char* kernel_class, double* ms_total, int64_t* launches) {
+  if (!p || !kernel_class) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  for (int i = 0; i < kNumClasses; ++i)
+    if (strcmp(kernel_class, kClassNames[i]) == 0) {
+      if (ms_total) *ms_total = p->prof_ms[i];
+      if (launches) *launches = p->prof_n[i];
+      return PBT_OK;
+    }
+  return fail(p, PBT_ERR_INVALID_ARG, "unknown kernel class '%s'", kernel_class);
+}
+
+}  // extern "C"

@@ -1,0 +1,163 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pbt.h"
+
+namespace pbt {
+
+typedef __nv_bfloat16 bf16;
+
+// ---------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11, Section 3.3), device + host.
+// counter = (member, round_or_step, stream, block), key = (seed_lo, seed_hi)
+// ---------------------------------------------------------------------------
+enum PhiloxStream : uint32_t { kStreamExploit = 0, kStreamExplore = 1, kStreamBatch = 2, kStreamInit = 3 };
+
+struct U4 {
+  uint32_t x[4];
+};
+
+__host__ __device__ inline U4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint64_t seed) {
+  const uint32_t kM0 = 0xD2511F53u, kM1 = 0xCD9E8D57u, kW0 = 0x9E3779B9u, kW1 = 0xBB67AE85u;
+  uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    if (r > 0) {
+      k0 += kW0;
+      k1 += kW1;
+    }
+    const uint64_t p0 = (uint64_t)kM0 * c0;
+    const uint64_t p1 = (uint64_t)kM1 * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    const uint32_t n1 = (uint32_t)p1;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    const uint32_t n3 = (uint32_t)p0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+  }
+  U4 o;
+  o.x[0] = c0; o.x[1] = c1; o.x[2] = c2; o.x[3] = c3;
+  return o;
+}
+
+// ---------------------------------------------------------------------------
+// Device-resident counters and status
+// ---------------------------------------------------------------------------
+struct Counters {
+  long long step;    // optimisation steps taken so far (lockstep: one value for the population)
+  long long round;   // ready points passed so far
+  int status;        // 0, or a pbt_status set by a kernel (bounded wait expired, ...)
+  int status_info;   // where it was set
+  int use_supplied_batch;  // next step trains on rows supplied by the caller
+  int pad;
+};
+
+// ---------------------------------------------------------------------------
+// GEMM description: C[m][n] = sum_k A(m,k) * B(n,k), one problem per member.
+// A_MN == false: A(m,k) = A[m*lda + k] (K contiguous); true: A(m,k) = A[k*lda + m].
+// B likewise over (n,k).  Strides are in elements of the operand type.
+// ---------------------------------------------------------------------------
+enum DType : int { kF32 = 0, kBF16 = 1 };
+
+struct GemmArgs {
+  int M, N, K, batch;
+  int in_dtype;   // DType of A and B
+  int out_dtype;  // DType of C
+  const void* A; long long lda, strideA; int a_mn;
+  const void* B; long long ldb, strideB; int b_mn;
+  void* C; long long ldc, strideC;
+  const float* bias; long long strideBias;  // added per column n (may be null)
+  int relu;                                 // max(., 0) after the bias
+  const void* mask; long long ldmask, strideMask;  // C *= (mask[m][n] > 0), operand type (may be null)
+};
+
+// launchers (each enqueues on `s` and returns the CUDA error of the launch)
+cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t s);
+// tensor-core path; returns cudaErrorNotSupported when the shape does not qualify
+bool gemm_tc_supported(const GemmArgs& g);
+cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s);
+
+struct OptArgs {
+  int n_members;
+  long long p_pad;           // slab stride in elements
+  long long begin, count;    // element range of the stack inside each slab (multiples of 8)
+  float* w32; float* opt1; float* opt2; const float* grad; bf16* w16;  // w16 may be null
+  const float* H; int nh_stride;  // per-member hyperparameters (float), row stride
+  int slot_lr, slot_momentum, slot_beta1, slot_wd;
+  float const_lr, const_momentum, const_beta1, const_beta2, const_eps, const_wd;
+  float* scalars; int scalar_base;   // scalars[m*PBT_N_SCALARS + scalar_base + {0,1}] = c1, c2
+};
+cudaError_t launch_sgdm(const OptArgs& a, cudaStream_t s);
+cudaError_t launch_adam(const OptArgs& a, cudaStream_t s);
+cudaError_t launch_adam_advance(const OptArgs& a, cudaStream_t s);
+
+struct SelectArgs {
+  int n, nh, n_cut;
+  int h_is_double;
+  void* H;            // [n][PBT_MAX_NH] float or double
+  void* fitness;      // [n] float or double
+  int* src;           // [n]
+  Counters* counters;
+  uint64_t seed;
+  uint32_t perturb_mask, flags;
+  double factor_lo, factor_hi;
+  double clamp_lo[PBT_MAX_NH], clamp_hi[PBT_MAX_NH];
+};
+cudaError_t launch_select_explore(const SelectArgs& a, cudaStream_t s);
+
+struct CopyArgs {
+  int n;
+  const int* src;
+  // up to 5 member-major arrays copied donor -> recipient; bytes per member, stride in bytes
+  int n_arrays;
+  char* base[5];
+  long long stride_bytes[5];
+  long long copy_bytes[5];  // multiples of 16
+};
+cudaError_t launch_slab_copy(const CopyArgs& a, cudaStream_t s);
+cudaError_t launch_copy_small(char* base, long long bytes, const int* src, int n, cudaStream_t s);
+
+// misc kernels -------------------------------------------------------------
+cudaError_t launch_init_weights(float* w32, long long p_pad, int n_members, long long w_off, int fan_out,
+                                int fan_in, int tensor_id, float bound, uint64_t seed, cudaStream_t s);
+cudaError_t launch_f32_to_bf16(const float* in, bf16* out, long long n, cudaStream_t s);
+// copy rows [off, off+rows) of a pool into dst + m*dst_stride_bytes (+ dst_offset_bytes) for every member;
+// off = 128 * ((word * n_win) >> 32), word = philox(seed; m, step, batch stream, block).x[word_index]
+cudaError_t launch_gather_window(char* dst, long long dst_stride_bytes, long long dst_offset_bytes,
+                                 const char* pool, int row_bytes, int rows, int pool_rows, int n_members,
+                                 int block, int word_index, uint64_t seed, const Counters* counters,
+                                 cudaStream_t s);
+// strided row copy with optional conversion (float -> operand type), per member
+cudaError_t launch_copy_rows(void* dst, int dst_dtype, long long dst_ld, long long dst_stride,
+                             const float* src, long long src_ld, long long src_stride, int rows, int cols,
+                             int n_members, cudaStream_t s);
+
+struct LossArgs {
+  int kind;        // pbt_loss
+  int n_members, rows, cols;
+  int n_real_rows; // GAN: rows < n_real_rows are labelled real
+  float inv_batch; // 1 / B  (scale of dL/dz and of the mean)
+  const float* logits; long long ld_logits, stride_logits;
+  const void* target; long long stride_target;   // elements of the target type; 0 = shared by all members
+  int target_dtype;                              // DType for MSE / CE_SOFT targets (MSE is always float)
+  void* dz; int dz_dtype; long long ld_dz, stride_dz;   // may be null (eval)
+  float* row_loss;   // [n_members][rows]
+};
+cudaError_t launch_loss_rows(const LossArgs& a, cudaStream_t s);
+// out[m*out_stride] = scale * sum_r row_loss[m][r], fixed summation order
+cudaError_t launch_reduce_rows(const float* row_loss, int rows, int n_members, float scale, void* out,
+                               int out_is_double, int out_stride, cudaStream_t s);
+cudaError_t launch_bias_grad(const void* dz, int dz_dtype, long long ld, long long stride, int rows, int cols,
+                             float* out, long long out_stride, int n_members, cudaStream_t s);
+cudaError_t launch_toy_step(double* theta, const double* H, int n_members, int dim, double eta, cudaStream_t s);
+cudaError_t launch_toy_eval(const double* theta, double* fitness, int n_members, int dim, cudaStream_t s);
+// fitness[m] = -(energy distance between x[m][n][2] and the eight-mode unit ring)
+cudaError_t launch_energy_distance(const float* x, long long stride, int n, int n_members, double* partial,
+                                   float* fitness, cudaStream_t s);
+int energy_partial_count(int n);  // doubles of scratch per member
+cudaError_t launch_advance_step(Counters* c, cudaStream_t s);
+
+}  // namespace pbt

@@ -1,0 +1,259 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Integer / index / hyperparameter results must be bit-exact;
+floating-point tensors must agree within tests/util.py's tolerances."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import pbt_oracle as O
+from workloads import configs as C
+from workloads import get_config, make_inputs
+
+from util import TOL, assert_state_close, push_oracle_state, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pkg():
+    import paper_1711_09846_b200 as p
+    p.load_library()
+    return p
+
+
+def _tol(cfg):
+    t = TOL[cfg.dtype]
+    return {"w": t["w"], "opt1": t["g"], "opt2": 2 * t["g"], "grad": t["g"]}
+
+
+# ---------------------------------------------------------------------------
+# config 1: the toy of Figure 2, fp64, everything bit-exact
+# ---------------------------------------------------------------------------
+def test_toy_full_run_bit_exact(pkg):
+    cfg = get_config("c1")
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    for t in range(1, cfg.total_steps + 1):
+        gpu.step(1)
+        cpu.step(1)
+        for m in range(2):
+            assert np.array_equal(gpu.get_state(m)["w"], cpu.theta[m]), (t, m)
+        if t % cfg.ready_interval == 0:
+            gpu.eval()
+            cpu.eval()
+            assert np.array_equal(gpu.fitness(), cpu.fitness), t
+            gpu.exploit_explore()
+            src = cpu.exploit_explore()
+            assert np.array_equal(gpu.copy_map(), src)
+            assert np.array_equal(gpu.hparams(), cpu.H)
+            assert np.array_equal(gpu.fitness(), cpu.fitness)
+            for m in range(2):
+                s = gpu.get_state(m)
+                assert np.array_equal(s["w"], cpu.theta[m]) and s["round"] == cpu.round and s["step"] == t
+    assert gpu.best() == cpu.best()
+    gpu.close()
+
+
+def test_toy_run_matches_oracle_run_and_leaves_the_plateau(pkg):
+    cfg = get_config("c1")
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    gpu.run(400)
+    cpu.run(400)
+    gpu.eval()
+    cpu.eval()
+    assert np.array_equal(gpu.fitness(), cpu.fitness)
+    assert max(gpu.fitness()) > 1.0          # Figure 2: PBT converges towards the optimum 1.2
+    gpu.close()
+
+
+# ---------------------------------------------------------------------------
+# exploit / explore decisions: bit-exact for injected fitness vectors
+# ---------------------------------------------------------------------------
+def _tiny_cfg(n, dtype=C.FP32, flags=C.COPY_WEIGHTS | C.COPY_HPARAMS | C.EXPLORE, num=1, den=5):
+    base = get_config("c3_mini" if dtype == C.BF16 else "c2_mini")
+    return base.replace(n_members=n, flags=flags, trunc_num=num, trunc_den=den, name=f"tiny{n}")
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 16, 24, 32, 45, 80, 200])
+@pytest.mark.parametrize("dtype", [C.FP32, C.BF16])
+def test_select_copy_explore_bit_exact(pkg, n, dtype):
+    cfg = _tiny_cfg(n, dtype)
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    rng = np.random.default_rng(n)
+    gpu.step(1)
+    cpu.step(1)
+    push_oracle_state(gpu, cpu)
+    for rnd in range(4):
+        f = rng.standard_normal(n).astype(np.float32)
+        if rnd == 1:
+            f = np.round(f)                           # many exact ties, signed zeros
+            f[::3] = -0.0
+        if rnd == 2 and n > 2:
+            f[rng.integers(0, n)] = np.nan
+            f[rng.integers(0, n)] = -np.inf
+        cpu.fitness[:] = f
+        gpu.set_fitness(f.astype(np.float64))
+        before = [gpu.get_state(m) for m in range(n)]
+        gpu.exploit_explore()
+        src = cpu.exploit_explore()
+        assert np.array_equal(gpu.copy_map(), src)
+        assert np.array_equal(gpu.hparams(), cpu.H.astype(np.float64))
+        assert np.array_equal(gpu.fitness(), cpu.fitness.astype(np.float64), equal_nan=True)
+        for m in range(n):
+            now = gpu.get_state(m)
+            assert now["round"] == cpu.round
+            d = int(src[m])
+            for key in ("w", "opt1", "opt2", "scalars"):
+                assert np.array_equal(now[key], before[d][key]), (rnd, m, key)   # copy is bit-exact
+                assert np.array_equal(now[key], cpu.get_flat(m)[key]), (rnd, m, key)
+    gpu.close()
+
+
+@pytest.mark.parametrize("flags", [0, C.COPY_WEIGHTS, C.COPY_HPARAMS | C.EXPLORE, C.COPY_WEIGHTS | C.EXPLORE])
+def test_flag_variants_bit_exact(pkg, flags):
+    cfg = _tiny_cfg(10, C.FP32, flags=flags, num=2, den=5)
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    f = np.arange(10, dtype=np.float32)[::-1].copy()
+    cpu.fitness[:] = f
+    gpu.set_fitness(f.astype(np.float64))
+    gpu.exploit_explore()
+    src = cpu.exploit_explore()
+    assert np.array_equal(gpu.copy_map(), src) and (src != np.arange(10)).sum() == 4
+    assert np.array_equal(gpu.hparams(), cpu.H.astype(np.float64))
+    assert np.array_equal(gpu.fitness(), cpu.fitness.astype(np.float64))
+    for m in range(10):
+        assert np.array_equal(gpu.get_state(m)["w"], cpu.get_flat(m)["w"])
+    gpu.close()
+
+
+# ---------------------------------------------------------------------------
+# initial population
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["c2_mini", "c3_mini", "c4_mini", "c5_mini"])
+def test_initial_population_bit_exact(pkg, name):
+    cfg = get_config(name)
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    for m in range(cfg.n_members):
+        g, c = gpu.get_state(m), cpu.get_flat(m)
+        assert np.array_equal(g["w"], c["w"])
+        assert not g["opt1"].any() and not g["opt2"].any()
+        assert list(g["scalars"]) == [1.0] * 4 and g["step"] == 0 and g["round"] == 0
+    assert np.array_equal(gpu.hparams(), cpu.H.astype(np.float64))
+    gpu.close()
+
+
+# ---------------------------------------------------------------------------
+# step / eval parity, step by step, re-seeding the GPU from the oracle at ready points
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["c2_mini", "c3_mini", "c4_mini", "c5_mini", "c3_mid", "c5_mid", "c4_mid"])
+def test_step_eval_exploit_parity(pkg, name):
+    cfg = get_config(name)
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    tol = _tol(cfg)
+    ftol = 1e-4 if cfg.dtype == C.FP32 else 2e-2
+    keys = ("w", "opt1", "grad") if cfg.optimizer == C.OPT_SGDM else ("w", "opt1", "opt2", "grad")
+    for t in range(1, cfg.total_steps + 1):
+        gpu.step(1)
+        cpu.step(1)
+        ll = gpu.last_loss()
+        for m in range(cfg.n_members):
+            g, c = gpu.get_state(m), cpu.get_flat(m)
+            assert g["step"] == t
+            assert_state_close(cfg, g, c, keys, tol, what=f"{name} step {t} member {m}")
+            assert np.array_equal(g["scalars"], c["scalars"])
+            ncols = 2 if cfg.model == C.GAN else 1
+            np.testing.assert_allclose(ll[m, :ncols], cpu.last_loss[m, :ncols], rtol=ftol, atol=1e-5)
+        if t % cfg.ready_interval == 0:
+            gpu.eval()
+            cpu.eval()
+            np.testing.assert_allclose(gpu.fitness(), cpu.fitness, rtol=ftol, atol=2e-5)
+            # selection is compared on identical fitness vectors
+            gpu.set_fitness(cpu.fitness.astype(np.float64))
+            gpu.exploit_explore()
+            src = cpu.exploit_explore()
+            assert np.array_equal(gpu.copy_map(), src)
+            assert np.array_equal(gpu.hparams(), cpu.H.astype(np.float64))
+            push_oracle_state(gpu, cpu)
+    gpu.close()
+
+
+def test_free_running_interval_stays_within_tolerance(pkg):
+    """A whole ready interval without re-seeding (fp32: errors do not compound beyond the bar)."""
+    cfg = get_config("c2_mini")
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    gpu.step(cfg.ready_interval)
+    cpu.step(cfg.ready_interval)
+    for m in range(cfg.n_members):
+        assert_state_close(cfg, gpu.get_state(m), cpu.get_flat(m), ("w",), {"w": 1e-5})
+    gpu.close()
+
+
+def test_exploit_off_members_are_isolated_and_runs_are_deterministic(pkg):
+    cfg = get_config("c3_mini").replace(flags=0)
+    inp = make_inputs(cfg)
+    a, b = pkg.Population(cfg, inp), pkg.Population(cfg, inp)
+    a.run(6)
+    # b: same seed, same steps -> bit-identical (fixed-order reductions, no float atomics)
+    b.run(6)
+    for m in range(cfg.n_members):
+        sa, sb = a.get_state(m), b.get_state(m)
+        for key in ("w", "opt1", "opt2", "grad"):
+            assert np.array_equal(sa[key], sb[key])
+    # a member's trajectory does not depend on the others: scramble every other member of b and re-run
+    c = pkg.Population(cfg, inp)
+    junk = np.random.default_rng(0).standard_normal(c.n_params).astype(np.float32)
+    for m in range(1, cfg.n_members):
+        c.set_state(m, w=junk)
+    c.run(6)
+    s0, c0 = a.get_state(0), c.get_state(0)
+    for key in ("w", "opt1", "opt2"):
+        assert np.array_equal(s0[key], c0[key])
+    assert np.array_equal(a.hparams(), np.asarray(inp.init_hparams))
+    for p in (a, b, c):
+        p.close()
+
+
+def test_supplied_batch_matches_oracle(pkg):
+    import torch
+    cfg = get_config("c2_mini")
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((cfg.batch, cfg.widths[0][0])).astype(np.float32)
+    y = rng.standard_normal((cfg.batch, 1)).astype(np.float32)
+    xd = torch.from_numpy(np.tile(x, (cfg.n_members, 1, 1))).cuda().contiguous()
+    yd = torch.from_numpy(np.tile(y, (cfg.n_members, 1, 1))).cuda().contiguous()
+    gpu.set_batch(xd, yd)
+    gpu.step(1)
+    cpu.step(1, batch=(x, y))
+    for m in range(cfg.n_members):
+        assert_state_close(cfg, gpu.get_state(m), cpu.get_flat(m), ("w", "grad"), {"w": 1e-5, "grad": 1e-4})
+    # the next step goes back to pool windows
+    gpu.step(1)
+    cpu.step(1)
+    for m in range(cfg.n_members):
+        assert_state_close(cfg, gpu.get_state(m), cpu.get_flat(m), ("w",), {"w": 1e-5})
+    gpu.close()
+
+
+def test_invalid_arguments_are_reported_not_fatal(pkg):
+    cfg = get_config("c2_mini")
+    inp = make_inputs(cfg)
+    gpu = pkg.Population(cfg, inp)
+    with pytest.raises(pkg.PbtError) as e:
+        gpu.get_state(99)
+    assert e.value.code == 1
+    with pytest.raises(pkg.PbtError):
+        gpu.step(-1)
+    gpu.step(1)      # the handle is still usable
+    gpu.close()
+    bad = cfg.replace(widths=((40, 0, 1),))
+    with pytest.raises(pkg.PbtError):
+        pkg.Population(bad, inp)

@@ -1,0 +1,53 @@
+"""Helpers shared by the parity tests (no method arithmetic here)."""
+import numpy as np
+
+# Tolerances, per tensor, as ||gpu - oracle||_2 / ||oracle||_2.
+#   fp32 populations: weights 1e-5 (the stated bar); gradients and optimiser state 1e-4
+#     (fp32 accumulation over K <= 2048 terms against float64: ~sqrt(K) * 6e-8).
+#   bf16 populations: 2e-2 for weights (the stated bar) and the same for gradients / state:
+#     both sides multiply identical bf16 operands; differences come from fp32 vs float64
+#     accumulation and from the rare activation whose bf16 rounding flips (one ulp = 2^-8).
+TOL = {"fp32": {"w": 1e-5, "g": 1e-4}, "bf16_fp32master": {"w": 2e-2, "g": 2e-2}}
+
+
+def tensor_slices(cfg):
+    """(name, slice) of every tensor in the interface's flat order: per stack, per layer, W then b."""
+    out, o = [], 0
+    for s, ws in enumerate(cfg.widths):
+        for l in range(len(ws) - 1):
+            n = ws[l] * ws[l + 1]
+            out.append((f"s{s}.W{l}", slice(o, o + n)))
+            o += n
+            out.append((f"s{s}.b{l}", slice(o, o + ws[l + 1])))
+            o += ws[l + 1]
+    return out
+
+
+def rel_err(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    nb = np.linalg.norm(b)
+    na = np.linalg.norm(a - b)
+    if nb == 0.0:
+        return 0.0 if na == 0.0 else float("inf")
+    return na / nb
+
+
+def assert_state_close(cfg, gpu_state, cpu_state, keys, tol, what=""):
+    for key in keys:
+        for name, sl in tensor_slices(cfg):
+            e = rel_err(gpu_state[key][sl], cpu_state[key][sl])
+            assert e <= tol[key], f"{what} {key} {name}: rel err {e:.3e} > {tol[key]:.1e}"
+
+
+def push_oracle_state(gpu, cpu):
+    """Overwrite the GPU population with the oracle's state (all members)."""
+    for m in range(cpu.N):
+        if cpu.toy:
+            gpu.set_state(m, w=cpu.theta[m], hparams=cpu.H[m].astype(np.float64),
+                          fitness=float(cpu.fitness[m]), step=cpu.step_count, round=cpu.round)
+        else:
+            f = cpu.get_flat(m)
+            gpu.set_state(m, w=f["w"], opt1=f["opt1"], opt2=f["opt2"], scalars=f["scalars"],
+                          hparams=cpu.H[m].astype(np.float64), fitness=float(cpu.fitness[m]),
+                          step=cpu.step_count, round=cpu.round)
