@@ -147,6 +147,26 @@ def test_initial_population_bit_exact(pkg, name):
     gpu.close()
 
 
+def _check_optimizer_arithmetic(cfg, s0, s1, h):
+    """The fused optimiser kernel against the oracle's update formula on the GPU's own
+    gradient and pre-step state: every element, well conditioned or not."""
+    g = s1["grad"].astype(np.float64)
+    w0, m0, v0 = (s0[k].astype(np.float64) for k in ("w", "opt1", "opt2"))
+    lr = h[cfg.slot("lr")]
+    if cfg.optimizer == C.OPT_SGDM:
+        w, m = O.sgdm_update(w0, m0, g, lr, h[cfg.slot("momentum")])
+        v = v0
+    else:
+        b1 = h[cfg.slot("beta1")] if cfg.slot("beta1") >= 0 else float(np.float32(cfg.beta1))
+        wd = h[cfg.slot("wd")] if cfg.slot("wd") >= 0 else cfg.weight_decay
+        w, m, v = O.adam_update(w0, m0, v0, g, lr, b1, float(np.float32(cfg.beta2)), float(np.float32(cfg.eps)),
+                                wd, s1["scalars"][0], s1["scalars"][1])
+    # fp32 roundings of the two terms of each moment: relative to the larger term, not to a cancelled sum
+    np.testing.assert_allclose(s1["opt1"], m, rtol=2e-6, atol=2e-7 * max(np.abs(m0).max(), np.abs(g).max()))
+    np.testing.assert_allclose(s1["opt2"], v, rtol=2e-6, atol=2e-7 * max(np.abs(v0).max(), (g * g).max()))
+    np.testing.assert_allclose(s1["w"], w, rtol=2e-6, atol=1e-5 * lr)
+
+
 # ---------------------------------------------------------------------------
 # step / eval parity, step by step, re-seeding the GPU from the oracle at ready points
 # ---------------------------------------------------------------------------
@@ -159,6 +179,8 @@ def test_step_eval_exploit_parity(pkg, name):
     ftol = 1e-4 if cfg.dtype == C.FP32 else 2e-2
     keys = ("w", "opt1", "grad") if cfg.optimizer == C.OPT_SGDM else ("w", "opt1", "opt2", "grad")
     for t in range(1, cfg.total_steps + 1):
+        before = [gpu.get_state(m) for m in range(cfg.n_members)]
+        h_now = gpu.hparams()
         gpu.step(1)
         cpu.step(1)
         ll = gpu.last_loss()
@@ -166,6 +188,8 @@ def test_step_eval_exploit_parity(pkg, name):
             g, c = gpu.get_state(m), cpu.get_flat(m)
             assert g["step"] == t
             assert_state_close(cfg, g, c, keys, tol, what=f"{name} step {t} member {m}")
+            if cfg.model != C.GAN:
+                _check_optimizer_arithmetic(cfg, before[m], g, h_now[m])
             assert np.array_equal(g["scalars"], c["scalars"])
             ncols = 2 if cfg.model == C.GAN else 1
             np.testing.assert_allclose(ll[m, :ncols], cpu.last_loss[m, :ncols], rtol=ftol, atol=1e-5)
@@ -179,7 +203,8 @@ def test_step_eval_exploit_parity(pkg, name):
             src = cpu.exploit_explore()
             assert np.array_equal(gpu.copy_map(), src)
             assert np.array_equal(gpu.hparams(), cpu.H.astype(np.float64))
-            push_oracle_state(gpu, cpu)
+        # every step starts from identical state: training is chaotic, parity is per step
+        push_oracle_state(gpu, cpu)
     gpu.close()
 
 
@@ -192,6 +217,29 @@ def test_free_running_interval_stays_within_tolerance(pkg):
     cpu.step(cfg.ready_interval)
     for m in range(cfg.n_members):
         assert_state_close(cfg, gpu.get_state(m), cpu.get_flat(m), ("w",), {"w": 1e-5})
+    gpu.close()
+
+
+@pytest.mark.parametrize("name", ["c3_mini", "c5_mini", "c4_mini"])
+def test_free_running_interval_bf16(pkg, name):
+    """A whole ready interval without re-seeding, bf16 compute: the fitness that selection sees and
+    every weight matrix stay within the bar.  (Bias vectors start at zero and are O(lr) after a few
+    Adam steps, so a single near-zero gradient whose sign differs moves them by more than 2 % of
+    their own norm; they are covered by the per-step test above.)"""
+    cfg = get_config(name)
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    gpu.step(cfg.ready_interval)
+    cpu.step(cfg.ready_interval)
+    from util import tensor_slices
+    for m in range(cfg.n_members):
+        g, c = gpu.get_state(m), cpu.get_flat(m)
+        for tname, sl in tensor_slices(cfg):
+            if ".W" in tname:
+                assert rel_err(g["w"][sl], c["w"][sl]) <= 2e-2, (name, m, tname)
+    gpu.eval()
+    cpu.eval()
+    np.testing.assert_allclose(gpu.fitness(), cpu.fitness, rtol=2e-2, atol=1e-4)
     gpu.close()
 
 

@@ -33,10 +33,31 @@ def rel_err(a, b):
     return na / nb
 
 
+def adam_well_conditioned(cfg, cpu_state, tol_g):
+    """Adam's normalised update lr * m / (sqrt(v) + eps) behaves like lr * sign(g) while the
+    moments are young: an element whose gradient could change sign under a perturbation that
+    the gradient tolerance itself allows (|g| < tol_g * rms(g) of its tensor) can move by a
+    full 2 lr, which swamps tensors whose norm is itself O(lr) (biases start at zero).  Such
+    elements are left out of the direct weight comparison only; they stay in the gradient,
+    moment and optimiser-arithmetic comparisons.  Decided from oracle values alone."""
+    keep = np.ones(cpu_state["grad"].shape, dtype=bool)
+    for _, sl in tensor_slices(cfg):
+        g = cpu_state["grad"][sl].astype(np.float64)
+        rms = np.sqrt(np.mean(g * g)) if g.size else 0.0
+        keep[sl] = np.abs(g) >= tol_g * rms if rms > 0 else False
+    return keep
+
+
 def assert_state_close(cfg, gpu_state, cpu_state, keys, tol, what=""):
+    keep = None
+    if cfg.optimizer == "adam" and "w" in keys and "grad" in cpu_state:
+        keep = adam_well_conditioned(cfg, cpu_state, tol.get("grad", 2e-2))
     for key in keys:
         for name, sl in tensor_slices(cfg):
-            e = rel_err(gpu_state[key][sl], cpu_state[key][sl])
+            a, b = gpu_state[key][sl], cpu_state[key][sl]
+            if key == "w" and keep is not None:
+                a = np.where(keep[sl], a, b)
+            e = rel_err(a, b)
             assert e <= tol[key], f"{what} {key} {name}: rel err {e:.3e} > {tol[key]:.1e}"
 
 
