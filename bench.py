@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Throughput of the PBT hot path on synthetic data: population member-samples per second.
+
+One "step" = one lockstep pass of the whole hot path over one batch per member: batch
+window, forward, loss, backward, fused optimiser; at every ready point (the workload's
+ready interval) also evaluation and exploit/explore.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--impl ours|reference]
+
+N > 1 (under torch.distributed.run) runs N independent replicas of the population, one per
+GPU, with no data-path collective ("replicas only"); the value is the sum over replicas
+divided by the slowest replica's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "population member-samples/sec"
+UNIT = "member-samples/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def _algorithmic_work(cfg, n_params_padded=None):
+    """FLOPs of the grouped GEMMs and optimiser bytes of ONE lockstep step of the whole population."""
+    flops = 0.0
+    updates = [(0, 1)] if cfg.model != "gan_pair" else [(0, 1), (1, cfg.gan_d_steps)]
+    B = cfg.batch
+    if cfg.model == "gan_pair":
+        g, d = cfg.widths
+        wg = sum(g[i] * g[i + 1] for i in range(len(g) - 1))
+        wd = sum(d[i] * d[i + 1] for i in range(len(d) - 1))
+        K = cfg.gan_d_steps
+        # K discriminator updates: G forward (B), D forward+wgrad on 2B rows, D dgrad above layer 0
+        flops += K * (2 * B * wg + 2 * (2 * B) * wd * 2 + 2 * (2 * B) * (wd - d[0] * d[1]))
+        # generator update: G fwd, D fwd, D dgrad to the input, G dgrad + wgrad
+        flops += 2 * B * wg + 2 * B * wd + 2 * B * wd + 2 * B * (wg - g[0] * g[1]) + 2 * B * wg
+        params = {0: wg + sum(g[1:]), 1: wd + sum(d[1:])}
+    else:
+        w = cfg.widths[0]
+        W = sum(w[i] * w[i + 1] for i in range(len(w) - 1))
+        flops += 2 * B * W + 2 * B * (W - w[0] * w[1]) + 2 * B * W
+        params = {0: W + sum(w[1:])}
+    bytes_per_param = {"adam": 16 + 12, "sgdm": 12 + 8}[cfg.optimizer] + (2 if cfg.dtype == "bf16_fp32master" else 0)
+    opt_bytes = sum(params[s] * k for s, k in updates) * bytes_per_param
+    return cfg.n_members * flops, cfg.n_members * opt_bytes
+
+
+def _cpu_count_used():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((i.get("num_threads", 1) for i in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def _oracle_sample(cfg, inp, members, steps):
+    """Time the CPU oracle, as it stands, on `members` members for `steps` steps."""
+    from oracle import pbt_oracle as O
+    sub = cfg.replace(n_members=members)
+    sub_inp = type(inp)(**{**inp.__dict__, "init_hparams": inp.init_hparams[:members]})
+    pop = O.Population(sub, sub_inp)
+    t0 = time.perf_counter()
+    pop.step(steps)
+    dt = time.perf_counter() - t0
+    return members * cfg.batch * steps / dt, dt
+
+
+def _oracle_budget(cfg):
+    """(members, steps) of the bounded oracle sample: roughly 10-30 s of CPU work."""
+    flops, _ = _algorithmic_work(cfg)
+    per_member = flops / cfg.n_members
+    target = 10.0 * 3e10          # ~10 s at an assumed ~30 GFLOP/s effective float64 rate
+    members = max(1, min(cfg.n_members, int(target // max(per_member, 1))))
+    steps = max(1, min(50, int(target // max(per_member * members, 1))))
+    return members, steps
+
+
+def run_reference(args, cfg, inp):
+    """The oracle as the reference arm: every step is a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import pbt_oracle as O
+    members, _ = _oracle_budget(cfg)
+    members = max(1, min(members, 4))
+    sub = cfg.replace(n_members=members)
+    sub_inp = type(inp)(**{**inp.__dict__, "init_hparams": inp.init_hparams[:members]})
+    pop = O.Population(sub, sub_inp)
+    for _ in range(args.warmup):
+        pop.step(1)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        pop.step(1)
+    dt = time.perf_counter() - t0
+    value = members * cfg.batch * args.steps / dt
+    cores = _cpu_count_used()
+    sample = f"{members} of {cfg.n_members} members x {args.steps} steps, float64 NumPy oracle"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "members": cfg.n_members, "batch": cfg.batch, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c5")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--pool-rows", type=int, default=0, help="override the training-pool size (default: the workload's)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from workloads import get_config, make_inputs
+    cfg = get_config(args.workload)
+    if args.pool_rows:
+        cfg = cfg.replace(pool_rows=args.pool_rows)
+
+    if args.impl == "reference":
+        if args.steps == 50:
+            args.steps = 3
+        if args.warmup >= 3:
+            args.warmup = 1
+        small = cfg.replace(pool_rows=min(cfg.pool_rows, 4096), eval_batch=min(cfg.eval_batch, 512))
+        run_reference(args, small, make_inputs(small))
+        return
+
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    import paper_1711_09846_b200 as pkg
+    inp = make_inputs(cfg)
+    pop = pkg.Population(cfg, inp, device=f"cuda:{local}")
+    interval = cfg.ready_interval
+
+    def hot_path_step(i, launches):
+        pop.step(1)
+        launches[0] += pop.launch_count()
+        if (i + 1) % interval == 0:
+            pop.eval()
+            launches[0] += pop.launch_count()
+            pop.exploit_explore()
+            launches[0] += pop.launch_count()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    scratch = [0]
+    for i in range(args.warmup):
+        hot_path_step(i, scratch)
+    # one ready point in the warm-up regardless of its length
+    pop.eval()
+    pop.exploit_explore()
+
+    # ---- timed region: device-resident inputs, CUDA events on the library's stream ----
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier()
+    launches = [0]
+    pop.profile_begin()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(pop.stream)
+    for i in range(args.steps):
+        hot_path_step(i, launches)
+    e1.record(pop.stream)
+    prof = pop.profile_end()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], device=f"cuda:{local}")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * cfg.n_members * cfg.batch * args.steps / (ms * 1e-3)
+
+    # ---- end to end: host buffers in, loss out, through the C ABI (MLP populations) ----
+    e2e = None
+    if cfg.model == "mlp":
+        op = torch.bfloat16 if cfg.dtype == "bf16_fp32master" else torch.float32
+        ydt = {"mse": torch.float32, "ce_hard": torch.int32, "ce_soft": op}[cfg.loss]
+        n_host = 2
+        xs, ys = [], []
+        for j in range(n_host):
+            off = 128 * j
+            xs.append(torch.from_numpy(inp.x_pool[off:off + cfg.batch]).to(op).unsqueeze(0)
+                      .repeat(cfg.n_members, 1, 1).contiguous().pin_memory())
+            yb = torch.from_numpy(inp.y_pool[off:off + cfg.batch]).to(ydt).unsqueeze(0)
+            ys.append(yb.repeat(cfg.n_members, *([1] * (yb.dim() - 1))).contiguous().pin_memory())
+        loss_out = np.zeros((cfg.n_members, 2), dtype=np.float64)
+        e2e_steps = max(3, min(args.steps, 20))
+        for j in range(2):
+            pop.step_host(xs[j % n_host], ys[j % n_host], loss_out)
+        barrier()
+        t0 = time.perf_counter()
+        for j in range(e2e_steps):
+            pop.step_host(xs[j % n_host], ys[j % n_host], loss_out)
+            if (j + 1) % interval == 0:
+                pop.eval()
+                pop.exploit_explore()
+        pop.synchronize()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], device=f"cuda:{local}")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        e2e = {"value": world * cfg.n_members * cfg.batch * e2e_steps / dt, "unit": UNIT,
+               "h2d_bytes_per_step": int(xs[0].numel() * xs[0].element_size() + ys[0].numel() * ys[0].element_size()),
+               "d2h_bytes_per_step": int(cfg.n_members * 2 * 4), "steps": e2e_steps,
+               "timing": "host wall clock around pbt_step_host (H2D of the batch, step, D2H of the losses)"}
+    else:
+        e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+               "note": "host-fed steps exist for MLP populations only"}
+
+    # ---- roofline of the dominant kernel class, from the events recorded inside the timed region ----
+    peaks = _peaks()
+    flops_step, opt_bytes_step = _algorithmic_work(cfg)
+    kern = {}
+    if prof["gemm"]["launches"]:
+        tf = flops_step * args.steps / (prof["gemm"]["ms"] * 1e-3) / 1e12
+        bound = "tensor" if cfg.dtype == "bf16_fp32master" else "alu"
+        peak = peaks["bf16_tflops_sustained"] if bound == "tensor" else 2 * 148 * 128 * 1.965e9 / 1e12
+        kern["gemm"] = {"bound": bound, "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                        "traffic": None, "ms_per_step": prof["gemm"]["ms"] / args.steps,
+                        "launches_per_step": prof["gemm"]["launches"] / args.steps,
+                        "peak_source": peaks["source"] + (" sustained bf16" if bound == "tensor" else
+                                                          " n/a: 148 SM x 128 FMA x 2 x 1.965 GHz fp32")}
+    if prof["optimizer"]["launches"] and cfg.model != "toy_quadratic":
+        gbs = opt_bytes_step * args.steps / (prof["optimizer"]["ms"] * 1e-3) / 1e9
+        kern["optimizer"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                             "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                             "ms_per_step": prof["optimizer"]["ms"] / args.steps,
+                             "launches_per_step": prof["optimizer"]["launches"] / args.steps,
+                             "peak_source": peaks["source"]}
+    shares = {k: v["ms"] for k, v in prof.items()}
+    dominant = max(kern, key=lambda k: kern[k]["ms_per_step"]) if kern else None
+    roofline = dict(kern[dominant], kernel=dominant) if dominant else None
+
+    # ---- exploit-copy bandwidth (once, outside the timed region) ----
+    copy_gbs = None
+    if cfg.model != "toy_quadratic":
+        f = np.arange(cfg.n_members, dtype=np.float64)
+        pop.set_fitness(f)
+        pop.profile_begin()
+        pop.exploit_explore()
+        pr = pop.profile_end()
+        n_cut = max(1, cfg.n_members * cfg.trunc_num // cfg.trunc_den)
+        per_member = pop.n_params * (12 if cfg.optimizer == "adam" else 8) + \
+            (pop.n_params * 2 if cfg.dtype == "bf16_fp32master" else 0)
+        if pr["copy"]["ms"] > 0:
+            copy_gbs = 2 * n_cut * per_member / (pr["copy"]["ms"] * 1e-3) / 1e9
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": {"bf16_fp32master": "bf16", "fp32": "f32", "fp64_toy": "f64"}[cfg.dtype], "data": "synthetic",
+        "config": {"workload": cfg.name, "members": cfg.n_members, "batch": cfg.batch, "widths": [list(w) for w in cfg.widths],
+                   "optimizer": cfg.optimizer, "ready_interval": interval, "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   "l2": "inputs larger than L2: population state %.1f GB" % (pop.workspace_bytes / 1e9)},
+        "e2e": e2e, "gpu_launches": int(launches[0]), "clocks": clocks, "roofline": roofline,
+        "kernels": kern, "class_ms": shares,
+        "exploit_copy": {"achieved": copy_gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"],
+                         "frac": (copy_gbs / peaks["hbm_gbs"]) if copy_gbs else None},
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        members, steps = _oracle_budget(cfg)
+        small = cfg.replace(pool_rows=min(cfg.pool_rows, 4096), eval_batch=min(cfg.eval_batch, 512))
+        v, dt = _oracle_sample(small, make_inputs(small), members, steps)
+        result["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": _cpu_count_used(), "kind": "oracle",
+                                  "sample": f"{members} of {cfg.n_members} members x {steps} step(s), {dt:.1f} s, "
+                                            f"float64 NumPy oracle, training step only"}
+    pop.close()
+    if rank == 0:
+        print(json.dumps(result))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -234,6 +234,15 @@ int pbt_get_last_loss(pbt_t* p, double* out_host);
  */
 int pbt_set_batch(pbt_t* p, const void* x_device, const void* y_device);
 
+/*
+ * One step fed from host memory, end to end: copies the caller's rows for every
+ * member (x_host [n_members][batch][in], y_host the matching targets, both in the
+ * pools' element types; pinned memory makes the copies asynchronous), runs one
+ * lockstep `step` (Eq. 2) on them, and, if loss_out_host is not NULL, copies the
+ * per-member training loss back ([n_members][2] doubles) and synchronises.  MLP only.
+ */
+int pbt_step_host(pbt_t* p, const void* x_host, const void* y_host, double* loss_out_host);
+
 /* Kernel launches issued by the last pbt_step / pbt_eval / pbt_exploit_explore call. */
 int pbt_get_launch_count(const pbt_t* p, int64_t* count);
 

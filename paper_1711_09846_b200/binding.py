@@ -62,7 +62,7 @@ EXPORTS = [
     "pbt_query_workspace", "pbt_param_count", "pbt_create", "pbt_destroy", "pbt_step", "pbt_eval",
     "pbt_exploit_explore", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
     "pbt_get_hparams", "pbt_set_hparams", "pbt_get_copy_map", "pbt_get_best", "pbt_get_last_loss",
-    "pbt_set_batch", "pbt_get_launch_count", "pbt_profile_begin", "pbt_profile_end", "pbt_profile_get",
+    "pbt_set_batch", "pbt_step_host", "pbt_get_launch_count", "pbt_profile_begin", "pbt_profile_end", "pbt_profile_get",
     "pbt_last_error",
 ]
 
@@ -102,6 +102,7 @@ def load_library() -> C.CDLL:
     lib.pbt_get_best.argtypes = [vp, C.POINTER(C.c_int32)]
     lib.pbt_get_last_loss.argtypes = [vp, C.POINTER(C.c_double)]
     lib.pbt_set_batch.argtypes = [vp, vp, vp]
+    lib.pbt_step_host.argtypes = [vp, vp, vp, C.POINTER(C.c_double)]
     lib.pbt_get_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
     lib.pbt_profile_begin.argtypes = [vp]
     lib.pbt_profile_end.argtypes = [vp]
@@ -351,6 +352,14 @@ class Population:
         """x_dev [N, batch, in], y_dev matching targets: device tensors in the pools' dtypes."""
         assert x_dev.is_cuda and y_dev.is_cuda and x_dev.is_contiguous() and y_dev.is_contiguous()
         self._check(self.lib.pbt_set_batch(self.handle, C.c_void_p(x_dev.data_ptr()), C.c_void_p(y_dev.data_ptr())))
+
+    def step_host(self, x_host, y_host, loss_out: Optional[np.ndarray] = None):
+        """One step on rows held in host memory (torch CPU tensors, ideally pinned); returns the losses."""
+        if loss_out is None:
+            loss_out = np.zeros((self.N, 2), dtype=np.float64)
+        self._check(self.lib.pbt_step_host(self.handle, C.c_void_p(x_host.data_ptr()), C.c_void_p(y_host.data_ptr()),
+                                           loss_out.ctypes.data_as(C.POINTER(C.c_double))))
+        return loss_out
 
     def launch_count(self) -> int:
         n = C.c_int64(0)

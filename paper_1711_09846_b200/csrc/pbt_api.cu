@@ -73,6 +73,7 @@ struct pbt_handle {
   bool profiling;
   std::vector<ProfRec> prof;
   std::vector<cudaEvent_t> event_pool;
+  std::vector<float> host_loss;  // staging for pbt_step_host
   double prof_ms[kNumClasses];
   int64_t prof_n[kNumClasses];
   cudaGraphExec_t step_graph;
@@ -620,6 +621,7 @@ int pbt_create(pbt_t** out, const pbt_spec* spec, const double* init_hparams, ui
   }
 #undef CREATE_CU
   h->err[0] = 0;
+  h->host_loss.assign((size_t)h->N * 2, 0.f);
   *out = h;
   return PBT_OK;
 }
@@ -956,6 +958,29 @@ int pbt_set_batch(pbt_t* p, const void* x, const void* y) {
   const int one = 1;
   CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &one, 4, cudaMemcpyHostToDevice, p->stream));
   CU(p, cudaStreamSynchronize(p->stream));
+  return PBT_OK;
+}
+
+int pbt_step_host(pbt_t* p, const void* x_host, const void* y_host, double* loss_out_host) {
+  if (!p || !x_host || !y_host) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  if (p->toy || p->gan) return fail(p, PBT_ERR_UNSUPPORTED, "host-fed steps are for MLP populations");
+  p->launches = 0;
+  const pbt_spec& s = p->spec;
+  const size_t xb = (size_t)p->N * s.batch * p->st[0].L[0].in * p->esz;
+  CU(p, cudaMemcpyAsync(p->act[0][0], x_host, xb, cudaMemcpyHostToDevice, p->stream));
+  const size_t trb = target_row_bytes(p) * s.batch;
+  const size_t tsz = s.loss == PBT_LOSS_CE_SOFT ? p->esz : 4;
+  CU(p, cudaMemcpy2DAsync(p->ybatch, p->ybatch_stride * tsz, y_host, trb, trb, p->N, cudaMemcpyHostToDevice, p->stream));
+  const int one = 1;
+  CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &one, 4, cudaMemcpyHostToDevice, p->stream));
+  int rc = one_step(p);
+  if (rc) return rc;
+  if (loss_out_host) {
+    float* tmp = p->host_loss.data();
+    CU(p, cudaMemcpyAsync(tmp, p->last_loss, (size_t)p->N * 2 * 4, cudaMemcpyDeviceToHost, p->stream));
+    CU(p, cudaStreamSynchronize(p->stream));
+    for (int i = 0; i < p->N * 2; ++i) loss_out_host[i] = tmp[i];
+  }
   return PBT_OK;
 }
 
