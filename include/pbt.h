@@ -256,6 +256,30 @@ int pbt_profile_begin(pbt_t* p);
 int pbt_profile_end(pbt_t* p);
 int pbt_profile_get(pbt_t* p, const char* kernel_class, double* ms_total, int64_t* launches);
 
+/*
+ * Allocation-free scorer (no counterpart in the paper: it exists for callers that are not
+ * allowed to allocate device memory, e.g. a plug-in inside an application that owns the
+ * whole device through its own arena, and so cannot provide the workspace pbt_create wants).
+ * Computes, for each of n_members sets of n two-dimensional points, the same fitness
+ * pbt_eval gives a GAN population: minus the energy distance between the set and the
+ * eight-mode unit ring.
+ *   x_device            [n_members][n][2] floats, device memory, caller-owned (input)
+ *   fitness_out_device  [n_members] floats, device memory, caller-owned (output)
+ *   stream              cudaStream_t as void* (NULL = default stream); the call only enqueues
+ * The partial sums of the reduction live in a fixed 1 MiB array inside the library image
+ * (held by every GPU that loads the library until the process exits), so the call performs
+ * no cudaMalloc / cudaFree.  Limits and rules:
+ *   - n_members * 2 * ceil(n / 256) must not exceed 131072, else PBT_ERR_WORKSPACE with a
+ *     message naming the size; NULL pointers or non-positive sizes give PBT_ERR_INVALID_ARG;
+ *   - the array is shared by all calls and keeps the previous call's contents; nothing in it
+ *     needs clearing, every slot read is first rewritten by the same call;
+ *   - calls that overlap on the GPU (other streams or threads) race on that array: serialise them;
+ *   - the first call on each device resolves the array's device address; make that first call
+ *     before starting any stream capture.
+ */
+int pbt_energy_fitness_static(const float* x_device, int n, int n_members, float* fitness_out_device,
+                              void* stream);
+
 const char* pbt_last_error(const pbt_t* p); /* p may be NULL: error of the last failed create/query */
 
 #ifdef __cplusplus

@@ -63,7 +63,7 @@ EXPORTS = [
     "pbt_exploit_explore", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
     "pbt_get_hparams", "pbt_set_hparams", "pbt_get_copy_map", "pbt_get_best", "pbt_get_last_loss",
     "pbt_set_batch", "pbt_step_host", "pbt_get_launch_count", "pbt_profile_begin", "pbt_profile_end", "pbt_profile_get",
-    "pbt_last_error",
+    "pbt_energy_fitness_static", "pbt_last_error",
 ]
 
 _LIB = None
@@ -107,6 +107,7 @@ def load_library() -> C.CDLL:
     lib.pbt_profile_begin.argtypes = [vp]
     lib.pbt_profile_end.argtypes = [vp]
     lib.pbt_profile_get.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    lib.pbt_energy_fitness_static.argtypes = [vp, C.c_int, C.c_int, vp, vp]
     lib.pbt_last_error.argtypes = [vp]
     lib.pbt_last_error.restype = C.c_char_p
     for name in EXPORTS:
@@ -170,6 +171,22 @@ def param_count(cfg) -> int:
     if rc:
         raise PbtError(rc, lib.pbt_last_error(None).decode())
     return n.value
+
+
+def energy_fitness_static(x_dev, fitness_out_dev, stream=None) -> None:
+    """Score point sets without any device allocation (see pbt_energy_fitness_static in pbt.h).
+
+    x_dev: CUDA float32 tensor [n_members, n, 2]; fitness_out_dev: CUDA float32 tensor [n_members],
+    written in place.  Only enqueues work on `stream` (a torch stream, or None for the default one).
+    Meant for hosts that may not allocate: the reduction's scratch is a fixed array in the library."""
+    lib = load_library()
+    assert x_dev.is_cuda and x_dev.is_contiguous() and x_dev.dim() == 3 and x_dev.shape[2] == 2
+    assert fitness_out_dev.is_cuda and fitness_out_dev.is_contiguous() and fitness_out_dev.numel() == x_dev.shape[0]
+    rc = lib.pbt_energy_fitness_static(C.c_void_p(x_dev.data_ptr()), int(x_dev.shape[1]), int(x_dev.shape[0]),
+                                       C.c_void_p(fitness_out_dev.data_ptr()),
+                                       C.c_void_p(stream.cuda_stream if stream is not None else None))
+    if rc:
+        raise PbtError(rc, lib.pbt_last_error(None).decode())
 
 
 class Population:

@@ -95,6 +95,12 @@ int fail(pbt_t* p, int code, const char* fmt, ...) {
   return code;
 }
 
+}  // namespace
+namespace pbt {
+void set_last_error(const char* msg) { snprintf(g_err, sizeof(g_err), "%s", msg); }
+}  // namespace pbt
+namespace {
+
 #define CU(p, expr)                                                                                   \
   do {                                                                                                \
     cudaError_t e_ = (expr);                                                                          \
