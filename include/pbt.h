@@ -257,6 +257,35 @@ int pbt_profile_end(pbt_t* p);
 int pbt_profile_get(pbt_t* p, const char* kernel_class, double* ms_total, int64_t* launches);
 
 /*
+ * The member-batched GEMM of the training step on its own (forward, data-gradient and
+ * weight-gradient contractions of Eq. 2's gradient step all have this form):
+ *   C_b[m][n] = epilogue( sum_k A_b(m,k) * B_b(n,k) ),  b = 0..batch-1.
+ * a_mn == 0: A_b(m,k) = A[b*strideA + m*lda + k] (K contiguous); a_mn == 1: A[b*strideA + k*lda + m].
+ * B likewise over (n,k).  Operands are float (in_bf16 == 0) or bfloat16; accumulation is fp32;
+ * C is float or bfloat16 (out_bf16).  Epilogue, in this order: + bias[b*strideBias + n] (if bias),
+ * max(.,0) (if relu), zero where mask[b*strideMask + m*ldmask + n] <= 0 (if mask; operand type).
+ * Strides are in elements; a stride of 0 shares the operand between all problems.
+ * engine: 0 = choose (tensor cores when operands are bf16 and the shape fills the tiles),
+ * 1 = FP32-ALU kernel, 2 = tcgen05 kernel (PBT_ERR_UNSUPPORTED if the shape does not qualify).
+ * status_device: 32 zeroed bytes of device memory; a bounded wait that expires inside the
+ * tensor-core kernel stores PBT_ERR_TIMEOUT in the int32 at byte offset 16.  All pointers are
+ * device pointers; the call only enqueues work on `stream`.
+ */
+typedef struct pbt_gemm_desc {
+  int32_t M, N, K, batch;
+  int32_t in_bf16, out_bf16;
+  int32_t a_mn, b_mn;
+  int32_t relu, engine;
+  const void* A; int64_t lda, strideA;
+  const void* B; int64_t ldb, strideB;
+  void* C; int64_t ldc, strideC;
+  const float* bias; int64_t strideBias;
+  const void* mask; int64_t ldmask, strideMask;
+  void* status_device;
+} pbt_gemm_desc;
+int pbt_grouped_gemm(const pbt_gemm_desc* desc, void* stream);
+
+/*
  * Allocation-free scorer (no counterpart in the paper: it exists for callers that are not
  * allowed to allocate device memory, e.g. a plug-in inside an application that owns the
  * whole device through its own arena, and so cannot provide the workspace pbt_create wants).

@@ -557,3 +557,22 @@ class Population:
         if self.toy:
             return self.theta.shape[1]
         return sum(fo * fi + fo for (_, _, fo, fi) in self.shapes)
+
+
+# --------------------------------------------------------------------------
+# the member-batched contraction on its own (forward / data-gradient / weight-gradient form)
+# --------------------------------------------------------------------------
+def grouped_gemm(A, B, bias=None, relu=False, mask=None):
+    """C_b[m][n] = sum_k A_b[m][k] B_b[n][k] in float64, then + bias_b[n], max(., 0), and zero
+    where mask_b[m][n] <= 0 -- the three epilogues of the layer equations in `forward` / `backward`."""
+    out = []
+    for b in range(A.shape[0]):
+        c = np.asarray(A[b], dtype=np.float64) @ np.asarray(B[b], dtype=np.float64).T
+        if bias is not None:
+            c = c + np.asarray(bias[b], dtype=np.float64)[None, :]
+        if relu:
+            c = np.maximum(c, 0.0)
+        if mask is not None:
+            c = c * (np.asarray(mask[b], dtype=np.float64) > 0.0)
+        out.append(c)
+    return np.stack(out)

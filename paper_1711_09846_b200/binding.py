@@ -58,12 +58,24 @@ class PbtStateView(C.Structure):
                 ("round", C.POINTER(C.c_int64))]
 
 
+class PbtGemmDesc(C.Structure):
+    _fields_ = [("M", C.c_int32), ("N", C.c_int32), ("K", C.c_int32), ("batch", C.c_int32),
+                ("in_bf16", C.c_int32), ("out_bf16", C.c_int32), ("a_mn", C.c_int32), ("b_mn", C.c_int32),
+                ("relu", C.c_int32), ("engine", C.c_int32),
+                ("A", C.c_void_p), ("lda", C.c_int64), ("strideA", C.c_int64),
+                ("B", C.c_void_p), ("ldb", C.c_int64), ("strideB", C.c_int64),
+                ("C", C.c_void_p), ("ldc", C.c_int64), ("strideC", C.c_int64),
+                ("bias", C.c_void_p), ("strideBias", C.c_int64),
+                ("mask", C.c_void_p), ("ldmask", C.c_int64), ("strideMask", C.c_int64),
+                ("status_device", C.c_void_p)]
+
+
 EXPORTS = [
     "pbt_query_workspace", "pbt_param_count", "pbt_create", "pbt_destroy", "pbt_step", "pbt_eval",
     "pbt_exploit_explore", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
     "pbt_get_hparams", "pbt_set_hparams", "pbt_get_copy_map", "pbt_get_best", "pbt_get_last_loss",
     "pbt_set_batch", "pbt_step_host", "pbt_get_launch_count", "pbt_profile_begin", "pbt_profile_end", "pbt_profile_get",
-    "pbt_energy_fitness_static", "pbt_last_error",
+    "pbt_grouped_gemm", "pbt_energy_fitness_static", "pbt_last_error",
 ]
 
 _LIB = None
@@ -107,6 +119,7 @@ def load_library() -> C.CDLL:
     lib.pbt_profile_begin.argtypes = [vp]
     lib.pbt_profile_end.argtypes = [vp]
     lib.pbt_profile_get.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    lib.pbt_grouped_gemm.argtypes = [C.POINTER(PbtGemmDesc), vp]
     lib.pbt_energy_fitness_static.argtypes = [vp, C.c_int, C.c_int, vp, vp]
     lib.pbt_last_error.argtypes = [vp]
     lib.pbt_last_error.restype = C.c_char_p
@@ -171,6 +184,36 @@ def param_count(cfg) -> int:
     if rc:
         raise PbtError(rc, lib.pbt_last_error(None).decode())
     return n.value
+
+
+def grouped_gemm(A, B, C_out, a_mn=False, b_mn=False, bias=None, relu=False, mask=None, engine=0, status=None,
+                 stream=None, shared_a=False, shared_b=False):
+    """C_b = epilogue(A_b B_b^T) for every b; torch CUDA tensors, marshalling only (see pbt_grouped_gemm).
+
+    A: [batch, M, K] (or [batch, K, M] when a_mn); B: [batch, N, K] (or [batch, K, N] when b_mn);
+    C_out: [batch, M, N] float32 or bfloat16, written in place.  bias: [batch, N] float32;
+    mask: [batch, M, N] in the operand dtype.  status: >= 8 zeroed int32 on the device."""
+    import torch
+    lib = load_library()
+    d = PbtGemmDesc()
+    batch, M, N = C_out.shape
+    K = A.shape[1] if a_mn else A.shape[2]
+    d.M, d.N, d.K, d.batch = M, N, K, batch
+    d.in_bf16 = 1 if A.dtype == torch.bfloat16 else 0
+    d.out_bf16 = 1 if C_out.dtype == torch.bfloat16 else 0
+    d.a_mn, d.b_mn, d.relu, d.engine = int(a_mn), int(b_mn), int(relu), int(engine)
+    d.A, d.lda, d.strideA = A.data_ptr(), A.stride(1), 0 if shared_a else A.stride(0)
+    d.B, d.ldb, d.strideB = B.data_ptr(), B.stride(1), 0 if shared_b else B.stride(0)
+    d.C, d.ldc, d.strideC = C_out.data_ptr(), C_out.stride(1), C_out.stride(0)
+    if bias is not None:
+        d.bias, d.strideBias = bias.data_ptr(), bias.stride(0)
+    if mask is not None:
+        d.mask, d.ldmask, d.strideMask = mask.data_ptr(), mask.stride(1), mask.stride(0)
+    if status is not None:
+        d.status_device = status.data_ptr()
+    rc = lib.pbt_grouped_gemm(C.byref(d), C.c_void_p(stream.cuda_stream if stream is not None else None))
+    if rc:
+        raise PbtError(rc, lib.pbt_last_error(None).decode())
 
 
 def energy_fitness_static(x_dev, fitness_out_dev, stream=None) -> None:

@@ -1,6 +1,448 @@
-// placeholder until the tensor-core path lands
+// Member-batched bf16 GEMM on the 5th-generation tensor cores (sm_100a):
+//   C[m][n] = sum_k A(m,k) * B(n,k),   one problem per population member,
+// covering the forward (both operands K-major), data-gradient (B MN-major) and
+// weight-gradient (both MN-major) contractions of the training step.
+//
+// Structure of one CTA (persistent, one per SM, static round-robin over tiles):
+//   warp 0      TMA producer: 3-D tiled bulk-tensor loads (member = outer coordinate), 128-byte swizzle,
+//               into a ring of shared-memory stages guarded by full/empty mbarriers; plain per-CTA loads
+//   warp 1      allocates tensor memory, one elected lane issues tcgen05.mma (128 x BN x 16 per
+//               instruction, fp32 accumulators in TMEM), tcgen05.commit frees the stage / publishes the tile
+//   warps 2..5  epilogue: tcgen05.ld of the accumulator (double-buffered in TMEM, so the next tile's
+//               main loop overlaps), bias / ReLU / ReLU-mask, conversion, 16-byte global stores
+// Every mbarrier wait is bounded; on expiry the kernel records PBT_ERR_TIMEOUT in the device status
+// word, all roles leave their loops, tensor memory is released and the kernel returns normally.
+#include <cuda.h>
+
 #include "pbt_common.cuh"
+
 namespace pbt {
-bool gemm_tc_supported(const GemmArgs&) { return false; }
-cudaError_t launch_gemm_tc(const GemmArgs&, Counters*, cudaStream_t) { return cudaErrorNotSupported; }
+
+namespace {
+
+constexpr int kBM = 128;
+constexpr int kBK = 64;
+constexpr int kThreads = 192;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct TcParams {
+  int M, N, K, batch;
+  int tiles_m, tiles_n, num_tiles, k_blocks;
+  int a_mn, b_mn, a_batched, b_batched;
+  void* C; long long ldc, strideC; int out_dtype;
+  const float* bias; long long strideBias; int relu;
+  const bf16* mask; long long ldmask, strideMask;
+  Counters* counters;
+};
+
+// ---- PTX wrappers -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// bounded wait: false when the limit ran out or another role already gave up
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (i > 64) {
+      if (*abort_flag) return false;
+      __nanosleep(64);
+    }
+  }
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives on the mbarrier once every tcgen05.mma issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// shared-memory matrix descriptor: 128-byte swizzle, addresses / offsets in 16-byte units
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;  // descriptor version of this architecture
+  d |= 2ull << 61;  // SWIZZLE_128B
+  return d;
+}
+
+template <int BN, int STAGES>
+struct Smem {
+  static constexpr int kABytes = kBM * kBK * 2;
+  static constexpr int kBBytes = BN * kBK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kBarOffset = STAGES * kStageBytes;
+  static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack for 1024-byte alignment
+};
+
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+  using L = Smem<BN, STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tfull = empty + STAGES;   // [2] accumulator ready for the epilogue
+  uint64_t* tempty = tfull + 2;       // [2] accumulator drained
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  constexpr uint32_t kTmemCols = 2 * BN;  // 256 or 512: a power of two >= 32
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+        const int member = tile / (p.tiles_m * p.tiles_n);
+        const int rem = tile % (p.tiles_m * p.tiles_n);
+        const int m0 = (rem / p.tiles_n) * kBM, n0 = (rem % p.tiles_n) * BN;
+        const int ca = p.a_batched ? member : 0, cb = p.b_batched ? member : 0;
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+          uint8_t* sa = smem + stage * L::kStageBytes;
+          uint8_t* sb = sa + L::kABytes;
+          mbar_expect_tx(&full[stage], L::kStageBytes);
+          const int k0 = kb * kBK;
+          if (!p.a_mn) {
+            tma_load_3d(sa, &tmA, &full[stage], k0, m0, ca);
+          } else {
+#pragma unroll
+            for (int j = 0; j < kBM / 64; ++j) tma_load_3d(sa + j * 8192, &tmA, &full[stage], m0 + j * 64, k0, ca);
+          }
+          if (!p.b_mn) {
+            tma_load_3d(sb, &tmB, &full[stage], k0, n0, cb);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j) tma_load_3d(sb + j * 8192, &tmB, &full[stage], n0 + j * 64, k0, cb);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicCAS(&p.counters->status, 0, PBT_ERR_TIMEOUT);
+        p.counters->status_info = 1;
+      }
+      // drain: every stage this thread armed must have landed before the CTA may exit; the
+      // consumer's commits are what flips `empty`, so wait (bounded) for the last STAGES of them
+      for (int s = 0; s < STAGES && ok; ++s) {
+        // a stage is idle once its `empty` phase matches the producer's next expectation
+        if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) break;
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
+                             ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+      uint32_t stage = 0, phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++it) {
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1;
+        if (!mbar_wait(&tempty[acc], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + acc * BN;
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          const uint32_t sb = sa + L::kABytes;
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) {
+            // K-major: 16 elements of K are 32 bytes inside the swizzled 128-byte row; 8-row groups 1024 B apart.
+            // MN-major: 16 rows of K are 2048 bytes; 64-element column blocks 8192 B apart, 8-row groups 1024 B.
+            const uint64_t ad = p.a_mn ? smem_desc(sa + k * 2048, 8192, 1024) : smem_desc(sa + k * 32, 16, 1024);
+            const uint64_t bd = p.b_mn ? smem_desc(sb + k * 2048, 8192, 1024) : smem_desc(sb + k * 32, 16, 1024);
+            umma_bf16(tmem_d, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(&empty[stage]);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) umma_commit(&tfull[acc]);
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicCAS(&p.counters->status, 0, PBT_ERR_TIMEOUT);
+        p.counters->status_info = 2;
+      }
+    }
+  } else {
+    // ------------------------------ epilogue ------------------------------
+    const int q = warp & 3;  // TMEM lane quadrant this warp may access
+    int it = 0;
+    bool ok = true;
+    const bool vec_ok = (((uintptr_t)p.C & 15) == 0) &&
+                        ((p.ldc * (p.out_dtype == kBF16 ? 2 : 4)) % 16 == 0) &&
+                        ((p.strideC * (p.out_dtype == kBF16 ? 2 : 4)) % 16 == 0) &&
+                        (!p.mask || ((((uintptr_t)p.mask & 15) == 0) && (p.ldmask % 8 == 0) && (p.strideMask % 8 == 0)));
+    for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++it) {
+      const int member = tile / (p.tiles_m * p.tiles_n);
+      const int rem = tile % (p.tiles_m * p.tiles_n);
+      const int m0 = (rem / p.tiles_n) * kBM, n0 = (rem % p.tiles_n) * BN;
+      const int acc = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1;
+      if (!mbar_wait(&tfull[acc], acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row = m0 + q * 32 + lane;
+      const float* bias = p.bias ? p.bias + member * p.strideBias : nullptr;
+      const bf16* mrow = p.mask ? p.mask + member * p.strideMask + (long long)row * p.ldmask : nullptr;
+      const long long crow = member * p.strideC + (long long)row * p.ldc;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        if (n0 + c0 >= p.N) break;  // uniform across the warp
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), r);
+        if (row < p.M) {
+          const int nbase = n0 + c0;
+          const bool full_chunk = vec_ok && nbase + 32 <= p.N;
+          float v[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+          if (bias) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) if (nbase + j < p.N) v[j] += __ldg(bias + nbase + j);
+          }
+          if (p.relu) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+          }
+          if (mrow) {
+            if (full_chunk) {
+              const uint4* mp = reinterpret_cast<const uint4*>(mrow + nbase);
+#pragma unroll
+              for (int g4 = 0; g4 < 4; ++g4) {
+                const uint4 mv = __ldg(mp + g4);
+                const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  // bf16 > 0  <=>  sign bit clear and magnitude non-zero
+                  const uint32_t lo = w[e] & 0xFFFFu, hi = w[e] >> 16;
+                  if (!(lo != 0 && lo < 0x8000u)) v[g4 * 8 + e * 2] = 0.f;
+                  if (!(hi != 0 && hi < 0x8000u)) v[g4 * 8 + e * 2 + 1] = 0.f;
+                }
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (nbase + j < p.N && !(__bfloat162float(mrow[nbase + j]) > 0.f)) v[j] = 0.f;
+            }
+          }
+          if (p.out_dtype == kBF16) {
+            bf16* cp = reinterpret_cast<bf16*>(p.C) + crow + nbase;
+            if (full_chunk) {
+#pragma unroll
+              for (int g4 = 0; g4 < 4; ++g4) {
+                uint4 o;
+                __nv_bfloat162 t0 = __floats2bfloat162_rn(v[g4 * 8 + 0], v[g4 * 8 + 1]);
+                __nv_bfloat162 t1 = __floats2bfloat162_rn(v[g4 * 8 + 2], v[g4 * 8 + 3]);
+                __nv_bfloat162 t2 = __floats2bfloat162_rn(v[g4 * 8 + 4], v[g4 * 8 + 5]);
+                __nv_bfloat162 t3 = __floats2bfloat162_rn(v[g4 * 8 + 6], v[g4 * 8 + 7]);
+                o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
+                o.z = *reinterpret_cast<uint32_t*>(&t2); o.w = *reinterpret_cast<uint32_t*>(&t3);
+                reinterpret_cast<uint4*>(cp)[g4] = o;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) if (nbase + j < p.N) cp[j] = __float2bfloat16_rn(v[j]);
+            }
+          } else {
+            float* cp = reinterpret_cast<float*>(p.C) + crow + nbase;
+            if (full_chunk) {
+#pragma unroll
+              for (int g4 = 0; g4 < 8; ++g4)
+                reinterpret_cast<float4*>(cp)[g4] = make_float4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) if (nbase + j < p.N) cp[j] = v[j];
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[acc]);
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      atomicCAS(&p.counters->status, 0, PBT_ERR_TIMEOUT);
+      p.counters->status_info = 3;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// 3-D map over a row-major [batch][rows][cols] bf16 tensor (cols contiguous); box = {64, box_rows, 1}
+bool make_map(CUtensorMap* map, const void* base, long long cols, long long rows, long long ld, long long batch,
+              long long batch_stride, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)batch};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)(batch > 1 ? batch_stride : rows * ld) * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+template <int BN, int STAGES>
+cudaError_t launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, TcParams& p, cudaStream_t s) {
+  using L = Smem<BN, STAGES>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  p.tiles_n = (p.N + BN - 1) / BN;
+  p.num_tiles = p.tiles_m * p.tiles_n * p.batch;
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms <= 0) sms = 148;
+  }
+  const int grid = p.num_tiles < sms ? p.num_tiles : sms;
+  k_gemm_tc<BN, STAGES><<<grid, kThreads, L::kTotal, s>>>(tmA, tmB, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool gemm_tc_supported(const GemmArgs& g) {
+  if (g.in_dtype != kBF16) return false;
+  if (g.M < 128 || g.N < 128 || g.K < 64 || g.batch < 1) return false;  // every TMA box fits inside its tensor
+  if (g.lda % 8 || g.ldb % 8) return false;
+  if (g.batch > 1 && ((g.strideA != 0 && g.strideA % 8) || (g.strideB != 0 && g.strideB % 8))) return false;
+  if (((uintptr_t)g.A & 15) || ((uintptr_t)g.B & 15)) return false;
+  return encode_fn() != nullptr;
+}
+
+cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s) {
+  TcParams p;
+  p.M = g.M; p.N = g.N; p.K = g.K; p.batch = g.batch;
+  p.tiles_m = (g.M + kBM - 1) / kBM;
+  p.k_blocks = (g.K + kBK - 1) / kBK;
+  p.a_mn = g.a_mn; p.b_mn = g.b_mn;
+  p.a_batched = (g.batch > 1 && g.strideA != 0) ? 1 : 0;
+  p.b_batched = (g.batch > 1 && g.strideB != 0) ? 1 : 0;
+  p.C = g.C; p.ldc = g.ldc; p.strideC = g.strideC; p.out_dtype = g.out_dtype;
+  p.bias = g.bias; p.strideBias = g.strideBias; p.relu = g.relu;
+  p.mask = reinterpret_cast<const bf16*>(g.mask); p.ldmask = g.ldmask; p.strideMask = g.strideMask;
+  p.counters = counters;
+  const int BN = g.N >= 256 ? 256 : 128;
+  CUtensorMap tmA, tmB;
+  bool ok;
+  // K-major operand: rows = M (or N), cols = K.  MN-major operand: rows = K, cols = M (or N), boxes of 64 x 64.
+  if (!g.a_mn) ok = make_map(&tmA, g.A, g.K, g.M, g.lda, p.a_batched ? g.batch : 1, g.strideA, kBM);
+  else ok = make_map(&tmA, g.A, g.M, g.K, g.lda, p.a_batched ? g.batch : 1, g.strideA, kBK);
+  if (!ok) return cudaErrorInvalidValue;
+  if (!g.b_mn) ok = make_map(&tmB, g.B, g.K, g.N, g.ldb, p.b_batched ? g.batch : 1, g.strideB, BN);
+  else ok = make_map(&tmB, g.B, g.N, g.K, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kBK);
+  if (!ok) return cudaErrorInvalidValue;
+  if (BN == 256) return launch_cfg<256, 4>(tmA, tmB, p, s);
+  return launch_cfg<128, 6>(tmA, tmB, p, s);
+}
+
+}  // namespace pbt

@@ -990,6 +990,31 @@ int pbt_step_host(pbt_t* p, const void* x_host, const void* y_host, double* loss
   return PBT_OK;
 }
 
+int pbt_grouped_gemm(const pbt_gemm_desc* d, void* stream) {
+  if (!d || !d->A || !d->B || !d->C) return fail(nullptr, PBT_ERR_INVALID_ARG, "NULL argument");
+  if (d->M < 1 || d->N < 1 || d->K < 0 || d->batch < 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "bad GEMM shape");
+  GemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.M = d->M; g.N = d->N; g.K = d->K; g.batch = d->batch;
+  g.in_dtype = d->in_bf16 ? kBF16 : kF32; g.out_dtype = d->out_bf16 ? kBF16 : kF32;
+  g.A = d->A; g.lda = d->lda; g.strideA = d->strideA; g.a_mn = d->a_mn;
+  g.B = d->B; g.ldb = d->ldb; g.strideB = d->strideB; g.b_mn = d->b_mn;
+  g.C = d->C; g.ldc = d->ldc; g.strideC = d->strideC;
+  g.bias = d->bias; g.strideBias = d->strideBias; g.relu = d->relu;
+  g.mask = d->mask; g.ldmask = d->ldmask; g.strideMask = d->strideMask;
+  const bool tc = gemm_tc_supported(g);
+  cudaError_t e;
+  if (d->engine == 2 || (d->engine == 0 && tc && d->status_device)) {
+    if (!tc) return fail(nullptr, PBT_ERR_UNSUPPORTED, "shape / alignment does not qualify for the tensor-core kernel");
+    if (!d->status_device) return fail(nullptr, PBT_ERR_INVALID_ARG, "status_device is required by the tensor-core kernel");
+    e = launch_gemm_tc(g, (Counters*)d->status_device, (cudaStream_t)stream);
+  } else {
+    e = launch_gemm_simt(g, (cudaStream_t)stream);
+  }
+  if (e != cudaSuccess) return fail(nullptr, PBT_ERR_CUDA, "grouped GEMM launch: %s", cudaGetErrorString(e));
+  return PBT_OK;
+}
+
 int pbt_get_launch_count(const pbt_t* p, int64_t* count) {
   if (!p || !count) return fail(nullptr, PBT_ERR_INVALID_ARG, "NULL argument");
   *count = p->launches;
