@@ -186,6 +186,7 @@ def main():
     ap.add_argument("--workload", default="c5")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--members", type=int, default=0, help="override the population size (profiling a small case)")
     ap.add_argument("--pool-rows", type=int, default=0, help="override the training-pool size (default: the workload's)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -194,6 +195,8 @@ def main():
     cfg = get_config(args.workload)
     if args.pool_rows:
         cfg = cfg.replace(pool_rows=args.pool_rows)
+    if args.members:
+        cfg = cfg.replace(n_members=args.members, name=f"{cfg.name}[members={args.members}]")
 
     if args.impl == "reference":
         if args.steps == 50:
