@@ -107,7 +107,8 @@ typedef struct pbt_spec {
   uint32_t perturb_mask; /* bit k set: explore may perturb slot k */
   uint32_t flags;        /* PBT_COPY_WEIGHTS | PBT_COPY_HPARAMS | PBT_EXPLORE */
   int32_t trunc_num, trunc_den; /* truncation fraction, 1/5 in the paper */
-  int32_t reserved0;
+  int32_t keep_grad; /* 1: weight gradients are also stored (pbt_get_state .grad is then valid for every tensor);
+                        0: layers whose Adam update is fused into the weight-gradient GEMM never write theirs */
   double const_lr, const_momentum, const_beta1, const_beta2, const_eps, const_wd;
   double toy_eta;                 /* toy step size */
   double toy_theta0[PBT_MAX_NH];  /* toy initial theta (same for all members) */

@@ -8,11 +8,15 @@
 //               into a ring of shared-memory stages guarded by full/empty mbarriers; plain per-CTA loads
 //   warp 1      allocates tensor memory, one elected lane issues tcgen05.mma (128 x BN x 16 per
 //               instruction, fp32 accumulators in TMEM), tcgen05.commit frees the stage / publishes the tile
-//   warps 2..5  epilogue: tcgen05.ld of the accumulator (double-buffered in TMEM, so the next tile's
-//               main loop overlaps), bias / ReLU / ReLU-mask, conversion, 16-byte global stores
+//   warps 2..   epilogue (4 or 8 warps): tcgen05.ld of the accumulator (double-buffered in TMEM, so the next
+//               tile's main loop overlaps), a 32 x 32 transpose through padded shared memory so that global
+//               accesses are whole 128-byte lines, then either bias / ReLU / ReLU-mask / conversion, or --
+//               for weight gradients -- the member's Adam update applied in place (the gradient never
+//               goes to HBM unless asked for)
 // Every mbarrier wait is bounded; on expiry the kernel records PBT_ERR_TIMEOUT in the device status
 // word, all roles leave their loops, tensor memory is released and the kernel returns normally.
 #include <cuda.h>
+#include <string.h>
 
 #include "pbt_common.cuh"
 
@@ -22,7 +26,7 @@ namespace {
 
 constexpr int kBM = 128;
 constexpr int kBK = 64;
-constexpr int kThreads = 192;
+constexpr int kEpiPitch = 36;  // floats per row of the epilogue transpose buffer (16-byte aligned, conflict-free)
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 struct TcParams {
@@ -33,6 +37,7 @@ struct TcParams {
   const float* bias; long long strideBias; int relu;
   const bf16* mask; long long ldmask, strideMask;
   Counters* counters;
+  OptArgs opt;  // fused Adam epilogue only
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
@@ -125,19 +130,23 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
   return d;
 }
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, int NEPIW>
 struct Smem {
   static constexpr int kABytes = kBM * kBK * 2;
   static constexpr int kBBytes = BN * kBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kBarOffset = STAGES * kStageBytes;
+  static constexpr int kEpiOffset = STAGES * kStageBytes;
+  static constexpr int kEpiBytesPerWarp = 32 * kEpiPitch * 4;
+  static constexpr int kBarOffset = kEpiOffset + NEPIW * kEpiBytesPerWarp;
   static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack for 1024-byte alignment
+  static_assert(kTotal <= 232448, "shared memory budget of one CTA");
 };
 
-template <int BN, int STAGES>
-__global__ void __launch_bounds__(kThreads, 1)
+// EPI 0: C = epilogue(acc).  EPI 1: acc is a weight gradient; Adam update of the member's slab in place.
+template <int BN, int STAGES, int EPI, int NEPIW>
+__global__ void __launch_bounds__(64 + 32 * NEPIW, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
-  using L = Smem<BN, STAGES>;
+  using L = Smem<BN, STAGES, NEPIW>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
@@ -151,7 +160,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], NEPIW); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -246,13 +255,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     }
   } else {
     // ------------------------------ epilogue ------------------------------
-    const int q = warp & 3;  // TMEM lane quadrant this warp may access
+    const int q = warp & 3;            // TMEM lane quadrant this warp may access
+    const int e = warp - 2;            // 0 .. NEPIW-1
+    const int half = e >> 2;           // with 8 warps two warps share a quadrant and alternate 32-column chunks
+    float* buf = reinterpret_cast<float*>(smem + L::kEpiOffset + e * L::kEpiBytesPerWarp);
     int it = 0;
     bool ok = true;
-    const bool vec_ok = (((uintptr_t)p.C & 15) == 0) &&
-                        ((p.ldc * (p.out_dtype == kBF16 ? 2 : 4)) % 16 == 0) &&
-                        ((p.strideC * (p.out_dtype == kBF16 ? 2 : 4)) % 16 == 0) &&
-                        (!p.mask || ((((uintptr_t)p.mask & 15) == 0) && (p.ldmask % 8 == 0) && (p.strideMask % 8 == 0)));
+    const int esz = p.out_dtype == kBF16 ? 2 : 4;
+    const bool vec_ok = EPI == 1 ? (p.ldc % 4 == 0)
+                                 : ((((uintptr_t)p.C & 15) == 0) && ((p.ldc * esz) % 16 == 0) && ((p.strideC * esz) % 16 == 0) &&
+                                    (!p.mask || ((((uintptr_t)p.mask & 7) == 0) && (p.ldmask % 4 == 0) && (p.strideMask % 4 == 0))) &&
+                                    (!p.bias || ((((uintptr_t)p.bias & 15) == 0) && (p.strideBias % 4 == 0))));
+    const int rsub = lane >> 3, cc = (lane & 7) * 4;   // phase 2: 4 rows x 8 column-quads per warp instruction
     for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++it) {
       const int member = tile / (p.tiles_m * p.tiles_n);
       const int rem = tile % (p.tiles_m * p.tiles_n);
@@ -261,77 +275,144 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       const uint32_t acc_phase = (it >> 1) & 1;
       if (!mbar_wait(&tfull[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const int row = m0 + q * 32 + lane;
+      // per-member optimiser constants (fused mode)
+      float lr = 0.f, b1 = 0.f, omb1 = 0.f, b2 = 0.f, omb2 = 0.f, inv_bc1 = 0.f, inv_bc2 = 0.f, eps = 0.f, lrwd = 0.f;
+      if (EPI == 1) {
+        const float* Hrow = p.opt.H + (long long)member * p.opt.nh_stride;
+        lr = hp(Hrow, p.opt.slot_lr, p.opt.const_lr);
+        b1 = hp(Hrow, p.opt.slot_beta1, p.opt.const_beta1);
+        const float wd = hp(Hrow, p.opt.slot_wd, p.opt.const_wd);
+        b2 = p.opt.const_beta2; eps = p.opt.const_eps;
+        const float c1 = __fmul_rn(p.opt.scalars[member * PBT_N_SCALARS + p.opt.scalar_base + 0], b1);
+        const float c2 = __fmul_rn(p.opt.scalars[member * PBT_N_SCALARS + p.opt.scalar_base + 1], b2);
+        inv_bc1 = 1.f / (1.f - c1); inv_bc2 = 1.f / (1.f - c2);
+        omb1 = 1.f - b1; omb2 = 1.f - b2; lrwd = lr * wd;
+      }
       const float* bias = p.bias ? p.bias + member * p.strideBias : nullptr;
-      const bf16* mrow = p.mask ? p.mask + member * p.strideMask + (long long)row * p.ldmask : nullptr;
-      const long long crow = member * p.strideC + (long long)row * p.ldc;
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        if (n0 + c0 >= p.N) break;  // uniform across the warp
-        uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), r);
-        if (row < p.M) {
-          const int nbase = n0 + c0;
-          const bool full_chunk = vec_ok && nbase + 32 <= p.N;
-          float v[32];
+      for (int c0 = half * 32; c0 < BN; c0 += 32 * (NEPIW / 4)) {
+        const int nbase = n0 + c0;
+        if (nbase >= p.N) break;  // uniform across the warp
+        {
+          uint32_t r[32];
+          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), r);
+          __syncwarp();  // the previous chunk's phase-2 reads of `buf` are complete
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-          if (bias) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) if (nbase + j < p.N) v[j] += __ldg(bias + nbase + j);
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<uint4*>(&buf[lane * kEpiPitch + j * 4]) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+          __syncwarp();
+        }
+        const int col = nbase + cc;
+        const bool full4 = vec_ok && col + 3 < p.N;
+        if (EPI == 0) {
+          float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (bias && col < p.N) {
+            if (full4) bv = __ldg(reinterpret_cast<const float4*>(bias + col));
+            else {
+              bv.x = bias[col];
+              if (col + 1 < p.N) bv.y = bias[col + 1];
+              if (col + 2 < p.N) bv.z = bias[col + 2];
+              if (col + 3 < p.N) bv.w = bias[col + 3];
+            }
           }
-          if (p.relu) {
+#pragma unroll 4
+          for (int i = 0; i < 8; ++i) {
+            const int rr = i * 4 + rsub;
+            const int row = m0 + q * 32 + rr;
+            if (row >= p.M || col >= p.N) continue;
+            const float4 a4 = *reinterpret_cast<const float4*>(&buf[rr * kEpiPitch + cc]);
+            float v[4] = {a4.x + bv.x, a4.y + bv.y, a4.z + bv.z, a4.w + bv.w};
+            if (p.relu) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
-          }
-          if (mrow) {
-            if (full_chunk) {
-              const uint4* mp = reinterpret_cast<const uint4*>(mrow + nbase);
+              for (int j = 0; j < 4; ++j) v[j] = fmaxf(v[j], 0.f);
+            }
+            if (p.mask) {
+              const bf16* mp = p.mask + member * p.strideMask + (long long)row * p.ldmask + col;
+              if (full4) {
+                const uint2 mv = __ldg(reinterpret_cast<const uint2*>(mp));
+                const uint32_t w[2] = {mv.x, mv.y};
 #pragma unroll
-              for (int g4 = 0; g4 < 4; ++g4) {
-                const uint4 mv = __ldg(mp + g4);
-                const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
+                for (int h2 = 0; h2 < 2; ++h2) {
                   // bf16 > 0  <=>  sign bit clear and magnitude non-zero
-                  const uint32_t lo = w[e] & 0xFFFFu, hi = w[e] >> 16;
-                  if (!(lo != 0 && lo < 0x8000u)) v[g4 * 8 + e * 2] = 0.f;
-                  if (!(hi != 0 && hi < 0x8000u)) v[g4 * 8 + e * 2 + 1] = 0.f;
+                  const uint32_t lo = w[h2] & 0xFFFFu, hi = w[h2] >> 16;
+                  if (!(lo != 0 && lo < 0x8000u)) v[h2 * 2] = 0.f;
+                  if (!(hi != 0 && hi < 0x8000u)) v[h2 * 2 + 1] = 0.f;
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                  if (col + j < p.N && !(__bfloat162float(mp[j]) > 0.f)) v[j] = 0.f;
+              }
+            }
+            const long long ci = member * p.strideC + (long long)row * p.ldc + col;
+            if (p.out_dtype == kBF16) {
+              bf16* cp = reinterpret_cast<bf16*>(p.C) + ci;
+              if (full4) {
+                __nv_bfloat162 t0 = __floats2bfloat162_rn(v[0], v[1]);
+                __nv_bfloat162 t1 = __floats2bfloat162_rn(v[2], v[3]);
+                uint2 o;
+                o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
+                *reinterpret_cast<uint2*>(cp) = o;
+              } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) if (col + j < p.N) cp[j] = __float2bfloat16_rn(v[j]);
+              }
+            } else {
+              float* cp = reinterpret_cast<float*>(p.C) + ci;
+              if (full4) *reinterpret_cast<float4*>(cp) = make_float4(v[0], v[1], v[2], v[3]);
+              else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) if (col + j < p.N) cp[j] = v[j];
+              }
+            }
+          }
+        } else {
+          // fused Adam: element (row, col) of this layer's weight matrix lives at begin + row*ldc + col of the slab
+          const long long slab = (long long)member * p.opt.p_pad + p.opt.begin;
+          float* gout = reinterpret_cast<float*>(p.C);
+#pragma unroll 1
+          for (int i0 = 0; i0 < 8; i0 += 4) {
+            float4 ww[4], aa[4], bb[4];
+            bool live[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int rr = (i0 + u) * 4 + rsub;
+              const int row = m0 + q * 32 + rr;
+              live[u] = row < p.M && full4;
+              if (live[u]) {
+                const long long off = slab + (long long)row * p.ldc + col;
+                ww[u] = ld_stream(p.opt.w32 + off);
+                aa[u] = ld_stream(p.opt.opt1 + off);
+                bb[u] = ld_stream(p.opt.opt2 + off);
+              }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int rr = (i0 + u) * 4 + rsub;
+              const int row = m0 + q * 32 + rr;
+              const float4 g4 = *reinterpret_cast<const float4*>(&buf[rr * kEpiPitch + cc]);
+              const long long off = slab + (long long)row * p.ldc + col;
+              if (live[u]) {
+                float4 nw;
+                nw.x = adam_one(ww[u].x, aa[u].x, bb[u].x, g4.x, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
+                nw.y = adam_one(ww[u].y, aa[u].y, bb[u].y, g4.y, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
+                nw.z = adam_one(ww[u].z, aa[u].z, bb[u].z, g4.z, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
+                nw.w = adam_one(ww[u].w, aa[u].w, bb[u].w, g4.w, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
+                st_stream(p.opt.opt1 + off, aa[u]);
+                st_stream(p.opt.opt2 + off, bb[u]);
+                st_stream(p.opt.w32 + off, nw);
+                if (p.opt.w16) st_bf16x4(p.opt.w16 + off, nw);
+                if (gout) st_stream(gout + member * p.strideC + (long long)row * p.ldc + col, g4);
+              } else if (row < p.M && col < p.N) {
+                const float gs[4] = {g4.x, g4.y, g4.z, g4.w};
+                for (int j = 0; j < 4 && col + j < p.N; ++j) {
+                  float m1 = p.opt.opt1[off + j], m2 = p.opt.opt2[off + j];
+                  const float nw = adam_one(p.opt.w32[off + j], m1, m2, gs[j], b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
+                  p.opt.opt1[off + j] = m1; p.opt.opt2[off + j] = m2; p.opt.w32[off + j] = nw;
+                  if (p.opt.w16) p.opt.w16[off + j] = __float2bfloat16_rn(nw);
+                  if (gout) gout[member * p.strideC + (long long)row * p.ldc + col + j] = gs[j];
                 }
               }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (nbase + j < p.N && !(__bfloat162float(mrow[nbase + j]) > 0.f)) v[j] = 0.f;
-            }
-          }
-          if (p.out_dtype == kBF16) {
-            bf16* cp = reinterpret_cast<bf16*>(p.C) + crow + nbase;
-            if (full_chunk) {
-#pragma unroll
-              for (int g4 = 0; g4 < 4; ++g4) {
-                uint4 o;
-                __nv_bfloat162 t0 = __floats2bfloat162_rn(v[g4 * 8 + 0], v[g4 * 8 + 1]);
-                __nv_bfloat162 t1 = __floats2bfloat162_rn(v[g4 * 8 + 2], v[g4 * 8 + 3]);
-                __nv_bfloat162 t2 = __floats2bfloat162_rn(v[g4 * 8 + 4], v[g4 * 8 + 5]);
-                __nv_bfloat162 t3 = __floats2bfloat162_rn(v[g4 * 8 + 6], v[g4 * 8 + 7]);
-                o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
-                o.z = *reinterpret_cast<uint32_t*>(&t2); o.w = *reinterpret_cast<uint32_t*>(&t3);
-                reinterpret_cast<uint4*>(cp)[g4] = o;
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) if (nbase + j < p.N) cp[j] = __float2bfloat16_rn(v[j]);
-            }
-          } else {
-            float* cp = reinterpret_cast<float*>(p.C) + crow + nbase;
-            if (full_chunk) {
-#pragma unroll
-              for (int g4 = 0; g4 < 8; ++g4)
-                reinterpret_cast<float4*>(cp)[g4] = make_float4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) if (nbase + j < p.N) cp[j] = v[j];
             }
           }
         }
@@ -385,12 +466,12 @@ bool make_map(CUtensorMap* map, const void* base, long long cols, long long rows
   return r == CUDA_SUCCESS;
 }
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, int EPI, int NEPIW>
 cudaError_t launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, TcParams& p, cudaStream_t s) {
-  using L = Smem<BN, STAGES>;
+  using L = Smem<BN, STAGES, NEPIW>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<BN, STAGES, EPI, NEPIW>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -404,7 +485,7 @@ cudaError_t launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, TcParams&
     if (sms <= 0) sms = 148;
   }
   const int grid = p.num_tiles < sms ? p.num_tiles : sms;
-  k_gemm_tc<BN, STAGES><<<grid, kThreads, L::kTotal, s>>>(tmA, tmB, p);
+  k_gemm_tc<BN, STAGES, EPI, NEPIW><<<grid, 64 + 32 * NEPIW, L::kTotal, s>>>(tmA, tmB, p);
   return cudaGetLastError();
 }
 
@@ -431,6 +512,8 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s
   p.bias = g.bias; p.strideBias = g.strideBias; p.relu = g.relu;
   p.mask = reinterpret_cast<const bf16*>(g.mask); p.ldmask = g.ldmask; p.strideMask = g.strideMask;
   p.counters = counters;
+  memset(&p.opt, 0, sizeof(p.opt));
+  if (g.adam) p.opt = *g.adam;
   const int BN = g.N >= 256 ? 256 : 128;
   CUtensorMap tmA, tmB;
   bool ok;
@@ -441,8 +524,13 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s
   if (!g.b_mn) ok = make_map(&tmB, g.B, g.K, g.N, g.ldb, p.b_batched ? g.batch : 1, g.strideB, BN);
   else ok = make_map(&tmB, g.B, g.N, g.K, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kBK);
   if (!ok) return cudaErrorInvalidValue;
-  if (BN == 256) return launch_cfg<256, 4>(tmA, tmB, p, s);
-  return launch_cfg<128, 6>(tmA, tmB, p, s);
+  if (g.adam) {
+    // epilogue-bound (26 bytes of HBM traffic per output element): 8 epilogue warps, shallower ring
+    if (BN == 256) return launch_cfg<256, 3, 1, 8>(tmA, tmB, p, s);
+    return launch_cfg<128, 4, 1, 8>(tmA, tmB, p, s);
+  }
+  if (BN == 256) return launch_cfg<256, 4, 0, 4>(tmA, tmB, p, s);
+  return launch_cfg<128, 6, 0, 4>(tmA, tmB, p, s);
 }
 
 }  // namespace pbt

@@ -10,30 +10,6 @@
 
 namespace pbt {
 
-__device__ __forceinline__ float hp(const float* __restrict__ Hrow, int slot, float fallback) {
-  return slot >= 0 ? Hrow[slot] : fallback;
-}
-
-__device__ __forceinline__ float4 ld_stream(const float* p) {
-  // read-once data: bypass L1 allocation
-  float4 v;
-  asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-               : "l"(p));
-  return v;
-}
-__device__ __forceinline__ void st_stream(float* p, float4 v) {
-  asm volatile("st.global.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
-}
-__device__ __forceinline__ void st_bf16x4(bf16* p, float4 v) {
-  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
-  __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
-  uint2 u;
-  u.x = *reinterpret_cast<uint32_t*>(&lo);
-  u.y = *reinterpret_cast<uint32_t*>(&hi);
-  *reinterpret_cast<uint2*>(p) = u;
-}
-
 constexpr int kOptThreads = 256;
 constexpr int kOptVecPerThread = 2;                              // float4 per stream per thread per iteration
 constexpr int kOptTile = kOptThreads * kOptVecPerThread * 4;     // elements per block iteration
@@ -66,17 +42,6 @@ __global__ void __launch_bounds__(kOptThreads) k_sgdm(OptArgs a) {
       }
     }
   }
-}
-
-__device__ __forceinline__ float adam_one(float w, float& m1, float& m2, float g, float b1, float omb1, float b2,
-                                          float omb2, float inv_bc1, float inv_bc2, float lr, float eps,
-                                          float lrwd) {
-  m1 = __fmaf_rn(b1, m1, omb1 * g);
-  m2 = __fmaf_rn(b2, m2, omb2 * g * g);
-  const float mhat = m1 * inv_bc1;
-  const float vhat = m2 * inv_bc2;
-  const float upd = __fdividef(mhat, sqrtf(vhat) + eps);
-  return w - lr * upd - lrwd * w;
 }
 
 // m <- b1 m + (1-b1) g ; v <- b2 v + (1-b2) g^2 ;

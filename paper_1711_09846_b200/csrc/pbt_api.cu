@@ -340,27 +340,36 @@ int forward(pbt_handle* h, int k, int rows, const void* in, long long in_stride)
   return PBT_OK;
 }
 
+void fill_opt_args(pbt_handle* h, OptArgs* a, int slot_lr, int scalar_base) {
+  const pbt_spec& s = h->spec;
+  memset(a, 0, sizeof(*a));
+  a->n_members = h->N; a->p_pad = h->P_pad;
+  a->w32 = h->W32; a->opt1 = h->O1; a->opt2 = h->O2; a->grad = h->G; a->w16 = h->W16;
+  a->H = (const float*)h->H; a->nh_stride = PBT_MAX_NH;
+  a->slot_lr = slot_lr; a->slot_momentum = s.slot_momentum; a->slot_beta1 = s.slot_beta1; a->slot_wd = s.slot_wd;
+  a->const_lr = (float)s.const_lr; a->const_momentum = (float)s.const_momentum; a->const_beta1 = (float)s.const_beta1;
+  a->const_beta2 = (float)s.const_beta2; a->const_eps = (float)s.const_eps; a->const_wd = (float)s.const_wd;
+  a->scalars = h->scalars; a->scalar_base = scalar_base;
+}
+
 // dW_l = dZ_l^T a_{l-1}, db_l = column sums of dZ_l, dZ_{l-1} = (dZ_l W_l) * [a_{l-1} > 0].
 // dZ of the last layer is in h->dz[*cur]; on return *cur names the buffer written last.
+// With need_wgrad the optimiser update of the stack is part of this pass: layers whose weight
+// gradient runs on the tensor cores get their Adam update inside that GEMM's epilogue (after the
+// layer's data gradient has read the old weights); everything else (biases, skinny layers,
+// SGD-momentum) is updated by the element-wise kernel over the remaining slab ranges.
 int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride, bool need_wgrad,
-             bool need_input_grad, int* cur) {
+             bool need_input_grad, int* cur, int slot_lr, int scalar_base) {
   const Stack& st = h->st[k];
+  const pbt_spec& s = h->spec;
   const long long dzs = dz_stride(h);
+  OptArgs opt;
+  fill_opt_args(h, &opt, slot_lr, scalar_base);
+  bool fused[PBT_MAX_LAYERS] = {false};
   for (int l = st.nl - 1; l >= 0; --l) {
     const Layer& L = st.L[l];
     const void* dz = h->dz[*cur];
-    if (need_wgrad) {
-      GemmArgs g;
-      memset(&g, 0, sizeof(g));
-      g.M = L.out; g.N = L.in; g.K = rows; g.batch = h->N;
-      g.in_dtype = h->cdt; g.out_dtype = kF32;
-      g.A = dz; g.lda = L.out; g.strideA = dzs; g.a_mn = 1;
-      g.B = l == 0 ? in : h->act[k][l]; g.ldb = L.in; g.strideB = l == 0 ? in_stride : act_stride(h, k, l); g.b_mn = 1;
-      g.C = h->G + L.w_off; g.ldc = L.in; g.strideC = h->P_pad;
-      int rc = gemm(h, g);
-      if (rc) return rc;
-      LAUNCH(h, kLoss, launch_bias_grad(dz, h->cdt, L.out, dzs, rows, L.out, h->G + L.b_off, h->P_pad, h->N, h->stream));
-    }
+    bool wrote_dgrad = false;
     if (l > 0 || need_input_grad) {
       GemmArgs g;
       memset(&g, 0, sizeof(g));
@@ -372,29 +381,57 @@ int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride
       if (l > 0) { g.mask = h->act[k][l]; g.ldmask = L.in; g.strideMask = act_stride(h, k, l); }
       int rc = gemm(h, g);
       if (rc) return rc;
-      *cur = 1 - *cur;
+      wrote_dgrad = true;
     }
+    if (need_wgrad) {
+      GemmArgs g;
+      memset(&g, 0, sizeof(g));
+      g.M = L.out; g.N = L.in; g.K = rows; g.batch = h->N;
+      g.in_dtype = h->cdt; g.out_dtype = kF32;
+      g.A = dz; g.lda = L.out; g.strideA = dzs; g.a_mn = 1;
+      g.B = l == 0 ? in : h->act[k][l]; g.ldb = L.in; g.strideB = l == 0 ? in_stride : act_stride(h, k, l); g.b_mn = 1;
+      g.C = h->G + L.w_off; g.ldc = L.in; g.strideC = h->P_pad;
+      OptArgs lopt = opt;
+      if (s.optimizer == PBT_OPT_ADAM && gemm_tc_supported(g)) {
+        lopt.begin = L.w_off; lopt.count = (long long)L.in * L.out;
+        g.adam = &lopt;
+        if (!s.keep_grad) g.C = nullptr;
+        fused[l] = true;
+      }
+      int rc = gemm(h, g);
+      if (rc) return rc;
+      LAUNCH(h, kLoss, launch_bias_grad(dz, h->cdt, L.out, dzs, rows, L.out, h->G + L.b_off, h->P_pad, h->N, h->stream));
+    }
+    if (wrote_dgrad) *cur = 1 - *cur;
   }
-  return PBT_OK;
-}
-
-int optimizer(pbt_handle* h, int k, int slot_lr, int scalar_base) {
-  const pbt_spec& s = h->spec;
-  OptArgs a;
-  memset(&a, 0, sizeof(a));
-  a.n_members = h->N; a.p_pad = h->P_pad; a.begin = h->st[k].begin; a.count = h->st[k].count;
-  a.w32 = h->W32; a.opt1 = h->O1; a.opt2 = h->O2; a.grad = h->G; a.w16 = h->W16;
-  a.H = (const float*)h->H; a.nh_stride = PBT_MAX_NH;
-  a.slot_lr = slot_lr; a.slot_momentum = s.slot_momentum; a.slot_beta1 = s.slot_beta1; a.slot_wd = s.slot_wd;
-  a.const_lr = (float)s.const_lr; a.const_momentum = (float)s.const_momentum; a.const_beta1 = (float)s.const_beta1;
-  a.const_beta2 = (float)s.const_beta2; a.const_eps = (float)s.const_eps; a.const_wd = (float)s.const_wd;
-  a.scalars = h->scalars; a.scalar_base = scalar_base;
-  if (s.optimizer == PBT_OPT_SGDM) {
-    LAUNCH(h, kOpt, launch_sgdm(a, h->stream));
-  } else {
-    LAUNCH(h, kOpt, launch_adam(a, h->stream));
-    LAUNCH(h, kOther, launch_adam_advance(a, h->stream));
+  if (!need_wgrad) return PBT_OK;
+  // element-wise optimiser over what the fused epilogues did not cover; adjacent ranges are merged
+  long long rb = -1, re = -1;
+  auto flush = [&]() -> int {
+    if (rb < 0) return PBT_OK;
+    OptArgs a = opt;
+    a.begin = rb; a.count = re - rb;
+    rb = re = -1;
+    if (s.optimizer == PBT_OPT_SGDM) { LAUNCH(h, kOpt, launch_sgdm(a, h->stream)); }
+    else { LAUNCH(h, kOpt, launch_adam(a, h->stream)); }
+    return PBT_OK;
+  };
+  for (int l = 0; l < st.nl; ++l) {
+    const Layer& L = st.L[l];
+    const long long w_end = L.b_off, b_end = l + 1 < st.nl ? st.L[l + 1].w_off : st.begin + st.count;
+    if (!fused[l]) {
+      if (rb < 0) rb = L.w_off;
+      re = w_end;
+    } else {
+      int rc = flush();
+      if (rc) return rc;
+    }
+    if (rb < 0) rb = L.b_off;
+    re = b_end;
   }
+  int rc = flush();
+  if (rc) return rc;
+  if (s.optimizer == PBT_OPT_ADAM) LAUNCH(h, kOther, launch_adam_advance(opt, h->stream));
   return PBT_OK;
 }
 
@@ -439,9 +476,7 @@ int step_mlp(pbt_handle* h) {
   rc = loss_and_dz(h, 0, s.batch, s.batch, h->ybatch, h->ybatch_stride, true, 0, 1.0f / s.batch, h->last_loss, 2);
   if (rc) return rc;
   int cur = 0;
-  rc = backward(h, 0, s.batch, h->act[0][0], act_stride(h, 0, 0), true, false, &cur);
-  if (rc) return rc;
-  return optimizer(h, 0, s.slot_lr, 0);
+  return backward(h, 0, s.batch, h->act[0][0], act_stride(h, 0, 0), true, false, &cur, s.slot_lr, 0);
 }
 
 // Section 4.3.1: K discriminator updates, then one generator update.
@@ -471,16 +506,12 @@ int step_gan(pbt_handle* h) {
     if (rc) return rc;
     int cur = 0;
     if (d_phase) {
-      rc = backward(h, 1, rows, h->act[1][0], d_in_stride, true, false, &cur);
-      if (rc) return rc;
-      rc = optimizer(h, 1, s.slot_lr_d, 2);
+      rc = backward(h, 1, rows, h->act[1][0], d_in_stride, true, false, &cur, s.slot_lr_d, 2);
       if (rc) return rc;
     } else {
-      rc = backward(h, 1, rows, h->act[1][0], d_in_stride, false, true, &cur);
+      rc = backward(h, 1, rows, h->act[1][0], d_in_stride, false, true, &cur, s.slot_lr_d, 2);
       if (rc) return rc;
-      rc = backward(h, 0, B, h->act[0][0], act_stride(h, 0, 0), true, false, &cur);
-      if (rc) return rc;
-      rc = optimizer(h, 0, s.slot_lr, 0);
+      rc = backward(h, 0, B, h->act[0][0], act_stride(h, 0, 0), true, false, &cur, s.slot_lr, 0);
       if (rc) return rc;
     }
   }

@@ -61,6 +61,7 @@ struct Counters {
 // B likewise over (n,k).  Strides are in elements of the operand type.
 // ---------------------------------------------------------------------------
 enum DType : int { kF32 = 0, kBF16 = 1 };
+struct OptArgs;
 
 struct GemmArgs {
   int M, N, K, batch;
@@ -72,6 +73,10 @@ struct GemmArgs {
   const float* bias; long long strideBias;  // added per column n (may be null)
   int relu;                                 // max(., 0) after the bias
   const void* mask; long long ldmask, strideMask;  // C *= (mask[m][n] > 0), operand type (may be null)
+  // Weight-gradient GEMMs only (tensor-core path): when `adam` is set the epilogue applies the Adam update
+  // to the member's slab in place (C[m][n] is the gradient of element adam->begin + m*ldc + n) and stores the
+  // gradient itself only if C is not null.
+  const struct OptArgs* adam;
 };
 
 // launchers (each enqueues on `s` and returns the CUDA error of the launch)
@@ -93,6 +98,45 @@ struct OptArgs {
 cudaError_t launch_sgdm(const OptArgs& a, cudaStream_t s);
 cudaError_t launch_adam(const OptArgs& a, cudaStream_t s);
 cudaError_t launch_adam_advance(const OptArgs& a, cudaStream_t s);
+
+// ---- device helpers shared by the optimiser kernel and the fused weight-gradient epilogue ----
+#ifdef __CUDACC__
+__device__ __forceinline__ float hp(const float* __restrict__ Hrow, int slot, float fallback) {
+  return slot >= 0 ? Hrow[slot] : fallback;
+}
+
+__device__ __forceinline__ float4 ld_stream(const float* p) {
+  // read-once data: bypass L1 allocation
+  float4 v;
+  asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_stream(float* p, float4 v) {
+  asm volatile("st.global.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_bf16x4(bf16* p, float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+  __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u;
+  u.x = *reinterpret_cast<uint32_t*>(&lo);
+  u.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+
+__device__ __forceinline__ float adam_one(float w, float& m1, float& m2, float g, float b1, float omb1, float b2,
+                                          float omb2, float inv_bc1, float inv_bc2, float lr, float eps,
+                                          float lrwd) {
+  m1 = __fmaf_rn(b1, m1, omb1 * g);
+  m2 = __fmaf_rn(b2, m2, omb2 * g * g);
+  const float mhat = m1 * inv_bc1;
+  const float vhat = m2 * inv_bc2;
+  const float upd = __fdividef(mhat, sqrtf(vhat) + eps);
+  return w - lr * upd - lrwd * w;
+}
+
+#endif  // __CUDACC__
 
 struct SelectArgs {
   int n, nh, n_cut;

@@ -174,7 +174,8 @@ def _check_optimizer_arithmetic(cfg, s0, s1, h):
 def test_step_eval_exploit_parity(pkg, name):
     cfg = get_config(name)
     inp = make_inputs(cfg)
-    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    # keep_grad: the fused weight-gradient + Adam epilogue also stores the gradient it consumed
+    gpu, cpu = pkg.Population(cfg, inp, keep_grad=True), O.Population(cfg, inp)
     tol = _tol(cfg)
     ftol = 1e-4 if cfg.dtype == C.FP32 else 2e-2
     keys = ("w", "opt1", "grad") if cfg.optimizer == C.OPT_SGDM else ("w", "opt1", "opt2", "grad")
@@ -206,6 +207,25 @@ def test_step_eval_exploit_parity(pkg, name):
         # every step starts from identical state: training is chaotic, parity is per step
         push_oracle_state(gpu, cpu)
     gpu.close()
+
+
+@pytest.mark.parametrize("name", ["c3_mid", "c5_mid", "c4_mid", "c5_mini"])
+def test_fused_update_is_the_same_with_and_without_stored_gradients(pkg, name):
+    """The benchmarked configuration never writes the weight gradient of tensor-core layers to HBM.
+    It must produce bit-identical weights and moments to the gradient-keeping run compared above."""
+    cfg = get_config(name)
+    inp = make_inputs(cfg)
+    a, b = pkg.Population(cfg, inp, keep_grad=True), pkg.Population(cfg, inp, keep_grad=False)
+    for pop in (a, b):
+        pop.step(3)
+        pop.eval()
+    assert np.array_equal(a.fitness(), b.fitness())
+    for m in range(cfg.n_members):
+        sa, sb = a.get_state(m), b.get_state(m)
+        for key in ("w", "opt1", "opt2", "scalars"):
+            assert np.array_equal(sa[key], sb[key]), (name, m, key)
+    a.close()
+    b.close()
 
 
 def test_free_running_interval_stays_within_tolerance(pkg):
