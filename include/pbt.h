@@ -109,6 +109,10 @@ typedef struct pbt_spec {
   int32_t trunc_num, trunc_den; /* truncation fraction, 1/5 in the paper */
   int32_t keep_grad; /* 1: weight gradients are also stored (pbt_get_state .grad is then valid for every tensor);
                         0: layers whose Adam update is fused into the weight-gradient GEMM never write theirs */
+  int32_t fuse_adam; /* 1: apply Adam inside the epilogue of tensor-core weight-gradient GEMMs (the gradient of those
+                        layers never goes to HBM); 0: weight gradients are written once and one streaming pass over
+                        the slabs applies the update.  Results are bit-identical; only the traffic pattern differs. */
+  int32_t reserved1;
   double const_lr, const_momentum, const_beta1, const_beta2, const_eps, const_wd;
   double toy_eta;                 /* toy step size */
   double toy_theta0[PBT_MAX_NH];  /* toy initial theta (same for all members) */

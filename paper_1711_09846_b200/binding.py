@@ -37,7 +37,7 @@ class PbtSpec(C.Structure):
         ("slot_lr", C.c_int32), ("slot_lr_d", C.c_int32), ("slot_momentum", C.c_int32),
         ("slot_beta1", C.c_int32), ("slot_wd", C.c_int32),
         ("perturb_mask", C.c_uint32), ("flags", C.c_uint32),
-        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32),
+        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("reserved1", C.c_int32),
         ("const_lr", C.c_double), ("const_momentum", C.c_double), ("const_beta1", C.c_double),
         ("const_beta2", C.c_double), ("const_eps", C.c_double), ("const_wd", C.c_double),
         ("toy_eta", C.c_double), ("toy_theta0", C.c_double * PBT_MAX_NH),
@@ -136,7 +136,7 @@ class PbtError(RuntimeError):
         self.code = code
 
 
-def spec_from_config(cfg, keep_grad: bool = False) -> PbtSpec:
+def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = False) -> PbtSpec:
     """Translate a declarative population description (see workloads.configs.PBTConfig) into pbt_spec."""
     s = PbtSpec()
     s.n_members = cfg.n_members
@@ -164,6 +164,7 @@ def spec_from_config(cfg, keep_grad: bool = False) -> PbtSpec:
     s.flags = cfg.flags
     s.trunc_num, s.trunc_den = cfg.trunc_num, cfg.trunc_den
     s.keep_grad = 1 if keep_grad else 0
+    s.fuse_adam = 1 if fuse_adam else 0
     s.const_lr = 0.0
     s.const_momentum = cfg.momentum
     s.const_beta1, s.const_beta2, s.const_eps, s.const_wd = cfg.beta1, cfg.beta2, cfg.eps, cfg.weight_decay
@@ -236,7 +237,8 @@ def energy_fitness_static(x_dev, fitness_out_dev, stream=None) -> None:
 class Population:
     """One population living on one GPU.  Thin wrapper over the pbt_* calls."""
 
-    def __init__(self, cfg, inputs, seed: Optional[int] = None, device: str = "cuda:0", keep_grad: bool = False):
+    def __init__(self, cfg, inputs, seed: Optional[int] = None, device: str = "cuda:0", keep_grad: bool = False,
+                 fuse_adam: bool = False):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -245,7 +247,7 @@ class Population:
         self.cfg = cfg
         self.device = torch.device(device)
         self.seed = int(cfg.seed if seed is None else seed)
-        self.spec = spec_from_config(cfg, keep_grad)
+        self.spec = spec_from_config(cfg, keep_grad, fuse_adam)
         self.N, self.nh = cfg.n_members, cfg.nh
         self.toy = cfg.model == "toy_quadratic"
         torch.cuda.set_device(self.device)

@@ -26,6 +26,7 @@ namespace {
 
 constexpr int kBM = 128;
 constexpr int kBK = 64;
+constexpr int kFuseBatch = 4;  // row-quads of master / moment loads in flight per lane in the fused Adam epilogue
 constexpr int kEpiPitch = 36;  // floats per row of the epilogue transpose buffer (16-byte aligned, conflict-free)
 constexpr uint32_t kSpinLimit = 1u << 22;
 
@@ -105,6 +106,7 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// asynchronous: issue only
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -116,8 +118,9 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// the registers written by tmem_ld32 are valid only after this
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // shared-memory matrix descriptor: 128-byte swizzle, addresses / offsets in 16-byte units
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -257,7 +260,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     // ------------------------------ epilogue ------------------------------
     const int q = warp & 3;            // TMEM lane quadrant this warp may access
     const int e = warp - 2;            // 0 .. NEPIW-1
-    const int half = e >> 2;           // with 8 warps two warps share a quadrant and alternate 32-column chunks
+    const int half = e >> 2;           // warps that share a quadrant interleave over the 32-column chunks
     float* buf = reinterpret_cast<float*>(smem + L::kEpiOffset + e * L::kEpiBytesPerWarp);
     int it = 0;
     bool ok = true;
@@ -289,21 +292,35 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         omb1 = 1.f - b1; omb2 = 1.f - b2; lrwd = lr * wd;
       }
       const float* bias = p.bias ? p.bias + member * p.strideBias : nullptr;
+      // The accumulator chunk for iteration c+1 is requested from tensor memory while chunk c is being
+      // transposed and written out, and the ReLU-mask words are requested before the transpose, so that
+      // neither latency sits on the warp's critical path.
+      constexpr int kChunkStep = 32 * (NEPIW / 4);
+      uint32_t r[32];
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+      if (n0 + half * 32 < p.N) tmem_ld32(tacc + half * 32, r);
 #pragma unroll 1
-      for (int c0 = half * 32; c0 < BN; c0 += 32 * (NEPIW / 4)) {
+      for (int c0 = half * 32; c0 < BN; c0 += kChunkStep) {
         const int nbase = n0 + c0;
         if (nbase >= p.N) break;  // uniform across the warp
-        {
-          uint32_t r[32];
-          tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), r);
-          __syncwarp();  // the previous chunk's phase-2 reads of `buf` are complete
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            *reinterpret_cast<uint4*>(&buf[lane * kEpiPitch + j * 4]) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-          __syncwarp();
-        }
         const int col = nbase + cc;
         const bool full4 = vec_ok && col + 3 < p.N;
+        uint2 mk[8];
+        if (EPI == 0 && p.mask && full4) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int row = m0 + q * 32 + i * 4 + rsub;
+            mk[i] = row < p.M ? __ldg(reinterpret_cast<const uint2*>(p.mask + member * p.strideMask + (long long)row * p.ldmask + col))
+                              : make_uint2(0u, 0u);
+          }
+        }
+        tmem_ld_wait();
+        __syncwarp();  // the previous chunk's phase-2 reads of `buf` are complete
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          *reinterpret_cast<uint4*>(&buf[lane * kEpiPitch + j * 4]) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        if (c0 + kChunkStep < BN && nbase + kChunkStep < p.N) tmem_ld32(tacc + c0 + kChunkStep, r);
+        __syncwarp();
         if (EPI == 0) {
           float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
           if (bias && col < p.N) {
@@ -315,7 +332,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
               if (col + 3 < p.N) bv.w = bias[col + 3];
             }
           }
-#pragma unroll 4
+#pragma unroll
           for (int i = 0; i < 8; ++i) {
             const int rr = i * 4 + rsub;
             const int row = m0 + q * 32 + rr;
@@ -329,8 +346,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             if (p.mask) {
               const bf16* mp = p.mask + member * p.strideMask + (long long)row * p.ldmask + col;
               if (full4) {
-                const uint2 mv = __ldg(reinterpret_cast<const uint2*>(mp));
-                const uint32_t w[2] = {mv.x, mv.y};
+                const uint32_t w[2] = {mk[i].x, mk[i].y};
 #pragma unroll
                 for (int h2 = 0; h2 < 2; ++h2) {
                   // bf16 > 0  <=>  sign bit clear and magnitude non-zero
@@ -371,11 +387,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           const long long slab = (long long)member * p.opt.p_pad + p.opt.begin;
           float* gout = reinterpret_cast<float*>(p.C);
 #pragma unroll 1
-          for (int i0 = 0; i0 < 8; i0 += 4) {
-            float4 ww[4], aa[4], bb[4];
-            bool live[4];
+          for (int i0 = 0; i0 < 8; i0 += kFuseBatch) {
+            float4 ww[kFuseBatch], aa[kFuseBatch], bb[kFuseBatch];
+            bool live[kFuseBatch];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < kFuseBatch; ++u) {
               const int rr = (i0 + u) * 4 + rsub;
               const int row = m0 + q * 32 + rr;
               live[u] = row < p.M && full4;
@@ -387,7 +403,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
               }
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < kFuseBatch; ++u) {
               const int rr = (i0 + u) * 4 + rsub;
               const int row = m0 + q * 32 + rr;
               const float4 g4 = *reinterpret_cast<const float4*>(&buf[rr * kEpiPitch + cc]);
@@ -525,9 +541,16 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s
   else ok = make_map(&tmB, g.B, g.N, g.K, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kBK);
   if (!ok) return cudaErrorInvalidValue;
   if (g.adam) {
-    // epilogue-bound (26 bytes of HBM traffic per output element): 8 epilogue warps, shallower ring
+    // epilogue-bound: 26 bytes of HBM traffic per output element; 8 epilogue warps (2 per TMEM lane quadrant,
+    // interleaved over 32-column chunks)
     if (BN == 256) return launch_cfg<256, 3, 1, 8>(tmA, tmB, p, s);
     return launch_cfg<128, 4, 1, 8>(tmA, tmB, p, s);
+  }
+  // short contractions (weight gradients: K = batch) are bound by writing the tile out: more epilogue warps,
+  // shallower operand ring
+  if (p.k_blocks <= 12) {
+    if (BN == 256) return launch_cfg<256, 3, 0, 8>(tmA, tmB, p, s);
+    return launch_cfg<128, 4, 0, 8>(tmA, tmB, p, s);
   }
   if (BN == 256) return launch_cfg<256, 4, 0, 4>(tmA, tmB, p, s);
   return launch_cfg<128, 6, 0, 4>(tmA, tmB, p, s);

@@ -392,7 +392,7 @@ int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride
       g.B = l == 0 ? in : h->act[k][l]; g.ldb = L.in; g.strideB = l == 0 ? in_stride : act_stride(h, k, l); g.b_mn = 1;
       g.C = h->G + L.w_off; g.ldc = L.in; g.strideC = h->P_pad;
       OptArgs lopt = opt;
-      if (s.optimizer == PBT_OPT_ADAM && gemm_tc_supported(g)) {
+      if (s.fuse_adam && s.optimizer == PBT_OPT_ADAM && gemm_tc_supported(g)) {
         lopt.begin = L.w_off; lopt.count = (long long)L.in * L.out;
         g.adam = &lopt;
         if (!s.keep_grad) g.C = nullptr;
