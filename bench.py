@@ -186,6 +186,7 @@ def main():
     ap.add_argument("--workload", default="c5")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fuse-adam", type=int, default=-1, help="1/0: apply Adam inside the weight-gradient GEMM (default: the library's choice)")
     ap.add_argument("--members", type=int, default=0, help="override the population size (profiling a small case)")
     ap.add_argument("--pool-rows", type=int, default=0, help="override the training-pool size (default: the workload's)")
     args = ap.parse_args()
@@ -218,7 +219,8 @@ def main():
 
     import paper_1711_09846_b200 as pkg
     inp = make_inputs(cfg)
-    pop = pkg.Population(cfg, inp, device=f"cuda:{local}")
+    kw = {} if args.fuse_adam < 0 else {"fuse_adam": bool(args.fuse_adam)}
+    pop = pkg.Population(cfg, inp, device=f"cuda:{local}", **kw)
     interval = cfg.ready_interval
 
     def hot_path_step(i, launches):

@@ -301,7 +301,9 @@ struct LaunchScope {
   } while (0)
 
 int gemm(pbt_handle* h, const GemmArgs& g) {
-  if (gemm_tc_supported(g)) {
+  if (g.adam) {
+    LAUNCH(h, kGemm, launch_wgrad_adam(g, h->counters, h->stream));
+  } else if (gemm_tc_supported(g)) {
     LAUNCH(h, kGemm, launch_gemm_tc(g, h->counters, h->stream));
   } else {
     LAUNCH(h, kGemm, launch_gemm_simt(g, h->stream));
