@@ -91,29 +91,49 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def _algorithmic_work(cfg, n_params_padded=None):
-    """FLOPs of the grouped GEMMs and optimiser bytes of ONE lockstep step of the whole population."""
-    flops = 0.0
-    updates = [(0, 1)] if cfg.model != "gan_pair" else [(0, 1), (1, cfg.gan_d_steps)]
+def _tc_layer(fan_in, fan_out, rows):
+    """Layers whose weight gradient qualifies for the tensor-core kernel (the library's own rule)."""
+    return fan_in >= 128 and fan_out >= 128 and rows >= 64 and fan_in % 8 == 0 and fan_out % 8 == 0
+
+
+def _algorithmic_work(cfg):
+    """Algorithmic work of ONE lockstep step of the whole population: GEMM FLOPs, optimiser traffic."""
     B = cfg.batch
+    fused_flops = fused_params = 0.0
+    adam_bf16 = cfg.optimizer == "adam" and cfg.dtype == "bf16_fp32master"
     if cfg.model == "gan_pair":
         g, d = cfg.widths
         wg = sum(g[i] * g[i + 1] for i in range(len(g) - 1))
         wd = sum(d[i] * d[i + 1] for i in range(len(d) - 1))
         K = cfg.gan_d_steps
-        # K discriminator updates: G forward (B), D forward+wgrad on 2B rows, D dgrad above layer 0
-        flops += K * (2 * B * wg + 2 * (2 * B) * wd * 2 + 2 * (2 * B) * (wd - d[0] * d[1]))
+        # K discriminator updates: G forward (B rows), D forward + wgrad on 2B rows, D dgrad above layer 0
+        flops = K * (2 * B * wg + 2 * (2 * B) * wd * 2 + 2 * (2 * B) * (wd - d[0] * d[1]))
         # generator update: G fwd, D fwd, D dgrad to the input, G dgrad + wgrad
         flops += 2 * B * wg + 2 * B * wd + 2 * B * wd + 2 * B * (wg - g[0] * g[1]) + 2 * B * wg
-        params = {0: wg + sum(g[1:]), 1: wd + sum(d[1:])}
+        opt_params = (wg + sum(g[1:])) + K * (wd + sum(d[1:]))
+        if adam_bf16:
+            for i in range(len(g) - 1):
+                if _tc_layer(g[i], g[i + 1], B):
+                    fused_params += g[i] * g[i + 1]
+                    fused_flops += 2 * B * g[i] * g[i + 1]
+            for i in range(len(d) - 1):
+                if _tc_layer(d[i], d[i + 1], 2 * B):
+                    fused_params += K * d[i] * d[i + 1]
+                    fused_flops += K * 2 * (2 * B) * d[i] * d[i + 1]
     else:
         w = cfg.widths[0]
         W = sum(w[i] * w[i + 1] for i in range(len(w) - 1))
-        flops += 2 * B * W + 2 * B * (W - w[0] * w[1]) + 2 * B * W
-        params = {0: W + sum(w[1:])}
-    bytes_per_param = {"adam": 16 + 12, "sgdm": 12 + 8}[cfg.optimizer] + (2 if cfg.dtype == "bf16_fp32master" else 0)
-    opt_bytes = sum(params[s] * k for s, k in updates) * bytes_per_param
-    return cfg.n_members * flops, cfg.n_members * opt_bytes
+        flops = 2 * B * W + 2 * B * (W - w[0] * w[1]) + 2 * B * W
+        opt_params = W + sum(w[1:])
+        if adam_bf16:
+            for i in range(len(w) - 1):
+                if _tc_layer(w[i], w[i + 1], B):
+                    fused_params += w[i] * w[i + 1]
+                    fused_flops += 2 * B * w[i] * w[i + 1]
+    bpp = {"adam": 16 + 12, "sgdm": 12 + 8, "sgd_plain": 0}[cfg.optimizer] + (2 if cfg.dtype == "bf16_fp32master" else 0)
+    n = cfg.n_members
+    return {"flops": n * flops, "fused_flops": n * fused_flops, "fused_params": n * fused_params,
+            "opt_params": n * opt_params, "opt_bytes_per_param": bpp}
 
 
 def _cpu_count_used():
@@ -139,8 +159,7 @@ def _oracle_sample(cfg, inp, members, steps):
 
 def _oracle_budget(cfg):
     """(members, steps) of the bounded oracle sample: roughly 10-30 s of CPU work."""
-    flops, _ = _algorithmic_work(cfg)
-    per_member = flops / cfg.n_members
+    per_member = _algorithmic_work(cfg)["flops"] / cfg.n_members
     target = 10.0 * 3e10          # ~10 s at an assumed ~30 GFLOP/s effective float64 rate
     members = max(1, min(cfg.n_members, int(target // max(per_member, 1))))
     steps = max(1, min(50, int(target // max(per_member * members, 1))))
@@ -303,26 +322,30 @@ def main():
         e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                "note": "host-fed steps exist for MLP populations only"}
 
-    # ---- roofline of the dominant kernel class, from the events recorded inside the timed region ----
+    # ---- roofline per kernel class, from the CUDA events recorded inside the timed region ----
     peaks = _peaks()
-    flops_step, opt_bytes_step = _algorithmic_work(cfg)
+    work = _algorithmic_work(cfg)
     kern = {}
-    if prof["gemm"]["launches"]:
-        tf = flops_step * args.steps / (prof["gemm"]["ms"] * 1e-3) / 1e12
-        bound = "tensor" if cfg.dtype == "bf16_fp32master" else "alu"
-        peak = peaks["bf16_tflops_sustained"] if bound == "tensor" else 2 * 148 * 128 * 1.965e9 / 1e12
-        kern["gemm"] = {"bound": bound, "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
-                        "traffic": None, "ms_per_step": prof["gemm"]["ms"] / args.steps,
-                        "launches_per_step": prof["gemm"]["launches"] / args.steps,
-                        "peak_source": peaks["source"] + (" sustained bf16" if bound == "tensor" else
-                                                          " n/a: 148 SM x 128 FMA x 2 x 1.965 GHz fp32")}
-    if prof["optimizer"]["launches"] and cfg.model != "toy_quadratic":
-        gbs = opt_bytes_step * args.steps / (prof["optimizer"]["ms"] * 1e-3) / 1e9
-        kern["optimizer"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                             "frac": gbs / peaks["hbm_gbs"], "traffic": None,
-                             "ms_per_step": prof["optimizer"]["ms"] / args.steps,
-                             "launches_per_step": prof["optimizer"]["launches"] / args.steps,
-                             "peak_source": peaks["source"]}
+
+    def add(name, bound, amount, unit, peak, src):
+        if prof[name]["launches"] and amount > 0:
+            ach = amount * args.steps / (prof[name]["ms"] * 1e-3) / (1e12 if unit == "TFLOP/s" else 1e9)
+            kern[name] = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak, "traffic": None,
+                          "ms_per_step": prof[name]["ms"] / args.steps,
+                          "launches_per_step": prof[name]["launches"] / args.steps, "peak_source": src}
+
+    fused = prof["wgrad_adam"]["launches"] > 0
+    tensor = cfg.dtype == "bf16_fp32master"
+    gemm_flops = work["flops"] - (work["fused_flops"] if fused else 0.0)
+    add("gemm", "tensor" if tensor else "alu", gemm_flops, "TFLOP/s",
+        peaks["bf16_tflops_sustained"] if tensor else 2 * 148 * 128 * 1.965e9 / 1e12,
+        peaks["source"] + (" sustained bf16" if tensor else ": n/a, 148 SM x 128 FMA x 2 x 1.965 GHz fp32"))
+    if fused:
+        # HBM-bound: 12 B read + 14 B written per weight (master, two moments, bf16 shadow); the gradient stays on chip
+        add("wgrad_adam", "hbm", work["fused_params"] * 26.0, "GB/s", peaks["hbm_gbs"], peaks["source"])
+        kern.get("wgrad_adam", {}).update(tflops=work["fused_flops"] * args.steps / (prof["wgrad_adam"]["ms"] * 1e-3) / 1e12)
+    opt_params = work["opt_params"] - (work["fused_params"] if fused else 0)
+    add("optimizer", "hbm", opt_params * work["opt_bytes_per_param"], "GB/s", peaks["hbm_gbs"], peaks["source"])
     shares = {k: v["ms"] for k, v in prof.items()}
     dominant = max(kern, key=lambda k: kern[k]["ms_per_step"]) if kern else None
     roofline = dict(kern[dominant], kernel=dominant) if dominant else None

@@ -253,7 +253,8 @@ int pbt_get_launch_count(const pbt_t* p, int64_t* count);
 
 /*
  * Elapsed device time, in milliseconds, of one named kernel class accumulated
- * since pbt_profile_begin: "gemm", "optimizer", "loss", "copy", "select".
+ * since pbt_profile_begin: "gemm", "wgrad_adam" (weight gradient with the Adam update fused in),
+ * "optimizer" (the separate update pass), "loss", "copy", "select", "other".
  * Profiling brackets each launch with events on the handle's stream and
  * therefore slows the step down; it is off unless begun.
  */

@@ -136,7 +136,7 @@ class PbtError(RuntimeError):
         self.code = code
 
 
-def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = False) -> PbtSpec:
+def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True) -> PbtSpec:
     """Translate a declarative population description (see workloads.configs.PBTConfig) into pbt_spec."""
     s = PbtSpec()
     s.n_members = cfg.n_members
@@ -238,7 +238,7 @@ class Population:
     """One population living on one GPU.  Thin wrapper over the pbt_* calls."""
 
     def __init__(self, cfg, inputs, seed: Optional[int] = None, device: str = "cuda:0", keep_grad: bool = False,
-                 fuse_adam: bool = False):
+                 fuse_adam: bool = True):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -435,7 +435,7 @@ class Population:
     def profile_end(self) -> Dict[str, Dict[str, float]]:
         self._check(self.lib.pbt_profile_end(self.handle))
         out = {}
-        for cls in ("gemm", "optimizer", "loss", "copy", "select", "other"):
+        for cls in ("gemm", "wgrad_adam", "optimizer", "loss", "copy", "select", "other"):
             ms, n = C.c_double(0), C.c_int64(0)
             self._check(self.lib.pbt_profile_get(self.handle, cls.encode(), C.byref(ms), C.byref(n)))
             out[cls] = {"ms": ms.value, "launches": n.value}

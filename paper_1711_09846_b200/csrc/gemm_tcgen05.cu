@@ -10,9 +10,7 @@
 //               instruction, fp32 accumulators in TMEM), tcgen05.commit frees the stage / publishes the tile
 //   warps 2..   epilogue (4 or 8 warps): tcgen05.ld of the accumulator (double-buffered in TMEM, so the next
 //               tile's main loop overlaps), a 32 x 32 transpose through padded shared memory so that global
-//               accesses are whole 128-byte lines, then either bias / ReLU / ReLU-mask / conversion, or --
-//               for weight gradients -- the member's Adam update applied in place (the gradient never
-//               goes to HBM unless asked for)
+//               accesses are whole 128-byte lines, then bias / ReLU / ReLU-mask / conversion
 // Every mbarrier wait is bounded; on expiry the kernel records PBT_ERR_TIMEOUT in the device status
 // word, all roles leave their loops, tensor memory is released and the kernel returns normally.
 #include <string.h>
@@ -27,7 +25,6 @@ using namespace tc;
 
 constexpr int kBM = 128;
 constexpr int kBK = 64;
-constexpr int kFuseBatch = 4;  // row-quads of master / moment loads in flight per lane in the fused Adam epilogue
 constexpr int kEpiPitch = 36;  // floats per row of the epilogue transpose buffer (16-byte aligned, conflict-free)
 
 struct TcParams {
@@ -38,7 +35,6 @@ struct TcParams {
   const float* bias; long long strideBias; int relu;
   const bf16* mask; long long ldmask, strideMask;
   Counters* counters;
-  OptArgs opt;  // fused Adam epilogue only
 };
 
 template <int BN, int STAGES, int NEPIW>
@@ -53,7 +49,6 @@ struct Smem {
   static_assert(kTotal <= 232448, "shared memory budget of one CTA");
 };
 
-// EPI 0: C = epilogue(acc).  EPI 1: acc is a weight gradient; Adam update of the member's slab in place.
 template <int BN, int STAGES, int EPI, int NEPIW>
 __global__ void __launch_bounds__(64 + 32 * NEPIW, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
@@ -173,10 +168,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     int it = 0;
     bool ok = true;
     const int esz = p.out_dtype == kBF16 ? 2 : 4;
-    const bool vec_ok = EPI == 1 ? (p.ldc % 4 == 0)
-                                 : ((((uintptr_t)p.C & 15) == 0) && ((p.ldc * esz) % 16 == 0) && ((p.strideC * esz) % 16 == 0) &&
-                                    (!p.mask || ((((uintptr_t)p.mask & 7) == 0) && (p.ldmask % 4 == 0) && (p.strideMask % 4 == 0))) &&
-                                    (!p.bias || ((((uintptr_t)p.bias & 15) == 0) && (p.strideBias % 4 == 0))));
+    const bool vec_ok = (((uintptr_t)p.C & 15) == 0) && ((p.ldc * esz) % 16 == 0) && ((p.strideC * esz) % 16 == 0) &&
+                        (!p.mask || ((((uintptr_t)p.mask & 7) == 0) && (p.ldmask % 4 == 0) && (p.strideMask % 4 == 0))) &&
+                        (!p.bias || ((((uintptr_t)p.bias & 15) == 0) && (p.strideBias % 4 == 0)));
     const int rsub = lane >> 3, cc = (lane & 7) * 4;   // phase 2: 4 rows x 8 column-quads per warp instruction
     for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++it) {
       const int member = tile / (p.tiles_m * p.tiles_n);
@@ -186,19 +180,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       const uint32_t acc_phase = (it >> 1) & 1;
       if (!mbar_wait(&tfull[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      // per-member optimiser constants (fused mode)
-      float lr = 0.f, b1 = 0.f, omb1 = 0.f, b2 = 0.f, omb2 = 0.f, inv_bc1 = 0.f, inv_bc2 = 0.f, eps = 0.f, lrwd = 0.f;
-      if (EPI == 1) {
-        const float* Hrow = p.opt.H + (long long)member * p.opt.nh_stride;
-        lr = hp(Hrow, p.opt.slot_lr, p.opt.const_lr);
-        b1 = hp(Hrow, p.opt.slot_beta1, p.opt.const_beta1);
-        const float wd = hp(Hrow, p.opt.slot_wd, p.opt.const_wd);
-        b2 = p.opt.const_beta2; eps = p.opt.const_eps;
-        const float c1 = __fmul_rn(p.opt.scalars[member * PBT_N_SCALARS + p.opt.scalar_base + 0], b1);
-        const float c2 = __fmul_rn(p.opt.scalars[member * PBT_N_SCALARS + p.opt.scalar_base + 1], b2);
-        inv_bc1 = 1.f / (1.f - c1); inv_bc2 = 1.f / (1.f - c2);
-        omb1 = 1.f - b1; omb2 = 1.f - b2; lrwd = lr * wd;
-      }
       const float* bias = p.bias ? p.bias + member * p.strideBias : nullptr;
       // The accumulator chunk for iteration c+1 is requested from tensor memory while chunk c is being
       // transposed and written out, and the ReLU-mask words are requested before the transpose, so that
@@ -214,7 +195,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         const int col = nbase + cc;
         const bool full4 = vec_ok && col + 3 < p.N;
         uint2 mk[8];
-        if (EPI == 0 && p.mask && full4) {
+        if (p.mask && full4) {
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const int row = m0 + q * 32 + i * 4 + rsub;
@@ -229,7 +210,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           *reinterpret_cast<uint4*>(&buf[lane * kEpiPitch + j * 4]) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
         if (c0 + kChunkStep < BN && nbase + kChunkStep < p.N) tmem_ld32(tacc + c0 + kChunkStep, r);
         __syncwarp();
-        if (EPI == 0) {
+        {
           float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
           if (bias && col < p.N) {
             if (full4) bv = __ldg(reinterpret_cast<const float4*>(bias + col));
@@ -287,55 +268,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
               else {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) if (col + j < p.N) cp[j] = v[j];
-              }
-            }
-          }
-        } else {
-          // fused Adam: element (row, col) of this layer's weight matrix lives at begin + row*ldc + col of the slab
-          const long long slab = (long long)member * p.opt.p_pad + p.opt.begin;
-          float* gout = reinterpret_cast<float*>(p.C);
-#pragma unroll 1
-          for (int i0 = 0; i0 < 8; i0 += kFuseBatch) {
-            float4 ww[kFuseBatch], aa[kFuseBatch], bb[kFuseBatch];
-            bool live[kFuseBatch];
-#pragma unroll
-            for (int u = 0; u < kFuseBatch; ++u) {
-              const int rr = (i0 + u) * 4 + rsub;
-              const int row = m0 + q * 32 + rr;
-              live[u] = row < p.M && full4;
-              if (live[u]) {
-                const long long off = slab + (long long)row * p.ldc + col;
-                ww[u] = ld_stream(p.opt.w32 + off);
-                aa[u] = ld_stream(p.opt.opt1 + off);
-                bb[u] = ld_stream(p.opt.opt2 + off);
-              }
-            }
-#pragma unroll
-            for (int u = 0; u < kFuseBatch; ++u) {
-              const int rr = (i0 + u) * 4 + rsub;
-              const int row = m0 + q * 32 + rr;
-              const float4 g4 = *reinterpret_cast<const float4*>(&buf[rr * kEpiPitch + cc]);
-              const long long off = slab + (long long)row * p.ldc + col;
-              if (live[u]) {
-                float4 nw;
-                nw.x = adam_one(ww[u].x, aa[u].x, bb[u].x, g4.x, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
-                nw.y = adam_one(ww[u].y, aa[u].y, bb[u].y, g4.y, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
-                nw.z = adam_one(ww[u].z, aa[u].z, bb[u].z, g4.z, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
-                nw.w = adam_one(ww[u].w, aa[u].w, bb[u].w, g4.w, b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
-                st_stream(p.opt.opt1 + off, aa[u]);
-                st_stream(p.opt.opt2 + off, bb[u]);
-                st_stream(p.opt.w32 + off, nw);
-                if (p.opt.w16) st_bf16x4(p.opt.w16 + off, nw);
-                if (gout) st_stream(gout + member * p.strideC + (long long)row * p.ldc + col, g4);
-              } else if (row < p.M && col < p.N) {
-                const float gs[4] = {g4.x, g4.y, g4.z, g4.w};
-                for (int j = 0; j < 4 && col + j < p.N; ++j) {
-                  float m1 = p.opt.opt1[off + j], m2 = p.opt.opt2[off + j];
-                  const float nw = adam_one(p.opt.w32[off + j], m1, m2, gs[j], b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
-                  p.opt.opt1[off + j] = m1; p.opt.opt2[off + j] = m2; p.opt.w32[off + j] = nw;
-                  if (p.opt.w16) p.opt.w16[off + j] = __float2bfloat16_rn(nw);
-                  if (gout) gout[member * p.strideC + (long long)row * p.ldc + col + j] = gs[j];
-                }
               }
             }
           }
@@ -402,8 +334,6 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s
   p.bias = g.bias; p.strideBias = g.strideBias; p.relu = g.relu;
   p.mask = reinterpret_cast<const bf16*>(g.mask); p.ldmask = g.ldmask; p.strideMask = g.strideMask;
   p.counters = counters;
-  memset(&p.opt, 0, sizeof(p.opt));
-  if (g.adam) p.opt = *g.adam;
   const int BN = g.N >= 256 ? 256 : 128;
   CUtensorMap tmA, tmB;
   bool ok;
@@ -414,12 +344,7 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s
   if (!g.b_mn) ok = make_map(&tmB, g.B, g.K, g.N, g.ldb, p.b_batched ? g.batch : 1, g.strideB, BN);
   else ok = make_map(&tmB, g.B, g.N, g.K, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kBK);
   if (!ok) return cudaErrorInvalidValue;
-  if (g.adam) {
-    // epilogue-bound: 26 bytes of HBM traffic per output element; 8 epilogue warps (2 per TMEM lane quadrant,
-    // interleaved over 32-column chunks)
-    if (BN == 256) return launch_cfg<256, 3, 1, 8>(tmA, tmB, p, s);
-    return launch_cfg<128, 4, 1, 8>(tmA, tmB, p, s);
-  }
+  if (g.adam) return cudaErrorInvalidValue;  // the fused weight-gradient + Adam kernel has its own launcher
   // short contractions (weight gradients: K = batch) are bound by writing the tile out: more epilogue warps,
   // shallower operand ring
   if (p.k_blocks <= 12) {

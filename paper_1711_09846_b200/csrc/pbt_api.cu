@@ -28,8 +28,8 @@ struct Stack {
   int rows_cap;            // rows the activation buffers can hold
 };
 
-enum KClass { kGemm = 0, kOpt, kLoss, kCopy, kSelect, kOther, kNumClasses };
-const char* const kClassNames[kNumClasses] = {"gemm", "optimizer", "loss", "copy", "select", "other"};
+enum KClass { kGemm = 0, kOpt, kLoss, kCopy, kSelect, kOther, kFused, kNumClasses };
+const char* const kClassNames[kNumClasses] = {"gemm", "optimizer", "loss", "copy", "select", "other", "wgrad_adam"};
 
 struct ProfRec {
   int cls;
@@ -302,7 +302,7 @@ struct LaunchScope {
 
 int gemm(pbt_handle* h, const GemmArgs& g) {
   if (g.adam) {
-    LAUNCH(h, kGemm, launch_wgrad_adam(g, h->counters, h->stream));
+    LAUNCH(h, kFused, launch_wgrad_adam(g, h->counters, h->stream));
   } else if (gemm_tc_supported(g)) {
     LAUNCH(h, kGemm, launch_gemm_tc(g, h->counters, h->stream));
   } else {

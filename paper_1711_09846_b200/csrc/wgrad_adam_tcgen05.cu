@@ -10,9 +10,9 @@
 //   warp 1       tensor-memory allocation + tcgen05.mma issue (128 x 256 tile, accumulator double-buffered)
 //   warp 2       TMA loader for the optimiser state: per 32-column chunk of the tile one 128 x 32 fp32 box each of
 //                master weights, first and second moment into a ring of two slots (128-byte swizzle)
-//   warp 3       TMA storer: when the eight update warps are done with a slot, stores the three boxes back in
+//   warp 3       TMA storer: when the sixteen update warps are done with a slot, stores the three boxes back in
 //                place plus the bf16 shadow box, and hands the slot back to the loader once it has been read
-//   warps 4..11  update: tcgen05.ld of 16 gradient columns of the thread's row, Adam on the slot in shared memory
+//   warps 4..19  update: tcgen05.ld of 8 gradient columns of the thread's row, Adam on the slot in shared memory
 // All mbarrier waits are bounded; on expiry PBT_ERR_TIMEOUT is recorded and every role leaves its loop.
 #include <string.h>
 
@@ -25,7 +25,9 @@ namespace {
 using namespace tc;
 
 constexpr int kBM = 128, kBN = 256, kBK = 64;
-constexpr int kStages = 2, kSlots = 2, kChunk = 32, kUpdWarps = 8;
+constexpr int kStages = 2, kSlots = 2, kChunk = 32, kUpdWarps = 16;
+constexpr int kColsPerWarp = kChunk / (kUpdWarps / 4);   // gradient columns one update thread handles per chunk
+static_assert(kColsPerWarp == 8 || kColsPerWarp == 16, "update warps per TMEM lane quadrant");
 constexpr int kThreads = 32 * (4 + kUpdWarps);
 constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2, kStageBytes = kABytes + kBBytes;
 constexpr int kBoxBytes = kBM * kChunk * 4;     // one fp32 state box
@@ -186,7 +188,7 @@ k_wgrad_adam(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
   } else {
     // ------------------------------ update warps ------------------------------
     const int q = warp & 3;               // TMEM lane quadrant this warp may access
-    const int half = (warp - 4) >> 2;     // which 16 of the chunk's 32 columns
+    const int half = (warp - 4) >> 2;     // which kColsPerWarp of the chunk's 32 columns
     const int rloc = q * 32 + lane;       // row of the tile handled by this thread
     uint32_t slot = 0, sphase = 0;
     int it = 0;
@@ -206,20 +208,21 @@ k_wgrad_adam(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const float c2 = __fmul_rn(p.opt.scalars[member * PBT_N_SCALARS + p.opt.scalar_base + 1], b2);
       const float inv_bc1 = 1.f / (1.f - c1), inv_bc2 = 1.f / (1.f - c2);
       const float omb1 = 1.f - b1, omb2 = 1.f - b2, lrwd = lr * wd;
-      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kBN + half * 16);
-      uint32_t g[16];
-      tmem_ld16(tacc, g);
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kBN + half * kColsPerWarp);
+      uint32_t g[kColsPerWarp];
+      if (kColsPerWarp == 16) tmem_ld16(tacc, g); else tmem_ld8(tacc, g);
 #pragma unroll 1
       for (int c = 0; c < kChunks; ++c) {
         const int col0 = n0 + c * kChunk;
         if (col0 >= p.N) break;
         tmem_ld_wait();
-        float gf[16];
+        float gf[kColsPerWarp];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) gf[j] = __uint_as_float(g[j]);
+        for (int j = 0; j < kColsPerWarp; ++j) gf[j] = __uint_as_float(g[j]);
         const bool last = (c + 1 == kChunks) || (col0 + kChunk >= p.N);
         if (!last) {
-          tmem_ld16(tacc + (c + 1) * kChunk, g);   // next chunk's gradient while this one is applied
+          // next chunk's gradient while this one is applied
+          if (kColsPerWarp == 16) tmem_ld16(tacc + (c + 1) * kChunk, g); else tmem_ld8(tacc + (c + 1) * kChunk, g);
         } else {
           tc_fence_before();
           __syncwarp();
@@ -227,11 +230,11 @@ k_wgrad_adam(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         }
         if (!mbar_wait(&sfull[slot], sphase, abort_flag)) { ok = false; break; }
         uint8_t* box = smem + kSlotOffset + slot * kSlotBytes;
-        uint8_t* w16row = smem + kW16Offset + slot * kW16Bytes + rloc * (kChunk * 2) + half * 32;
+        uint8_t* w16row = smem + kW16Offset + slot * kW16Bytes + rloc * (kChunk * 2) + half * (kColsPerWarp * 2);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          // 16-byte piece (half*4 + j) of this thread's 128-byte row sits at position piece ^ (row & 7)
-          const int off = rloc * 128 + (((half * 4 + j) ^ (rloc & 7)) << 4);
+        for (int j = 0; j < kColsPerWarp / 4; ++j) {
+          // 16-byte piece (half * kColsPerWarp/4 + j) of this thread's 128-byte row sits at position piece ^ (row & 7)
+          const int off = rloc * 128 + (((half * (kColsPerWarp / 4) + j) ^ (rloc & 7)) << 4);
           float4 w = *reinterpret_cast<float4*>(box + off);
           float4 m1 = *reinterpret_cast<float4*>(box + kBoxBytes + off);
           float4 m2 = *reinterpret_cast<float4*>(box + 2 * kBoxBytes + off);
@@ -254,8 +257,8 @@ k_wgrad_adam(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           if (row < p.M) {
             float* gp = p.gout + member * p.strideC + (long long)row * p.ldc;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int col = col0 + half * 16 + j;
+            for (int j = 0; j < kColsPerWarp; ++j) {
+              const int col = col0 + half * kColsPerWarp + j;
               if (col < p.N) gp[col] = gf[j];
             }
           }
