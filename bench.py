@@ -91,6 +91,25 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+# DRAM bytes per parameter of the fused weight-gradient + Adam kernel, from one `ncu --set full` capture of a
+# small case (profiles/k_wgrad_adam_c5_8members.md), valid for the source file with this sha1 only.
+_NCU_TRAFFIC = {"wgrad_adam": {"bytes_per_param": 25.48, "source": "paper_1711_09846_b200/csrc/wgrad_adam_tcgen05.cu",
+                               "sha1": "8e5c237a7aac9a20bd38b2f8e9693f2484a05f1d"}}
+
+
+def _ncu_traffic(name, params_per_launch):
+    """Measured DRAM traffic of one launch, scaled from the captured small case; None once the kernel changed."""
+    import hashlib
+    rec = _NCU_TRAFFIC.get(name)
+    if not rec:
+        return None
+    try:
+        sha = hashlib.sha1(open(os.path.join(ROOT, rec["source"]), "rb").read()).hexdigest()
+    except OSError:
+        return None
+    return rec["bytes_per_param"] * params_per_launch if sha == rec["sha1"] else None
+
+
 def _tc_layer(fan_in, fan_out, rows):
     """Layers whose weight gradient qualifies for the tensor-core kernel (the library's own rule)."""
     return fan_in >= 128 and fan_out >= 128 and rows >= 64 and fan_in % 8 == 0 and fan_out % 8 == 0
@@ -343,7 +362,11 @@ def main():
     if fused:
         # HBM-bound: 12 B read + 14 B written per weight (master, two moments, bf16 shadow); the gradient stays on chip
         add("wgrad_adam", "hbm", work["fused_params"] * 26.0, "GB/s", peaks["hbm_gbs"], peaks["source"])
-        kern.get("wgrad_adam", {}).update(tflops=work["fused_flops"] * args.steps / (prof["wgrad_adam"]["ms"] * 1e-3) / 1e12)
+        if "wgrad_adam" in kern:
+            k = kern["wgrad_adam"]
+            k["tflops"] = work["fused_flops"] * args.steps / (prof["wgrad_adam"]["ms"] * 1e-3) / 1e12
+            k["algorithmic_bytes_per_launch"] = work["fused_params"] * 26.0 / k["launches_per_step"]
+            k["traffic"] = _ncu_traffic("wgrad_adam", work["fused_params"] / k["launches_per_step"])
     opt_params = work["opt_params"] - (work["fused_params"] if fused else 0)
     add("optimizer", "hbm", opt_params * work["opt_bytes_per_param"], "GB/s", peaks["hbm_gbs"], peaks["source"])
     shares = {k: v["ms"] for k, v in prof.items()}
