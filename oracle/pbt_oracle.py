@@ -236,11 +236,14 @@ def adam_update(theta, m, v, g, lr, b1, b2, eps, wd, c1, c2):
 class Population:
     """State (theta, h, p, t) of every member (Algorithm 1) plus optimiser state."""
 
-    def __init__(self, cfg, inputs, seed: Optional[int] = None):
+    def __init__(self, cfg, inputs, seed: Optional[int] = None, only_members=None):
+        """only_members: build (and later step / evaluate) just these members of the population; the
+        others stay empty.  For checking a sample of a large population member by member."""
         self.cfg = cfg
         self.inp = inputs
         self.seed = int(cfg.seed if seed is None else seed)
         self.N = cfg.n_members
+        self.members = list(range(self.N)) if only_members is None else [int(m) for m in only_members]
         self.toy = cfg.model == "toy_quadratic"
         self.gan = cfg.model == "gan_pair"
         self.bf16 = cfg.dtype == "bf16_fp32master"
@@ -265,12 +268,12 @@ class Population:
                     self.shapes.append((s, l, ws[l + 1], ws[l]))
             self.W = [[None] * len(self.shapes) for _ in range(self.N)]
             self.b = [[None] * len(self.shapes) for _ in range(self.N)]
-            for m in range(self.N):
+            for m in self.members:
                 for t, (s, l, fo, fi) in enumerate(self.shapes):
                     self.W[m][t] = self._init_weight(m, s, l, fo, fi)
                     self.b[m][t] = np.zeros(fo, dtype=np.float32)
-            z = lambda: [[np.zeros_like(x) for x in row] for row in self.W]
-            zb = lambda: [[np.zeros_like(x) for x in row] for row in self.b]
+            z = lambda: [[None if x is None else np.zeros_like(x) for x in row] for row in self.W]
+            zb = lambda: [[None if x is None else np.zeros_like(x) for x in row] for row in self.b]
             self.o1W, self.o1b = z(), zb()      # momentum / Adam m
             self.o2W, self.o2b = z(), zb()      # Adam v
             self.gW, self.gb = z(), zb()        # last gradient (for inspection)
@@ -435,7 +438,7 @@ class Population:
 
     def step(self, k: int = 1, members=None, batch=None):
         """k lockstep steps for all (or the given) members (Algorithm 1, line `step`)."""
-        members = range(self.N) if members is None else members
+        members = self.members if members is None else members
         for _ in range(k):
             for m in members:
                 if self.toy:
@@ -462,7 +465,7 @@ class Population:
         return -loss
 
     def eval(self, members=None):
-        members = range(self.N) if members is None else members
+        members = self.members if members is None else members
         for m in members:
             self.fitness[m] = self.master(self.eval_member(m))
         return self.fitness.copy()
