@@ -91,6 +91,156 @@ __global__ void __launch_bounds__(256) k_gemm_simt(GemmArgs g) {
   }
 }
 
+// ---------------------------------------------------------------------------
+// Skinny shapes (a dimension of 16 or less: one-, two- and ten-wide output layers, two-wide inputs).
+// The 64x64 tile kernel above spends its time in shared-memory round trips there; these three kernels
+// read every operand once, coalesced, and reduce in a fixed order.
+// ---------------------------------------------------------------------------
+constexpr int kSkinny = 16;
+
+__device__ __forceinline__ float epilogue_one(const GemmArgs& g, int member, int m, int n, float v, int in_is_bf16) {
+  if (g.bias) v += g.bias[member * g.strideBias + n];
+  if (g.relu) v = fmaxf(v, 0.f);
+  if (g.mask) {
+    const long long mi = member * g.strideMask + (long long)m * g.ldmask + n;
+    const float mv = in_is_bf16 ? __bfloat162float(reinterpret_cast<const bf16*>(g.mask)[mi])
+                                : reinterpret_cast<const float*>(g.mask)[mi];
+    if (!(mv > 0.f)) v = 0.f;
+  }
+  return v;
+}
+__device__ __forceinline__ void store_one(const GemmArgs& g, int member, int m, int n, float v) {
+  const long long ci = member * g.strideC + (long long)m * g.ldc + n;
+  if (g.out_dtype == kBF16) reinterpret_cast<bf16*>(g.C)[ci] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float*>(g.C)[ci] = v;
+}
+
+// N <= NT <= 16, A K-major: one warp per output row, lanes stride over K, shuffle reduction.
+template <typename T, bool B_MN, int NT>
+__global__ void __launch_bounds__(256) k_gemm_rowdot(GemmArgs g) {
+  const int member = blockIdx.y, lane = threadIdx.x & 31;
+  const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (m >= g.M) return;
+  const T* __restrict__ A = reinterpret_cast<const T*>(g.A) + member * g.strideA + (long long)m * g.lda;
+  const T* __restrict__ B = reinterpret_cast<const T*>(g.B) + member * g.strideB;
+  float acc[NT];
+#pragma unroll
+  for (int n = 0; n < NT; ++n) acc[n] = 0.f;
+#pragma unroll 4
+  for (int k = lane; k < g.K; k += 32) {
+    const float a = to_f<T>(A[k]);
+#pragma unroll
+    for (int n = 0; n < NT; ++n)
+      if (NT == 1 || n < g.N) acc[n] = fmaf(a, to_f<T>(B_MN ? B[(long long)k * g.ldb + n] : B[(long long)n * g.ldb + k]), acc[n]);
+  }
+#pragma unroll
+  for (int n = 0; n < NT; ++n) {
+    float v = acc[n];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (lane == n && n < g.N) store_one(g, member, m, n, epilogue_one(g, member, m, n, v, sizeof(T) == 2));
+  }
+}
+
+// Both operands MN-major (weight gradients), the short one of M, N at most ST <= 16: thread per index of the
+// long dimension, 16 slices of K per block combined in a fixed order.  LONG_A: M is the long dimension, else N.
+template <typename T, bool LONG_A, int ST>
+__global__ void __launch_bounds__(512) k_gemm_colacc(GemmArgs g) {
+  __shared__ float red[16][32][ST + 1];
+  const int member = blockIdx.y, tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int L = LONG_A ? g.M : g.N, S = LONG_A ? g.N : g.M;
+  const long long ldx = LONG_A ? g.lda : g.ldb, ldy = LONG_A ? g.ldb : g.lda;
+  const T* __restrict__ X = reinterpret_cast<const T*>(LONG_A ? g.A : g.B) + member * (LONG_A ? g.strideA : g.strideB);
+  const T* __restrict__ Y = reinterpret_cast<const T*>(LONG_A ? g.B : g.A) + member * (LONG_A ? g.strideB : g.strideA);
+  const int l = blockIdx.x * 32 + tx;
+  float acc[ST];
+#pragma unroll
+  for (int s = 0; s < ST; ++s) acc[s] = 0.f;
+  if (l < L) {
+#pragma unroll 4
+    for (int k = ty; k < g.K; k += 16) {
+      const float x = to_f<T>(X[(long long)k * ldx + l]);
+#pragma unroll
+      for (int s = 0; s < ST; ++s)
+        if (ST == 1 || s < S) acc[s] = fmaf(x, to_f<T>(Y[(long long)k * ldy + s]), acc[s]);
+    }
+  }
+#pragma unroll
+  for (int s = 0; s < ST; ++s) red[ty][tx][s] = acc[s];
+  __syncthreads();
+  if (ty == 0 && l < L) {
+#pragma unroll
+    for (int s = 0; s < ST; ++s) {
+      if (s < S) {
+        float v = 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v += red[j][tx][s];
+        const int m = LONG_A ? l : s, n = LONG_A ? s : l;
+        store_one(g, member, m, n, epilogue_one(g, member, m, n, v, sizeof(T) == 2));
+      }
+    }
+  }
+}
+
+// K <= 16: every output element is a short dot product; block = 256 consecutive n of one row m.
+template <typename T>
+__global__ void __launch_bounds__(256) k_gemm_smallk(GemmArgs g) {
+  const int member = blockIdx.z, m = blockIdx.y;
+  const int n = blockIdx.x * 256 + threadIdx.x;
+  if (n >= g.N) return;
+  const T* __restrict__ A = reinterpret_cast<const T*>(g.A) + member * g.strideA;
+  const T* __restrict__ B = reinterpret_cast<const T*>(g.B) + member * g.strideB;
+  float v = 0.f;
+  for (int k = 0; k < g.K; ++k) {
+    const float a = to_f<T>(g.a_mn ? A[(long long)k * g.lda + m] : A[(long long)m * g.lda + k]);
+    const float b = to_f<T>(g.b_mn ? B[(long long)k * g.ldb + n] : B[(long long)n * g.ldb + k]);
+    v = fmaf(a, b, v);
+  }
+  store_one(g, member, m, n, epilogue_one(g, member, m, n, v, sizeof(T) == 2));
+}
+
+template <typename T, bool B_MN>
+static void launch_rowdot(const GemmArgs& g, cudaStream_t s) {
+  dim3 grid((g.M + 7) / 8, g.batch);
+  if (g.N == 1) k_gemm_rowdot<T, B_MN, 1><<<grid, 256, 0, s>>>(g);
+  else if (g.N == 2) k_gemm_rowdot<T, B_MN, 2><<<grid, 256, 0, s>>>(g);
+  else if (g.N <= 4) k_gemm_rowdot<T, B_MN, 4><<<grid, 256, 0, s>>>(g);
+  else if (g.N <= 8) k_gemm_rowdot<T, B_MN, 8><<<grid, 256, 0, s>>>(g);
+  else k_gemm_rowdot<T, B_MN, 16><<<grid, 256, 0, s>>>(g);
+}
+template <typename T, bool LONG_A>
+static void launch_colacc(const GemmArgs& g, cudaStream_t s) {
+  const int L = LONG_A ? g.M : g.N, S = LONG_A ? g.N : g.M;
+  dim3 grid((L + 31) / 32, g.batch);
+  if (S == 1) k_gemm_colacc<T, LONG_A, 1><<<grid, 512, 0, s>>>(g);
+  else if (S == 2) k_gemm_colacc<T, LONG_A, 2><<<grid, 512, 0, s>>>(g);
+  else if (S <= 4) k_gemm_colacc<T, LONG_A, 4><<<grid, 512, 0, s>>>(g);
+  else if (S <= 8) k_gemm_colacc<T, LONG_A, 8><<<grid, 512, 0, s>>>(g);
+  else k_gemm_colacc<T, LONG_A, 16><<<grid, 512, 0, s>>>(g);
+}
+
+template <typename T>
+static bool launch_skinny(const GemmArgs& g, cudaStream_t s) {
+  if (g.K <= kSkinny && g.K > 0 && g.M <= 65535 && g.batch <= 65535) {
+    k_gemm_smallk<T><<<dim3((g.N + 255) / 256, g.M, g.batch), 256, 0, s>>>(g);
+    return true;
+  }
+  if (g.N <= kSkinny && !g.a_mn) {
+    if (g.b_mn) launch_rowdot<T, true>(g, s);
+    else launch_rowdot<T, false>(g, s);
+    return true;
+  }
+  if (g.a_mn && g.b_mn && g.N <= kSkinny) {
+    launch_colacc<T, true>(g, s);
+    return true;
+  }
+  if (g.a_mn && g.b_mn && g.M <= kSkinny) {
+    launch_colacc<T, false>(g, s);
+    return true;
+  }
+  return false;
+}
+
 template <typename T>
 static cudaError_t launch_t(const GemmArgs& g, cudaStream_t s) {
   dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.batch);
@@ -103,6 +253,7 @@ static cudaError_t launch_t(const GemmArgs& g, cudaStream_t s) {
 
 cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t s) {
   if (g.M <= 0 || g.N <= 0 || g.batch <= 0) return cudaSuccess;
+  if (g.in_dtype == kBF16 ? launch_skinny<bf16>(g, s) : launch_skinny<float>(g, s)) return cudaGetLastError();
   return g.in_dtype == kBF16 ? launch_t<bf16>(g, s) : launch_t<float>(g, s);
 }
 
