@@ -41,6 +41,22 @@ def _peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def max_over_ranks(x: float, device=None) -> float:
+    """Slowest rank's time: the population replicas are independent, the job is as slow as its slowest replica."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(cfg, world: int, steps: int, ms: float) -> float:
+    """member-samples/s of the whole job: every rank trains its own replica of the population."""
+    return world * cfg.n_members * max(cfg.batch, 1) * steps / (ms * 1e-3)
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -318,11 +334,8 @@ def main():
         for i in range(args.steps):
             hot_path_step(i, [0])
         prof = pop.profile_end()
-    if world > 1:
-        t = torch.tensor([ms], device=f"cuda:{local}")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * cfg.n_members * max(cfg.batch, 1) * args.steps / (ms * 1e-3)
+    ms = max_over_ranks(ms, f"cuda:{local}")
+    value = job_value(cfg, world, args.steps, ms)
 
     # ---- end to end: host buffers in, loss out, through the C ABI (MLP populations) ----
     e2e = None
@@ -350,10 +363,7 @@ def main():
                 pop.exploit_explore()
         pop.synchronize()
         dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], device=f"cuda:{local}")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = max_over_ranks(dt, f"cuda:{local}")
         e2e = {"value": world * cfg.n_members * cfg.batch * e2e_steps / dt, "unit": UNIT,
                "h2d_bytes_per_step": int(xs[0].numel() * xs[0].element_size() + ys[0].numel() * ys[0].element_size()),
                "d2h_bytes_per_step": int(cfg.n_members * 2 * 4), "steps": e2e_steps,

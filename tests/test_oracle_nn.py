@@ -297,3 +297,19 @@ def test_gan_finite_difference_of_generator_loss():
         pop.W[0][0] = Wm
         lm = LG()
         assert abs((lp - lm) / (2 * e) - g[o, i]) < 1e-6 * max(1.0, abs(g[o, i]))
+
+
+def test_grouped_gemm_against_triple_loop():
+    rng = np.random.default_rng(13)
+    A, B = rng.standard_normal((2, 3, 5)), rng.standard_normal((2, 4, 5))
+    bias, mask = rng.standard_normal((2, 4)), rng.standard_normal((2, 3, 4))
+    mask[0, 1, 2] = 0.0
+    got = O.grouped_gemm(A, B, bias, True, mask)
+    for b in range(2):
+        for m in range(3):
+            for n in range(4):
+                s = sum(A[b, m, k] * B[b, n, k] for k in range(5)) + bias[b, n]
+                s = max(s, 0.0) if mask[b, m, n] > 0 else 0.0
+                assert abs(got[b, m, n] - s) < 1e-13
+    plain = O.grouped_gemm(A, B)
+    assert abs(plain[1, 2, 3] - float(A[1, 2] @ B[1, 3])) < 1e-13
