@@ -8,7 +8,7 @@
 //               into a ring of shared-memory stages guarded by full/empty mbarriers; plain per-CTA loads
 //   warp 1      allocates tensor memory, one elected lane issues tcgen05.mma (128 x BN x 16 per
 //               instruction, fp32 accumulators in TMEM), tcgen05.commit frees the stage / publishes the tile
-//   warps 2..   epilogue (4 or 8 warps): tcgen05.ld of the accumulator (double-buffered in TMEM, so the next
+//   warps 2..9  epilogue (8 warps, two per TMEM lane quadrant): tcgen05.ld of the accumulator (double-buffered in TMEM, so the next
 //               tile's main loop overlaps), a 32 x 32 transpose through padded shared memory so that global
 //               accesses are whole 128-byte lines, then bias / ReLU / ReLU-mask / conversion
 // Every mbarrier wait is bounded; on expiry the kernel records PBT_ERR_TIMEOUT in the device status
@@ -345,14 +345,10 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s
   else ok = make_map(&tmB, g.B, g.N, g.K, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kBK);
   if (!ok) return cudaErrorInvalidValue;
   if (g.adam) return cudaErrorInvalidValue;  // the fused weight-gradient + Adam kernel has its own launcher
-  // short contractions (weight gradients: K = batch) are bound by writing the tile out: more epilogue warps,
-  // shallower operand ring
-  if (p.k_blocks <= 12) {
-    if (BN == 256) return launch_cfg<256, 3, 0, 8>(tmA, tmB, p, s);
-    return launch_cfg<128, 4, 0, 8>(tmA, tmB, p, s);
-  }
-  if (BN == 256) return launch_cfg<256, 4, 0, 4>(tmA, tmB, p, s);
-  return launch_cfg<128, 6, 0, 4>(tmA, tmB, p, s);
+  // 8 epilogue warps (two per TMEM lane quadrant) keep the tile write-out and the ReLU-mask reads off the critical
+  // path; a 3-stage operand ring is as fast as 4 stages here and leaves the shared memory for them
+  if (BN == 256) return launch_cfg<256, 3, 0, 8>(tmA, tmB, p, s);
+  return launch_cfg<128, 4, 0, 8>(tmA, tmB, p, s);
 }
 
 }  // namespace pbt
