@@ -248,6 +248,18 @@ int pbt_set_batch(pbt_t* p, const void* x_device, const void* y_device);
  */
 int pbt_step_host(pbt_t* p, const void* x_host, const void* y_host, double* loss_out_host);
 
+/*
+ * The same step with the upload taken off the critical path: pbt_prefetch_host_batch starts copying the
+ * next step's rows (same layout as pbt_step_host; use pinned memory) into a spare buffer on a copy stream of the
+ * library's own and returns at once; pbt_step_prefetched makes the stream wait for that copy and enqueues one
+ * training step on it.  With loss_out_host == NULL it returns without synchronising, so the caller can prefetch
+ * the rows of step t+1 while step t runs and read the losses afterwards (pbt_get_last_loss); otherwise it copies
+ * the losses back and synchronises.  PBT_ERR_STATE if nothing was prefetched, or if a prefetched batch is still
+ * waiting to be consumed.  MLP only.
+ */
+int pbt_prefetch_host_batch(pbt_t* p, const void* x_host, const void* y_host);
+int pbt_step_prefetched(pbt_t* p, double* loss_out_host);
+
 /* Kernel launches issued by the last pbt_step / pbt_eval / pbt_exploit_explore call. */
 int pbt_get_launch_count(const pbt_t* p, int64_t* count);
 

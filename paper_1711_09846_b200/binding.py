@@ -74,7 +74,7 @@ EXPORTS = [
     "pbt_query_workspace", "pbt_param_count", "pbt_create", "pbt_destroy", "pbt_step", "pbt_eval",
     "pbt_exploit_explore", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
     "pbt_get_hparams", "pbt_set_hparams", "pbt_get_copy_map", "pbt_get_best", "pbt_get_last_loss",
-    "pbt_set_batch", "pbt_step_host", "pbt_get_launch_count", "pbt_profile_begin", "pbt_profile_end", "pbt_profile_get",
+    "pbt_set_batch", "pbt_step_host", "pbt_prefetch_host_batch", "pbt_step_prefetched", "pbt_get_launch_count", "pbt_profile_begin", "pbt_profile_end", "pbt_profile_get",
     "pbt_grouped_gemm", "pbt_energy_fitness_static", "pbt_last_error",
 ]
 
@@ -115,6 +115,8 @@ def load_library() -> C.CDLL:
     lib.pbt_get_last_loss.argtypes = [vp, C.POINTER(C.c_double)]
     lib.pbt_set_batch.argtypes = [vp, vp, vp]
     lib.pbt_step_host.argtypes = [vp, vp, vp, C.POINTER(C.c_double)]
+    lib.pbt_prefetch_host_batch.argtypes = [vp, vp, vp]
+    lib.pbt_step_prefetched.argtypes = [vp, C.POINTER(C.c_double)]
     lib.pbt_get_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
     lib.pbt_profile_begin.argtypes = [vp]
     lib.pbt_profile_end.argtypes = [vp]
@@ -422,6 +424,20 @@ class Population:
             loss_out = np.zeros((self.N, 2), dtype=np.float64)
         self._check(self.lib.pbt_step_host(self.handle, C.c_void_p(x_host.data_ptr()), C.c_void_p(y_host.data_ptr()),
                                            loss_out.ctypes.data_as(C.POINTER(C.c_double))))
+        return loss_out
+
+    def prefetch_host_batch(self, x_host, y_host):
+        """Start uploading the next step's rows (pinned torch CPU tensors) while the current step runs."""
+        self._check(self.lib.pbt_prefetch_host_batch(self.handle, C.c_void_p(x_host.data_ptr()), C.c_void_p(y_host.data_ptr())))
+
+    def step_prefetched(self, loss_out: Optional[np.ndarray] = None, wait: bool = True):
+        """One step on the prefetched rows.  wait=False only enqueues (read the losses later with last_loss())."""
+        if not wait:
+            self._check(self.lib.pbt_step_prefetched(self.handle, None))
+            return None
+        if loss_out is None:
+            loss_out = np.zeros((self.N, 2), dtype=np.float64)
+        self._check(self.lib.pbt_step_prefetched(self.handle, loss_out.ctypes.data_as(C.POINTER(C.c_double))))
         return loss_out
 
     def launch_count(self) -> int:

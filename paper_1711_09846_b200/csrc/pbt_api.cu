@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "pbt_common.cuh"
@@ -65,6 +66,14 @@ struct pbt_handle {
   void* dz[2];                   // ping-pong deltas [N][dz_rows_cap][max_width]
   void* ybatch;
   long long ybatch_stride;  // elements of the target type per member
+  // second copy of the training-row buffers: host batches are uploaded here on a copy stream while the step
+  // on the current buffers runs (pbt_prefetch_host_batch / pbt_step_prefetched)
+  void* act0_alt;
+  void* ybatch_alt;
+  cudaStream_t copy_stream;
+  cudaEvent_t ev_copied, ev_stepdone[2];
+  bool prefetched;
+  long long pf_steps;  // prefetched steps taken so far
   float* row_loss;
   double* ed_partial;
   size_t workspace_bytes;
@@ -237,8 +246,12 @@ size_t plan(pbt_handle* h, char* base) {
     const size_t tsz = s.loss == PBT_LOSS_CE_SOFT ? h->esz : 4;
     h->ybatch_stride = (h->ybatch_stride * tsz + 15) / 16 * 16 / tsz;
     h->ybatch = take(N * (size_t)h->ybatch_stride * tsz);
+    h->ybatch_alt = take(N * (size_t)h->ybatch_stride * tsz);
+    h->act0_alt = take(N * (size_t)s.batch * h->st[0].L[0].in * h->esz);
   } else {
     h->ybatch = nullptr;
+    h->ybatch_alt = nullptr;
+    h->act0_alt = nullptr;
     h->ybatch_stride = 0;
   }
   h->row_loss = (float*)take(N * (size_t)h->rowloss_cap * sizeof(float));
@@ -668,6 +681,13 @@ int pbt_create(pbt_t** out, const pbt_spec* spec, const double* init_hparams, ui
 int pbt_destroy(pbt_t* p) {
   if (!p) return PBT_OK;
   if (p->step_graph) cudaGraphExecDestroy(p->step_graph);
+  if (p->copy_stream) {
+    cudaStreamSynchronize(p->copy_stream);
+    cudaEventDestroy(p->ev_copied);
+    cudaEventDestroy(p->ev_stepdone[0]);
+    cudaEventDestroy(p->ev_stepdone[1]);
+    cudaStreamDestroy(p->copy_stream);
+  }
   for (auto& r : p->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
   for (auto e : p->event_pool) cudaEventDestroy(e);
   delete p;
@@ -1014,6 +1034,54 @@ int pbt_step_host(pbt_t* p, const void* x_host, const void* y_host, double* loss
   CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &one, 4, cudaMemcpyHostToDevice, p->stream));
   int rc = one_step(p);
   if (rc) return rc;
+  if (loss_out_host) {
+    float* tmp = p->host_loss.data();
+    CU(p, cudaMemcpyAsync(tmp, p->last_loss, (size_t)p->N * 2 * 4, cudaMemcpyDeviceToHost, p->stream));
+    CU(p, cudaStreamSynchronize(p->stream));
+    for (int i = 0; i < p->N * 2; ++i) loss_out_host[i] = tmp[i];
+  }
+  return PBT_OK;
+}
+
+int pbt_prefetch_host_batch(pbt_t* p, const void* x_host, const void* y_host) {
+  if (!p || !x_host || !y_host) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  if (p->toy || p->gan) return fail(p, PBT_ERR_UNSUPPORTED, "host-fed steps are for MLP populations");
+  if (!p->copy_stream) {
+    CU(p, cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking));
+    CU(p, cudaEventCreateWithFlags(&p->ev_copied, cudaEventDisableTiming));
+    CU(p, cudaEventCreateWithFlags(&p->ev_stepdone[0], cudaEventDisableTiming));
+    CU(p, cudaEventCreateWithFlags(&p->ev_stepdone[1], cudaEventDisableTiming));
+  }
+  if (p->prefetched) return fail(p, PBT_ERR_STATE, "the previously prefetched batch has not been consumed yet");
+  // the spare buffers were the active ones of the step BEFORE the latest one (which may still be running)
+  if (p->pf_steps >= 2) CU(p, cudaStreamWaitEvent(p->copy_stream, p->ev_stepdone[p->pf_steps & 1], 0));
+  const pbt_spec& s = p->spec;
+  const size_t xb = (size_t)p->N * s.batch * p->st[0].L[0].in * p->esz;
+  CU(p, cudaMemcpyAsync(p->act0_alt, x_host, xb, cudaMemcpyHostToDevice, p->copy_stream));
+  const size_t trb = target_row_bytes(p) * s.batch;
+  const size_t tsz = s.loss == PBT_LOSS_CE_SOFT ? p->esz : 4;
+  CU(p, cudaMemcpy2DAsync(p->ybatch_alt, p->ybatch_stride * tsz, y_host, trb, trb, p->N, cudaMemcpyHostToDevice, p->copy_stream));
+  CU(p, cudaEventRecord(p->ev_copied, p->copy_stream));
+  p->prefetched = true;
+  return PBT_OK;
+}
+
+int pbt_step_prefetched(pbt_t* p, double* loss_out_host) {
+  if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  if (!p->prefetched) return fail(p, PBT_ERR_STATE, "no batch has been prefetched");
+  p->launches = 0;
+  p->prefetched = false;
+  CU(p, cudaStreamWaitEvent(p->stream, p->ev_copied, 0));
+  // the uploaded buffers become the current ones; a captured step graph holds the old addresses
+  std::swap(p->act[0][0], p->act0_alt);
+  std::swap(p->ybatch, p->ybatch_alt);
+  if (p->step_graph) { cudaGraphExecDestroy(p->step_graph); p->step_graph = nullptr; }
+  const int one = 1;
+  CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &one, 4, cudaMemcpyHostToDevice, p->stream));
+  int rc = one_step(p);
+  if (rc) return rc;
+  CU(p, cudaEventRecord(p->ev_stepdone[p->pf_steps & 1], p->stream));
+  p->pf_steps++;
   if (loss_out_host) {
     float* tmp = p->host_loss.data();
     CU(p, cudaMemcpyAsync(tmp, p->last_loss, (size_t)p->N * 2 * 4, cudaMemcpyDeviceToHost, p->stream));

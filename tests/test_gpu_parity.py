@@ -315,6 +315,40 @@ def test_supplied_batch_matches_oracle(pkg):
     gpu.close()
 
 
+def test_host_fed_steps_plain_and_prefetched_agree(pkg):
+    import torch
+    cfg = get_config("c3_mini")
+    inp = make_inputs(cfg)
+    rng = np.random.default_rng(9)
+    xs = [torch.from_numpy(rng.random((cfg.n_members, cfg.batch, cfg.widths[0][0])).astype(np.float32)).bfloat16().pin_memory()
+          for _ in range(3)]
+    ys = [torch.from_numpy(rng.integers(0, 10, size=(cfg.n_members, cfg.batch)).astype(np.int32)).pin_memory() for _ in range(3)]
+    a, b = pkg.Population(cfg, inp), pkg.Population(cfg, inp)
+    la = [a.step_host(x, y).copy() for x, y in zip(xs, ys)]
+    b.prefetch_host_batch(xs[0], ys[0])
+    lb = []
+    for j in range(3):
+        b.step_prefetched(wait=False)
+        if j + 1 < 3:
+            b.prefetch_host_batch(xs[j + 1], ys[j + 1])      # uploads while step j runs
+            with pytest.raises(pkg.PbtError) as e:           # one batch may be pending at a time
+                b.prefetch_host_batch(xs[j + 1], ys[j + 1])
+            assert e.value.code == 6
+        lb.append(b.last_loss().copy())
+    with pytest.raises(pkg.PbtError) as e:
+        b.step_prefetched()
+    assert e.value.code == 6
+    assert all(np.array_equal(p, q) for p, q in zip(la, lb))
+    b.step(1)                                                 # pool-window steps still work after the buffer swaps
+    a.step(1)
+    for m in range(cfg.n_members):
+        sa, sb = a.get_state(m), b.get_state(m)
+        for key in ("w", "opt1", "opt2"):
+            assert np.array_equal(sa[key], sb[key])
+    a.close()
+    b.close()
+
+
 def test_invalid_arguments_are_reported_not_fatal(pkg):
     cfg = get_config("c2_mini")
     inp = make_inputs(cfg)
