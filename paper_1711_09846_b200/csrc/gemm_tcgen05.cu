@@ -15,27 +15,13 @@
 // word, all roles leave their loops, tensor memory is released and the kernel returns normally.
 #include <string.h>
 
-#include "tc_common.cuh"
+#include "tc_epilogue.cuh"
 
 namespace pbt {
 
 namespace {
 
 using namespace tc;
-
-constexpr int kBM = 128;
-constexpr int kBK = 64;
-constexpr int kEpiPitch = 36;  // floats per row of the epilogue transpose buffer (16-byte aligned, conflict-free)
-
-struct TcParams {
-  int M, N, K, batch;
-  int tiles_m, tiles_n, num_tiles, k_blocks;
-  int a_mn, b_mn, a_batched, b_batched;
-  void* C; long long ldc, strideC; int out_dtype;
-  const float* bias; long long strideBias; int relu;
-  const bf16* mask; long long ldmask, strideMask;
-  Counters* counters;
-};
 
 template <int BN, int STAGES, int NEPIW>
 struct Smem {
@@ -171,7 +157,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     const bool vec_ok = (((uintptr_t)p.C & 15) == 0) && ((p.ldc * esz) % 16 == 0) && ((p.strideC * esz) % 16 == 0) &&
                         (!p.mask || ((((uintptr_t)p.mask & 7) == 0) && (p.ldmask % 4 == 0) && (p.strideMask % 4 == 0))) &&
                         (!p.bias || ((((uintptr_t)p.bias & 15) == 0) && (p.strideBias % 4 == 0)));
-    const int rsub = lane >> 3, cc = (lane & 7) * 4;   // phase 2: 4 rows x 8 column-quads per warp instruction
     for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++it) {
       const int member = tile / (p.tiles_m * p.tiles_n);
       const int rem = tile % (p.tiles_m * p.tiles_n);
@@ -180,99 +165,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       const uint32_t acc_phase = (it >> 1) & 1;
       if (!mbar_wait(&tfull[acc], acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const float* bias = p.bias ? p.bias + member * p.strideBias : nullptr;
-      // The accumulator chunk for iteration c+1 is requested from tensor memory while chunk c is being
-      // transposed and written out, and the ReLU-mask words are requested before the transpose, so that
-      // neither latency sits on the warp's critical path.
-      constexpr int kChunkStep = 32 * (NEPIW / 4);
-      uint32_t r[32];
-      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-      if (n0 + half * 32 < p.N) tmem_ld32(tacc + half * 32, r);
-#pragma unroll 1
-      for (int c0 = half * 32; c0 < BN; c0 += kChunkStep) {
-        const int nbase = n0 + c0;
-        if (nbase >= p.N) break;  // uniform across the warp
-        const int col = nbase + cc;
-        const bool full4 = vec_ok && col + 3 < p.N;
-        uint2 mk[8];
-        if (p.mask && full4) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int row = m0 + q * 32 + i * 4 + rsub;
-            mk[i] = row < p.M ? __ldg(reinterpret_cast<const uint2*>(p.mask + member * p.strideMask + (long long)row * p.ldmask + col))
-                              : make_uint2(0u, 0u);
-          }
-        }
-        tmem_ld_wait();
-        __syncwarp();  // the previous chunk's phase-2 reads of `buf` are complete
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          *reinterpret_cast<uint4*>(&buf[lane * kEpiPitch + j * 4]) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-        if (c0 + kChunkStep < BN && nbase + kChunkStep < p.N) tmem_ld32(tacc + c0 + kChunkStep, r);
-        __syncwarp();
-        {
-          float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (bias && col < p.N) {
-            if (full4) bv = __ldg(reinterpret_cast<const float4*>(bias + col));
-            else {
-              bv.x = bias[col];
-              if (col + 1 < p.N) bv.y = bias[col + 1];
-              if (col + 2 < p.N) bv.z = bias[col + 2];
-              if (col + 3 < p.N) bv.w = bias[col + 3];
-            }
-          }
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int rr = i * 4 + rsub;
-            const int row = m0 + q * 32 + rr;
-            if (row >= p.M || col >= p.N) continue;
-            const float4 a4 = *reinterpret_cast<const float4*>(&buf[rr * kEpiPitch + cc]);
-            float v[4] = {a4.x + bv.x, a4.y + bv.y, a4.z + bv.z, a4.w + bv.w};
-            if (p.relu) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) v[j] = fmaxf(v[j], 0.f);
-            }
-            if (p.mask) {
-              const bf16* mp = p.mask + member * p.strideMask + (long long)row * p.ldmask + col;
-              if (full4) {
-                const uint32_t w[2] = {mk[i].x, mk[i].y};
-#pragma unroll
-                for (int h2 = 0; h2 < 2; ++h2) {
-                  // bf16 > 0  <=>  sign bit clear and magnitude non-zero
-                  const uint32_t lo = w[h2] & 0xFFFFu, hi = w[h2] >> 16;
-                  if (!(lo != 0 && lo < 0x8000u)) v[h2 * 2] = 0.f;
-                  if (!(hi != 0 && hi < 0x8000u)) v[h2 * 2 + 1] = 0.f;
-                }
-              } else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                  if (col + j < p.N && !(__bfloat162float(mp[j]) > 0.f)) v[j] = 0.f;
-              }
-            }
-            const long long ci = member * p.strideC + (long long)row * p.ldc + col;
-            if (p.out_dtype == kBF16) {
-              bf16* cp = reinterpret_cast<bf16*>(p.C) + ci;
-              if (full4) {
-                __nv_bfloat162 t0 = __floats2bfloat162_rn(v[0], v[1]);
-                __nv_bfloat162 t1 = __floats2bfloat162_rn(v[2], v[3]);
-                uint2 o;
-                o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
-                *reinterpret_cast<uint2*>(cp) = o;
-              } else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) if (col + j < p.N) cp[j] = __float2bfloat16_rn(v[j]);
-              }
-            } else {
-              float* cp = reinterpret_cast<float*>(p.C) + ci;
-              if (full4) *reinterpret_cast<float4*>(cp) = make_float4(v[0], v[1], v[2], v[3]);
-              else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) if (col + j < p.N) cp[j] = v[j];
-              }
-            }
-          }
-        }
-      }
+      epilogue_tile<BN, NEPIW>(p, buf, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), member, m0, n0, q, half, lane, vec_ok);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tempty[acc]);
