@@ -284,7 +284,8 @@ int pbt_profile_get(pbt_t* p, const char* kernel_class, double* ms_total, int64_
  * max(.,0) (if relu), zero where mask[b*strideMask + m*ldmask + n] <= 0 (if mask; operand type).
  * Strides are in elements; a stride of 0 shares the operand between all problems.
  * engine: 0 = choose (tensor cores when operands are bf16 and the shape fills the tiles),
- * 1 = FP32-ALU kernel, 2 = tcgen05 kernel (PBT_ERR_UNSUPPORTED if the shape does not qualify).
+ * 1 = FP32-ALU kernels, 2 = tcgen05 kernel, one CTA per tile, 3 = tcgen05 kernel with CTA pairs (M, N >= 256);
+ * PBT_ERR_UNSUPPORTED if the shape does not qualify for the engine asked for.
  * status_device: 32 zeroed bytes of device memory; a bounded wait that expires inside the
  * tensor-core kernel stores PBT_ERR_TIMEOUT in the int32 at byte offset 16.  All pointers are
  * device pointers; the call only enqueues work on `stream`.

@@ -17,7 +17,7 @@ OUT = os.path.join(HERE, "libpbt_b200.so")
 OBJ = os.path.join(HERE, "_build")
 
 SOURCES = ["pbt_api.cu", "kernels_misc.cu", "kernels_opt.cu", "kernels_exploit.cu", "gemm_simt.cu",
-           "gemm_tcgen05.cu", "wgrad_adam_tcgen05.cu", "energy_static.cu"]
+           "gemm_tcgen05.cu", "gemm_tcgen05_pair.cu", "wgrad_adam_tcgen05.cu", "energy_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

@@ -316,6 +316,8 @@ struct LaunchScope {
 int gemm(pbt_handle* h, const GemmArgs& g) {
   if (g.adam) {
     LAUNCH(h, kFused, launch_wgrad_adam(g, h->counters, h->stream));
+  } else if (gemm_tc_pair_supported(g)) {
+    LAUNCH(h, kGemm, launch_gemm_tc_pair(g, h->counters, h->stream));
   } else if (gemm_tc_supported(g)) {
     LAUNCH(h, kGemm, launch_gemm_tc(g, h->counters, h->stream));
   } else {
@@ -1103,9 +1105,13 @@ int pbt_grouped_gemm(const pbt_gemm_desc* d, void* stream) {
   g.C = d->C; g.ldc = d->ldc; g.strideC = d->strideC;
   g.bias = d->bias; g.strideBias = d->strideBias; g.relu = d->relu;
   g.mask = d->mask; g.ldmask = d->ldmask; g.strideMask = d->strideMask;
-  const bool tc = gemm_tc_supported(g);
+  const bool tc = gemm_tc_supported(g), pair = gemm_tc_pair_supported(g);
   cudaError_t e;
-  if (d->engine == 2 || (d->engine == 0 && tc && d->status_device)) {
+  if (d->engine == 3 || (d->engine == 0 && pair && d->status_device)) {
+    if (!pair) return fail(nullptr, PBT_ERR_UNSUPPORTED, "shape / alignment does not qualify for the CTA-pair tensor-core kernel");
+    if (!d->status_device) return fail(nullptr, PBT_ERR_INVALID_ARG, "status_device is required by the tensor-core kernels");
+    e = launch_gemm_tc_pair(g, (Counters*)d->status_device, (cudaStream_t)stream);
+  } else if (d->engine == 2 || (d->engine == 0 && tc && d->status_device)) {
     if (!tc) return fail(nullptr, PBT_ERR_UNSUPPORTED, "shape / alignment does not qualify for the tensor-core kernel");
     if (!d->status_device) return fail(nullptr, PBT_ERR_INVALID_ARG, "status_device is required by the tensor-core kernel");
     e = launch_gemm_tc(g, (Counters*)d->status_device, (cudaStream_t)stream);

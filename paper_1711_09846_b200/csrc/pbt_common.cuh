@@ -84,6 +84,9 @@ cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t s);
 // tensor-core path; returns cudaErrorNotSupported when the shape does not qualify
 bool gemm_tc_supported(const GemmArgs& g);
 cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s);
+// CTA-pair variant (256 x 256 tiles shared by two CTAs of a cluster) for shapes with M, N >= 256
+bool gemm_tc_pair_supported(const GemmArgs& g);
+cudaError_t launch_gemm_tc_pair(const GemmArgs& g, Counters* counters, cudaStream_t s);
 // weight gradient with the Adam update applied in the same kernel (g.adam must be set; tensor-core shapes only)
 cudaError_t launch_wgrad_adam(const GemmArgs& g, Counters* counters, cudaStream_t s);
 

@@ -112,3 +112,21 @@ def test_unsupported_shapes_are_refused_by_the_tensor_engine(env):
     with pytest.raises(pkg.PbtError) as e:
         pkg.grouped_gemm(A, A, Cd, engine=2, status=status)
     assert e.value.code == 2
+
+
+@pytest.mark.parametrize("a_mn,b_mn,epilogue,out_bf16", [(False, False, "none", False), (False, False, "bias_relu", True),
+                                                         (False, True, "mask", True), (True, True, "none", False)])
+@pytest.mark.parametrize("shape", [(256, 256, 64, 1), (512, 512, 256, 3), (304, 328, 136, 2), (512, 2048, 512, 2),
+                                   (768, 1024, 320, 5)])
+def test_tensor_core_cta_pairs(env, a_mn, b_mn, epilogue, out_bf16, shape):
+    """tcgen05 cta_group::2: two CTAs of a cluster share a 256 x 256 tile (engine 3)."""
+    pkg, torch = env
+    M, N, K, batch = shape
+    _run(pkg, torch, M, N, K, batch, a_mn, b_mn, engine=3, epilogue=epilogue, out_bf16=out_bf16, seed=17)
+
+
+def test_tensor_core_cta_pairs_many_tiles(env):
+    pkg, torch = env
+    # 2 x 4 x 12 = 96 pair tiles on 74 CTA pairs: the persistent loop and both accumulator buffers cycle
+    _run(pkg, torch, 512, 1024, 256, 12, False, False, engine=3, epilogue="bias_relu", out_bf16=True, seed=19)
+    _run(pkg, torch, 512, 1024, 256, 12, False, True, engine=3, epilogue="mask", out_bf16=True, seed=20)
