@@ -65,7 +65,12 @@ typedef enum pbt_loss {
   PBT_LOSS_GAN_LOGISTIC = 4 /* non-saturating logistic GAN losses */
 } pbt_loss;
 
-typedef enum pbt_optimizer { PBT_OPT_SGD_PLAIN = 0, PBT_OPT_SGDM = 1, PBT_OPT_ADAM = 2 } pbt_optimizer;
+typedef enum pbt_optimizer {
+  PBT_OPT_SGD_PLAIN = 0,
+  PBT_OPT_SGDM = 1,
+  PBT_OPT_ADAM = 2,
+  PBT_OPT_RMSPROP = 3 /* ms <- rho ms + (1-rho) g^2, theta <- theta - lr g / (sqrt(ms) + eps); rho = const_beta2; ms in opt1 */
+} pbt_optimizer;
 
 /* exploit / explore switches ("PBT targets" ablation, Section 4.4) */
 #define PBT_COPY_WEIGHTS 1u  /* exploit copies weights and optimiser state */

@@ -217,6 +217,13 @@ def sgdm_update(theta, vel, g, lr, mu):
     return theta - lr * vel, vel
 
 
+def rmsprop_update(theta, ms, g, lr, rho, eps):
+    """RMSProp (Tieleman & Hinton, 2012), the optimiser of the paper's RL experiments (Section 4.1.1):
+    ms <- rho ms + (1 - rho) g^2;  theta <- theta - lr g / (sqrt(ms) + eps)."""
+    ms = rho * ms + (1.0 - rho) * g * g
+    return theta - lr * g / (np.sqrt(ms) + eps), ms
+
+
 def adam_update(theta, m, v, g, lr, b1, b2, eps, wd, c1, c2):
     """m <- b1 m + (1-b1) g; v <- b2 v + (1-b2) g^2;
     theta <- theta - lr (m/(1-c1)) / (sqrt(v/(1-c2)) + eps) - lr wd theta,
@@ -352,6 +359,13 @@ class Population:
                     th, vel = sgdm_update(P[m][t].astype(np.float64), O[m][t].astype(np.float64),
                                           _f32(g).astype(np.float64), lr, mu)
                     P[m][t], O[m][t] = _f32(th), _f32(vel)
+        elif cfg.optimizer == "rmsprop":
+            rho, eps = float(np.float32(cfg.beta2)), float(np.float32(cfg.eps))
+            for t in ts:
+                for P, O, g in ((self.W, self.o1W, gW[t]), (self.b, self.o1b, gb[t])):
+                    th, ms = rmsprop_update(P[m][t].astype(np.float64), O[m][t].astype(np.float64),
+                                            _f32(g).astype(np.float64), lr, rho, eps)
+                    P[m][t], O[m][t] = _f32(th), _f32(ms)
         elif cfg.optimizer == "adam":
             b1 = self._hp(m, "beta1", cfg.beta1)
             b2 = float(np.float32(cfg.beta2))

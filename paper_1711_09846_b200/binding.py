@@ -21,7 +21,7 @@ PBT_N_SCALARS = 4
 _DTYPE = {"fp64_toy": 0, "fp32": 1, "bf16_fp32master": 2}
 _MODEL = {"toy_quadratic": 0, "mlp": 1, "gan_pair": 2}
 _LOSS = {"toy": 0, "mse": 1, "ce_hard": 2, "ce_soft": 3, "gan_logistic": 4}
-_OPT = {"sgd_plain": 0, "sgdm": 1, "adam": 2}
+_OPT = {"sgd_plain": 0, "sgdm": 1, "adam": 2, "rmsprop": 3}
 
 STATUS = {0: "PBT_OK", 1: "PBT_ERR_INVALID_ARG", 2: "PBT_ERR_UNSUPPORTED", 3: "PBT_ERR_WORKSPACE",
           4: "PBT_ERR_CUDA", 5: "PBT_ERR_TIMEOUT", 6: "PBT_ERR_STATE"}

@@ -92,6 +92,36 @@ __global__ void __launch_bounds__(kOptThreads) k_adam(OptArgs a) {
   }
 }
 
+// ms <- rho ms + (1-rho) g^2 ; theta <- theta - lr g / (sqrt(ms) + eps)
+__global__ void __launch_bounds__(kOptThreads) k_rmsprop(OptArgs a) {
+  const int m = blockIdx.y;
+  const float* Hrow = a.H + (long long)m * a.nh_stride;
+  const float lr = hp(Hrow, a.slot_lr, a.const_lr);
+  const float rho = a.const_beta2, omr = 1.f - a.const_beta2, eps = a.const_eps;
+  const long long base = (long long)m * a.p_pad + a.begin;
+  float* w = a.w32 + base;
+  float* ms = a.opt1 + base;
+  const float* g = a.grad + base;
+  bf16* w16 = a.w16 ? a.w16 + base : nullptr;
+  for (long long t0 = (long long)blockIdx.x * kOptTile; t0 < a.count; t0 += (long long)gridDim.x * kOptTile) {
+#pragma unroll
+    for (int j = 0; j < kOptVecPerThread; ++j) {
+      const long long i = t0 + ((long long)j * kOptThreads + threadIdx.x) * 4;
+      if (i < a.count) {
+        const float4 gw = ld_stream(g + i), ww = ld_stream(w + i), vv = ld_stream(ms + i);
+        float4 nv, nw;
+        nv.x = __fmaf_rn(rho, vv.x, omr * gw.x * gw.x); nv.y = __fmaf_rn(rho, vv.y, omr * gw.y * gw.y);
+        nv.z = __fmaf_rn(rho, vv.z, omr * gw.z * gw.z); nv.w = __fmaf_rn(rho, vv.w, omr * gw.w * gw.w);
+        nw.x = ww.x - lr * __fdividef(gw.x, sqrtf(nv.x) + eps); nw.y = ww.y - lr * __fdividef(gw.y, sqrtf(nv.y) + eps);
+        nw.z = ww.z - lr * __fdividef(gw.z, sqrtf(nv.z) + eps); nw.w = ww.w - lr * __fdividef(gw.w, sqrtf(nv.w) + eps);
+        st_stream(ms + i, nv);
+        st_stream(w + i, nw);
+        if (w16) st_bf16x4(w16 + i, nw);
+      }
+    }
+  }
+}
+
 // after the Adam pass of a stack: store the advanced beta products
 __global__ void k_adam_advance(OptArgs a) {
   const int m = blockIdx.x * blockDim.x + threadIdx.x;
@@ -116,6 +146,11 @@ static unsigned opt_grid_x(const OptArgs& a) {
 cudaError_t launch_sgdm(const OptArgs& a, cudaStream_t s) {
   dim3 grid(opt_grid_x(a), a.n_members);
   k_sgdm<<<grid, kOptThreads, 0, s>>>(a);
+  return cudaGetLastError();
+}
+cudaError_t launch_rmsprop(const OptArgs& a, cudaStream_t s) {
+  dim3 grid(opt_grid_x(a), a.n_members);
+  k_rmsprop<<<grid, kOptThreads, 0, s>>>(a);
   return cudaGetLastError();
 }
 cudaError_t launch_adam(const OptArgs& a, cudaStream_t s) {

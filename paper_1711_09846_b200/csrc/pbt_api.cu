@@ -135,8 +135,8 @@ int validate(const pbt_spec* s) {
   if (s->model != PBT_MLP && s->model != PBT_GAN_PAIR) return fail(nullptr, PBT_ERR_INVALID_ARG, "unknown model");
   if (s->dtype != PBT_FP32 && s->dtype != PBT_BF16_FP32MASTER)
     return fail(nullptr, PBT_ERR_UNSUPPORTED, "networks run in fp32 or bf16 with fp32 masters");
-  if (s->optimizer != PBT_OPT_SGDM && s->optimizer != PBT_OPT_ADAM)
-    return fail(nullptr, PBT_ERR_UNSUPPORTED, "network optimiser must be SGD-momentum or Adam");
+  if (s->optimizer != PBT_OPT_SGDM && s->optimizer != PBT_OPT_ADAM && s->optimizer != PBT_OPT_RMSPROP)
+    return fail(nullptr, PBT_ERR_UNSUPPORTED, "network optimiser must be SGD-momentum, RMSProp or Adam");
   const int ns = s->model == PBT_GAN_PAIR ? 2 : 1;
   for (int k = 0; k < ns; ++k) {
     if (s->n_layers[k] < 1 || s->n_layers[k] > PBT_MAX_LAYERS) return fail(nullptr, PBT_ERR_INVALID_ARG, "n_layers out of range");
@@ -430,6 +430,7 @@ int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride
     a.begin = rb; a.count = re - rb;
     rb = re = -1;
     if (s.optimizer == PBT_OPT_SGDM) { LAUNCH(h, kOpt, launch_sgdm(a, h->stream)); }
+    else if (s.optimizer == PBT_OPT_RMSPROP) { LAUNCH(h, kOpt, launch_rmsprop(a, h->stream)); }
     else { LAUNCH(h, kOpt, launch_adam(a, h->stream)); }
     return PBT_OK;
   };

@@ -102,6 +102,7 @@ struct OptArgs {
 };
 cudaError_t launch_sgdm(const OptArgs& a, cudaStream_t s);
 cudaError_t launch_adam(const OptArgs& a, cudaStream_t s);
+cudaError_t launch_rmsprop(const OptArgs& a, cudaStream_t s);
 cudaError_t launch_adam_advance(const OptArgs& a, cudaStream_t s);
 
 // ---- device helpers shared by the optimiser kernel and the fused weight-gradient epilogue ----

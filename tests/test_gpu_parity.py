@@ -156,6 +156,12 @@ def _check_optimizer_arithmetic(cfg, s0, s1, h):
     if cfg.optimizer == C.OPT_SGDM:
         w, m = O.sgdm_update(w0, m0, g, lr, h[cfg.slot("momentum")])
         v = v0
+    elif cfg.optimizer == C.OPT_RMSPROP:
+        w, m = O.rmsprop_update(w0, m0, g, lr, float(np.float32(cfg.beta2)), float(np.float32(cfg.eps)))
+        v = v0
+        np.testing.assert_allclose(s1["opt1"], m, rtol=2e-6, atol=2e-7 * max(np.abs(m0).max(), (g * g).max()))
+        np.testing.assert_allclose(s1["w"], w, rtol=2e-6, atol=1e-5 * lr)
+        return
     else:
         b1 = h[cfg.slot("beta1")] if cfg.slot("beta1") >= 0 else float(np.float32(cfg.beta1))
         wd = h[cfg.slot("wd")] if cfg.slot("wd") >= 0 else cfg.weight_decay
@@ -170,7 +176,8 @@ def _check_optimizer_arithmetic(cfg, s0, s1, h):
 # ---------------------------------------------------------------------------
 # step / eval parity, step by step, re-seeding the GPU from the oracle at ready points
 # ---------------------------------------------------------------------------
-@pytest.mark.parametrize("name", ["c2_mini", "c3_mini", "c4_mini", "c5_mini", "c3_mid", "c5_mid", "c4_mid"])
+@pytest.mark.parametrize("name", ["c2_mini", "c3_mini", "c4_mini", "c5_mini", "c3_mid", "c5_mid", "c4_mid", "c2_mini_rms",
+                                  "c3_mini_rms"])
 def test_step_eval_exploit_parity(pkg, name):
     cfg = get_config(name)
     inp = make_inputs(cfg)
@@ -178,7 +185,7 @@ def test_step_eval_exploit_parity(pkg, name):
     gpu, cpu = pkg.Population(cfg, inp, keep_grad=True), O.Population(cfg, inp)
     tol = _tol(cfg)
     ftol = 1e-4 if cfg.dtype == C.FP32 else 2e-2
-    keys = ("w", "opt1", "grad") if cfg.optimizer == C.OPT_SGDM else ("w", "opt1", "opt2", "grad")
+    keys = ("w", "opt1", "opt2", "grad") if cfg.optimizer == C.OPT_ADAM else ("w", "opt1", "grad")
     for t in range(1, cfg.total_steps + 1):
         before = [gpu.get_state(m) for m in range(cfg.n_members)]
         h_now = gpu.hparams()

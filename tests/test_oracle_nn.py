@@ -313,3 +313,38 @@ def test_grouped_gemm_against_triple_loop():
                 assert abs(got[b, m, n] - s) < 1e-13
     plain = O.grouped_gemm(A, B)
     assert abs(plain[1, 2, 3] - float(A[1, 2] @ B[1, 3])) < 1e-13
+
+
+def test_rmsprop_hand_trajectory_and_torch_optimizer():
+    # g = 1, rho = 0.9, lr = 0.1, eps = 0: ms = 0.1, 0.19; theta = -0.1/sqrt(0.1), then - 0.1/sqrt(0.19) more
+    th, ms = np.array([0.0]), np.array([0.0])
+    th, ms = O.rmsprop_update(th, ms, np.array([1.0]), 0.1, 0.9, 0.0)
+    assert abs(ms[0] - 0.1) < 1e-15 and abs(th[0] + 0.1 / math.sqrt(0.1)) < 1e-15
+    th, ms = O.rmsprop_update(th, ms, np.array([1.0]), 0.1, 0.9, 0.0)
+    assert abs(ms[0] - 0.19) < 1e-15 and abs(th[0] + 0.1 / math.sqrt(0.1) + 0.1 / math.sqrt(0.19)) < 1e-15
+    # against torch.optim.RMSprop (no momentum, not centred) on a random gradient sequence
+    rng = np.random.default_rng(21)
+    g = rng.standard_normal((6, 5))
+    w = torch.zeros(5, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.RMSprop([w], lr=3e-3, alpha=0.99, eps=1e-8)
+    th, ms = np.zeros(5), np.zeros(5)
+    for t in range(6):
+        w.grad = torch.tensor(g[t])
+        opt.step()
+        th, ms = O.rmsprop_update(th, ms, g[t], 3e-3, 0.99, 1e-8)
+        np.testing.assert_allclose(th, w.detach().numpy(), rtol=1e-12, atol=1e-15)
+
+
+def test_rmsprop_population_step_uses_the_gradient_of_the_loss():
+    rng = np.random.default_rng(22)
+    cfg = _mlp_cfg(C.LOSS_MSE, (4, 3, 2), n=1, batch=8).replace(optimizer=C.OPT_RMSPROP, slots=("lr",),
+                                                                priors=(("fixed", 0, 0),), perturb=(True,),
+                                                                clamp_lo=(-math.inf,), clamp_hi=(math.inf,), beta2=0.9)
+    inp = _inputs(cfg, rng, [1e-2])
+    pop = O.Population(cfg, inp, seed=3)
+    w0 = pop.W[0][0].astype(np.float64).copy()
+    pop.step(1)
+    g = pop.gW[0][0].astype(np.float64)
+    expect = w0 - 1e-2 * g / (np.sqrt(0.1 * g * g) + float(np.float32(1e-8)))
+    np.testing.assert_allclose(pop.W[0][0], expect, rtol=2e-6, atol=1e-9)
+    np.testing.assert_allclose(pop.o1W[0][0], np.float32(1.0 - np.float32(0.9)) * g * g, rtol=2e-6)

@@ -50,7 +50,7 @@ def adam_well_conditioned(cfg, cpu_state, tol_g):
 
 def assert_state_close(cfg, gpu_state, cpu_state, keys, tol, what=""):
     keep = None
-    if cfg.optimizer == "adam" and "w" in keys and "grad" in cpu_state:
+    if cfg.optimizer in ("adam", "rmsprop") and "w" in keys and "grad" in cpu_state:
         keep = adam_well_conditioned(cfg, cpu_state, tol.get("grad", 2e-2))
     for key in keys:
         for name, sl in tensor_slices(cfg):

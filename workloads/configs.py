@@ -35,6 +35,7 @@ LOSS_GAN = "gan_logistic"
 OPT_SGD = "sgd_plain"
 OPT_SGDM = "sgdm"
 OPT_ADAM = "adam"
+OPT_RMSPROP = "rmsprop"   # beta2 is the decay of the mean square
 
 COPY_WEIGHTS = 1
 COPY_HPARAMS = 2
@@ -173,6 +174,13 @@ CONFIGS: Dict[str, PBTConfig] = {
                    pool=512, interval=2, steps=6, name="c4_mini"),
     "c5_mini": _c5(n=10, widths=(128, 192, 256, 136, 72), batch=136, eval_batch=200,
                    pool=768, interval=2, steps=6, name="c5_mini"),
+    # RMSProp (the optimiser of the paper's RL experiments) on the same small shapes; learning rate is the only slot
+    "c2_mini_rms": _c2(n=5, widths=(40, 72, 56, 1), batch=24, eval_batch=40, pool=512, interval=3, steps=6,
+                       name="c2_mini_rms").replace(optimizer=OPT_RMSPROP, slots=("lr",), priors=(("logu", 1e-4, 1e-2),),
+                                                   perturb=(True,), clamp_lo=(-INF,), clamp_hi=(INF,), beta2=0.99),
+    "c3_mini_rms": _c3(n=6, widths=(72, 136, 200, 10), batch=40, eval_batch=96, pool=640, interval=3, steps=6,
+                       name="c3_mini_rms").replace(optimizer=OPT_RMSPROP, slots=("lr",), priors=(("logu", 1e-5, 1e-3),),
+                                                   perturb=(True,), clamp_lo=(-INF,), clamp_hi=(INF,), beta2=0.99),
     # mid-size: every big layer is a multiple of the tensor-core tile so the
     # tcgen05 path is exercised, still seconds on a CPU
     "c3_mid": _c3(n=4, widths=(784, 1024, 1024, 10), batch=256, eval_batch=512, pool=2048,
