@@ -117,7 +117,8 @@ typedef struct pbt_spec {
   int32_t fuse_adam; /* 1: apply Adam inside the epilogue of tensor-core weight-gradient GEMMs (the gradient of those
                         layers never goes to HBM); 0: weight gradients are written once and one streaming pass over
                         the slabs applies the update.  Results are bit-identical; only the traffic pattern differs. */
-  int32_t reserved1;
+  int32_t exploit_rule; /* 0: truncation selection (Section 4.1.1 (b)); 1: binary tournament (Section 4.3.1 (b)): every
+                           member draws one other member uniformly and copies it if its fitness is strictly higher */
   double const_lr, const_momentum, const_beta1, const_beta2, const_eps, const_wd;
   double toy_eta;                 /* toy step size */
   double toy_theta0[PBT_MAX_NH];  /* toy initial theta (same for all members) */

@@ -118,6 +118,25 @@ def truncation_select(fitness, seed: int, rnd: int, num: int = 1, den: int = 5) 
     return src
 
 
+def tournament_select(fitness, seed: int, rnd: int) -> np.ndarray:
+    """Binary tournament (Section 4.3.1 (b)): every member draws one OTHER member uniformly and copies it if that
+    member's score is strictly better (NaN counts as the worst score).  src[i] == i where nothing is copied.
+    All decisions use the fitness vector as it stands before any copy."""
+    n = len(fitness)
+    src = np.arange(n, dtype=np.int32)
+    if n < 2:
+        return src
+    f = [(-math.inf if math.isnan(float(x)) else float(x)) for x in fitness]
+    for i in range(n):
+        word = px.draw(seed, i, rnd, px.STREAM_EXPLOIT, 1)[0]
+        j = donor_index(word, n - 1)
+        if j >= i:
+            j += 1
+        if f[j] > f[i]:
+            src[i] = j
+    return src
+
+
 def explore_bits(seed: int, member: int, rnd: int, nh: int) -> List[int]:
     """One bit per hyperparameter slot: 1 -> multiply by the high factor, 0 -> low."""
     bits = []
@@ -487,14 +506,21 @@ class Population:
     # ----- exploit + explore at a ready point ---------------------------------
     def exploit_explore(self):
         cfg = self.cfg
-        src = truncation_select(self.fitness, self.seed, self.round, cfg.trunc_num, cfg.trunc_den)
+        if getattr(cfg, "exploit", "truncation") == "tournament":
+            src = tournament_select(self.fitness, self.seed, self.round)
+        else:
+            src = truncation_select(self.fitness, self.seed, self.round, cfg.trunc_num, cfg.trunc_den)
         copied = [b for b in range(self.N) if src[b] != b]
+        # every copy reads the donor's record as it was BEFORE this ready point (under the tournament rule a
+        # donor may itself be a recipient), so the donors are snapshotted first
+        old_H, old_fit = self.H.copy(), self.fitness.copy()
+        snap = {int(src[b]): self._snapshot_member(int(src[b])) for b in copied} if cfg.flags & COPY_WEIGHTS else {}
         for b in copied:
             d = int(src[b])
             if cfg.flags & COPY_WEIGHTS:
-                self._copy_member(b, d)
+                self._restore_member(b, snap[d])
             if cfg.flags & COPY_HPARAMS:
-                self.H[b] = self.H[d]
+                self.H[b] = old_H[d]
         if cfg.flags & EXPLORE:
             for b in copied:
                 bits = explore_bits(self.seed, b, self.round, cfg.nh)
@@ -503,10 +529,25 @@ class Population:
         if cfg.flags & COPY_WEIGHTS:
             for b in copied:
                 # eval depends on the weights only, so the copy's performance is the donor's
-                self.fitness[b] = self.fitness[int(src[b])]
+                self.fitness[b] = old_fit[int(src[b])]
         self.src = src
         self.round += 1
         return src
+
+    def _snapshot_member(self, m):
+        if self.toy:
+            return self.theta[m].copy()
+        return ([[x.copy() for x in A[m]] for A in (self.W, self.b, self.o1W, self.o1b, self.o2W, self.o2b)],
+                self.scalars[m].copy())
+
+    def _restore_member(self, dst, snap):
+        if self.toy:
+            self.theta[dst] = snap
+            return
+        arrays, scalars = snap
+        for A, rows in zip((self.W, self.b, self.o1W, self.o1b, self.o2W, self.o2b), arrays):
+            A[dst] = [x.copy() for x in rows]
+        self.scalars[dst] = scalars
 
     def _copy_member(self, dst, src):
         if self.toy:

@@ -37,7 +37,7 @@ class PbtSpec(C.Structure):
         ("slot_lr", C.c_int32), ("slot_lr_d", C.c_int32), ("slot_momentum", C.c_int32),
         ("slot_beta1", C.c_int32), ("slot_wd", C.c_int32),
         ("perturb_mask", C.c_uint32), ("flags", C.c_uint32),
-        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("reserved1", C.c_int32),
+        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("exploit_rule", C.c_int32),
         ("const_lr", C.c_double), ("const_momentum", C.c_double), ("const_beta1", C.c_double),
         ("const_beta2", C.c_double), ("const_eps", C.c_double), ("const_wd", C.c_double),
         ("toy_eta", C.c_double), ("toy_theta0", C.c_double * PBT_MAX_NH),
@@ -166,6 +166,7 @@ def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True) -> Pb
     s.flags = cfg.flags
     s.trunc_num, s.trunc_den = cfg.trunc_num, cfg.trunc_den
     s.keep_grad = 1 if keep_grad else 0
+    s.exploit_rule = {"truncation": 0, "tournament": 1}[getattr(cfg, "exploit", "truncation")]
     s.fuse_adam = 1 if fuse_adam else 0
     s.const_lr = 0.0
     s.const_momentum = cfg.momentum

@@ -58,6 +58,7 @@ struct pbt_handle {
   void* H;        // [N][PBT_MAX_NH] float (double for the toy)
   void* fitness;  // [N] float (double for the toy)
   int* src;
+  int* level;        // [N] copy pass of each recipient at the last ready point
   Counters* counters;
   float* last_loss;  // [N][2]
   double* theta;     // toy: [N][nh]
@@ -124,6 +125,7 @@ int validate(const pbt_spec* s) {
   if (s->n_members < 1 || s->n_members > 1024) return fail(nullptr, PBT_ERR_INVALID_ARG, "n_members must be in [1, 1024]");
   if (s->nh < 0 || s->nh > PBT_MAX_NH) return fail(nullptr, PBT_ERR_INVALID_ARG, "nh must be in [0, %d]", PBT_MAX_NH);
   if (s->trunc_num < 0 || s->trunc_den < 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "bad truncation fraction");
+  if (s->exploit_rule != 0 && s->exploit_rule != 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "unknown exploit rule");
   const int slots[5] = {s->slot_lr, s->slot_lr_d, s->slot_momentum, s->slot_beta1, s->slot_wd};
   for (int i = 0; i < 5; ++i)
     if (slots[i] < -1 || slots[i] >= s->nh) return fail(nullptr, PBT_ERR_INVALID_ARG, "hyperparameter slot out of range");
@@ -180,6 +182,7 @@ size_t plan(pbt_handle* h, char* base) {
   const size_t N = h->N;
   h->counters = (Counters*)take(sizeof(Counters));
   h->src = (int*)take(N * sizeof(int));
+  h->level = (int*)take(N * sizeof(int));
   h->H = take(N * PBT_MAX_NH * sizeof(double));
   h->fitness = take(N * sizeof(double));
   h->last_loss = (float*)take(N * 2 * sizeof(float));
@@ -784,32 +787,49 @@ int pbt_exploit_explore(pbt_t* p) {
   }
   a.n_cut = n_cut;
   a.h_is_double = p->toy ? 1 : 0;
-  a.H = p->H; a.fitness = p->fitness; a.src = p->src; a.counters = p->counters; a.seed = p->seed;
+  a.H = p->H; a.fitness = p->fitness; a.src = p->src; a.level = p->level; a.counters = p->counters; a.seed = p->seed;
+  a.rule = s.exploit_rule;
   a.perturb_mask = s.perturb_mask; a.flags = s.flags;
   a.factor_lo = s.factor_lo; a.factor_hi = s.factor_hi;
   for (int k = 0; k < PBT_MAX_NH; ++k) { a.clamp_lo[k] = s.clamp_lo[k]; a.clamp_hi[k] = s.clamp_hi[k]; }
   LAUNCH(p, kSelect, launch_select_explore(a, p->stream));
-  if (!(s.flags & PBT_COPY_WEIGHTS) || n_cut == 0) return PBT_OK;
+  if (!(s.flags & PBT_COPY_WEIGHTS) || p->N < 2 || (s.exploit_rule == 0 && n_cut == 0)) return PBT_OK;
+  // Truncation: donors are never recipients, one parallel copy pass.  Tournament: a donor may be a recipient
+  // too; recipients are copied in passes (deepest readers first) so that every copy reads the donor's record
+  // as it was before this ready point.  The number of passes is read back from the device.
+  int passes = 1;
+  if (s.exploit_rule == 1) {
+    Counters cnt;
+    CU(p, cudaMemcpyAsync(&cnt, p->counters, sizeof(cnt), cudaMemcpyDeviceToHost, p->stream));
+    CU(p, cudaStreamSynchronize(p->stream));
+    passes = cnt.max_level + 1;
+  }
   CopyArgs c;
   memset(&c, 0, sizeof(c));
   c.n = p->N; c.src = p->src;
+  c.level = s.exploit_rule == 1 ? p->level : nullptr;
   auto add = [&](void* base, long long stride, long long bytes) {
     if (!base) return;
     c.base[c.n_arrays] = (char*)base; c.stride_bytes[c.n_arrays] = stride; c.copy_bytes[c.n_arrays] = bytes;
     c.n_arrays++;
   };
-  if (p->toy) {
-    // nh doubles per member: tiny, and not a multiple of 16 bytes in general -> dedicated path below
-    LAUNCH(p, kCopy, launch_copy_small((char*)p->theta, (long long)p->nh * 8, p->src, p->N, p->stream));
-    return PBT_OK;
+  if (!p->toy) {
+    const long long slab = p->P_pad * 4;
+    add(p->W32, slab, slab);
+    add(p->O1, slab, slab);
+    add(p->O2, slab, slab);
+    add(p->W16, p->P_pad * 2, p->P_pad * 2);
+    add(p->scalars, PBT_N_SCALARS * 4, PBT_N_SCALARS * 4);
   }
-  const long long slab = p->P_pad * 4;
-  add(p->W32, slab, slab);
-  add(p->O1, slab, slab);
-  add(p->O2, slab, slab);
-  add(p->W16, p->P_pad * 2, p->P_pad * 2);
-  add(p->scalars, PBT_N_SCALARS * 4, PBT_N_SCALARS * 4);
-  LAUNCH(p, kCopy, launch_slab_copy(c, p->stream));
+  for (int pass = 0; pass < passes; ++pass) {
+    c.want_level = pass;
+    if (p->toy) {
+      // nh doubles per member: tiny, and not a multiple of 16 bytes in general
+      LAUNCH(p, kCopy, launch_copy_small((char*)p->theta, (long long)p->nh * 8, p->src, p->N, c.level, pass, p->stream));
+    } else {
+      LAUNCH(p, kCopy, launch_slab_copy(c, p->stream));
+    }
+  }
   return PBT_OK;
 }
 

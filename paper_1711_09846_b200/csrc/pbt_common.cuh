@@ -52,7 +52,7 @@ struct Counters {
   int status;        // 0, or a pbt_status set by a kernel (bounded wait expired, ...)
   int status_info;   // where it was set
   int use_supplied_batch;  // next step trains on rows supplied by the caller
-  int pad;
+  int max_level;           // copy passes minus one needed by the last ready point (tournament chains)
 };
 
 // ---------------------------------------------------------------------------
@@ -150,6 +150,8 @@ struct SelectArgs {
   void* H;            // [n][PBT_MAX_NH] float or double
   void* fitness;      // [n] float or double
   int* src;           // [n]
+  int* level;         // [n] copy pass of each recipient (0 unless its donor chain is longer)
+  int rule;           // 0 truncation selection, 1 binary tournament
   Counters* counters;
   uint64_t seed;
   uint32_t perturb_mask, flags;
@@ -161,6 +163,8 @@ cudaError_t launch_select_explore(const SelectArgs& a, cudaStream_t s);
 struct CopyArgs {
   int n;
   const int* src;
+  const int* level;   // optional: only recipients with level[b] == want_level are copied in this launch
+  int want_level;
   // up to 5 member-major arrays copied donor -> recipient; bytes per member, stride in bytes
   int n_arrays;
   char* base[5];
@@ -168,7 +172,8 @@ struct CopyArgs {
   long long copy_bytes[5];  // multiples of 16
 };
 cudaError_t launch_slab_copy(const CopyArgs& a, cudaStream_t s);
-cudaError_t launch_copy_small(char* base, long long bytes, const int* src, int n, cudaStream_t s);
+cudaError_t launch_copy_small(char* base, long long bytes, const int* src, int n, const int* level, int want_level,
+                              cudaStream_t s);
 
 // misc kernels -------------------------------------------------------------
 cudaError_t launch_init_weights(float* w32, long long p_pad, int n_members, long long w_off, int fan_out,

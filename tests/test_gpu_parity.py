@@ -112,6 +112,55 @@ def test_select_copy_explore_bit_exact(pkg, n, dtype):
     gpu.close()
 
 
+@pytest.mark.parametrize("n", [1, 2, 3, 6, 16, 45, 80, 200])
+@pytest.mark.parametrize("dtype", [C.FP32, C.BF16])
+def test_binary_tournament_bit_exact(pkg, n, dtype):
+    """Section 4.3.1 (b): partners, decisions, copied records (donors that are recipients too are read before
+    they are overwritten), explored hyperparameters and fitness, against the oracle, bit for bit."""
+    cfg = _tiny_cfg(n, dtype).replace(exploit="tournament")
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    rng = np.random.default_rng(100 + n)
+    gpu.step(1)
+    cpu.step(1)
+    push_oracle_state(gpu, cpu)
+    chains = 0
+    for rnd in range(5):
+        f = rng.standard_normal(n).astype(np.float32)
+        if rnd == 1:
+            f = np.round(f)                               # ties: nobody copies an equal
+        if rnd == 2 and n > 2:
+            f[rng.integers(0, n)] = np.nan
+        cpu.fitness[:] = f
+        gpu.set_fitness(f.astype(np.float64))
+        gpu.exploit_explore()
+        src = cpu.exploit_explore()
+        chains += sum(1 for i in range(n) if src[i] != i and src[src[i]] != src[i])
+        assert np.array_equal(gpu.copy_map(), src)
+        assert np.array_equal(gpu.hparams(), cpu.H.astype(np.float64))
+        assert np.array_equal(gpu.fitness(), cpu.fitness.astype(np.float64), equal_nan=True)
+        for m in range(n):
+            now, ref = gpu.get_state(m), cpu.get_flat(m)
+            assert now["round"] == cpu.round
+            for key in ("w", "opt1", "opt2", "scalars"):
+                assert np.array_equal(now[key], ref[key]), (rnd, m, key)
+    if n >= 16:
+        assert chains > 0                                 # the multi-pass copy was exercised
+    gpu.close()
+
+
+def test_toy_with_tournament_matches_oracle(pkg):
+    cfg = get_config("c1").replace(exploit="tournament", n_members=2)
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    gpu.run(40)
+    cpu.run(40)
+    for m in range(2):
+        assert np.array_equal(gpu.get_state(m)["w"], cpu.theta[m])
+    assert np.array_equal(gpu.hparams(), cpu.H)
+    gpu.close()
+
+
 @pytest.mark.parametrize("flags", [0, C.COPY_WEIGHTS, C.COPY_HPARAMS | C.EXPLORE, C.COPY_WEIGHTS | C.EXPLORE])
 def test_flag_variants_bit_exact(pkg, flags):
     cfg = _tiny_cfg(10, C.FP32, flags=flags, num=2, den=5)

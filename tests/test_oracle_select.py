@@ -148,3 +148,70 @@ def test_perturb_clamps_and_keeps_zero():
     out = O.perturb(h, [1, 1, 0], [True, True, True], 0.8, 1.2,
                     [-math.inf, -math.inf, 0.45], [0.999, math.inf, math.inf])
     assert out[0] == np.float32(0.999) and out[1] == 0.0 and out[2] == np.float32(0.45)
+
+
+# ---------------------------------------------------------------------------
+# binary tournament (Section 4.3.1 (b))
+# ---------------------------------------------------------------------------
+def test_tournament_brute_force_small_populations():
+    """Every fitness vector over {0,1,2}^N, N = 2..5: a member copies only a strictly better OTHER member,
+    the partner is the one the drawn word designates among the other N-1, and the best never copies."""
+    for n in range(2, 6):
+        for f in itertools.product((0.0, 1.0, 2.0), repeat=n):
+            for rnd in range(3):
+                src = O.tournament_select(f, seed=5, rnd=rnd)
+                for i in range(n):
+                    w = px.draw(5, i, rnd, px.STREAM_EXPLOIT, 1)[0]
+                    others = [j for j in range(n) if j != i]
+                    partner = others[min(int(w / 2**32 * (n - 1)), n - 2)]
+                    if f[partner] > f[i]:
+                        assert src[i] == partner
+                    else:
+                        assert src[i] == i
+                    if f[i] == max(f):
+                        assert src[i] == i
+
+
+def test_tournament_partner_is_uniform_over_the_others_and_uses_its_own_draw():
+    n = 7
+    f = list(range(n))                       # member 0 is the worst: it copies whoever it draws
+    seen = collections_counter = {}
+    for rnd in range(700):
+        s0 = int(O.tournament_select(f, seed=9, rnd=rnd)[0])
+        seen[s0] = seen.get(s0, 0) + 1
+    assert set(seen) == set(range(1, n))
+    assert max(seen.values()) - min(seen.values()) < 70          # ~117 each
+    # the tournament draw is not the truncation draw (different counter block)
+    a = [px.draw(9, 0, r, px.STREAM_EXPLOIT, 0)[0] for r in range(4)]
+    b = [px.draw(9, 0, r, px.STREAM_EXPLOIT, 1)[0] for r in range(4)]
+    assert a != b
+    # NaN is the worst score; a NaN member copies any real partner, nobody copies a NaN member
+    src = O.tournament_select([float("nan"), 1.0, 2.0], seed=1, rnd=0)
+    assert src[0] in (1, 2) and all(src[i] != 0 for i in (1, 2))
+
+
+def test_tournament_copies_read_the_state_before_the_ready_point():
+    """i <- j while j <- k: i must receive j's OLD record.  Searched over rounds until a chain occurs."""
+    from workloads import get_config, make_inputs
+    cfg = get_config("c2_mini").replace(n_members=6, exploit="tournament")
+    inp = make_inputs(cfg)
+    found = False
+    for rnd in range(40):
+        p = O.Population(cfg, inp)
+        p.round = rnd
+        p.fitness[:] = np.arange(6, dtype=np.float32)
+        for m in range(6):
+            p.W[m][0][:] = float(m)                      # tag every member's weights with its index
+        before_H = p.H.copy()
+        src = p.exploit_explore()
+        chain = [i for i in range(6) if src[i] != i and src[src[i]] != src[i]]
+        for i in range(6):
+            assert np.all(p.W[i][0] == float(src[i]))    # the donor's pre-copy weights, even when the donor copied too
+            assert p.fitness[i] == float(src[i])
+            if src[i] != i:
+                for k in range(cfg.nh):
+                    lo, hi = np.float32(cfg.clamp_lo[k]), np.float32(cfg.clamp_hi[k])
+                    cands = {min(max(np.float32(before_H[src[i], k] * np.float32(fc)), lo), hi) for fc in (0.8, 1.2)}
+                    assert p.H[i, k] in cands
+        found = found or bool(chain)
+    assert found

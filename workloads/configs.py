@@ -77,6 +77,7 @@ class PBTConfig:
     factor_lo: float = 0.8
     factor_hi: float = 1.2
     flags: int = COPY_WEIGHTS | COPY_HPARAMS | EXPLORE
+    exploit: str = "truncation"   # or "tournament" (Section 4.3.1 (b))
     ready_interval: int = 1
     total_steps: int = 0
     seed: int = 0
