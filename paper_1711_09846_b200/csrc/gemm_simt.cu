@@ -20,8 +20,9 @@ __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloat162float(v)
 
 template <typename T, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(256) k_gemm_simt(GemmArgs g) {
-  __shared__ float As[BK][BM + 4];
-  __shared__ float Bs[BK][BN + 4];
+  // double-buffered k-slabs: the global loads of slab k+1 are in flight (in registers) while slab k is multiplied
+  __shared__ float As[2][BK][BM + 4];
+  __shared__ float Bs[2][BK][BN + 4];
   const int member = blockIdx.z;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const T* __restrict__ A = reinterpret_cast<const T*>(g.A) + member * g.strideA;
@@ -33,33 +34,51 @@ __global__ void __launch_bounds__(256) k_gemm_simt(GemmArgs g) {
   for (int i = 0; i < TM; ++i)
 #pragma unroll
     for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
+  constexpr int kPerThread = (BM * BK) / 256;
+  float ra[kPerThread], rb[kPerThread];
 
-  for (int k0 = 0; k0 < g.K; k0 += BK) {
+  auto load_slab = [&](int k0) {
 #pragma unroll
-    for (int i = 0; i < (BM * BK) / 256; ++i) {
+    for (int i = 0; i < kPerThread; ++i) {
       const int idx = tid + i * 256;
       int mm, kk;
       if (A_MN) { mm = idx % BM; kk = idx / BM; } else { kk = idx % BK; mm = idx / BK; }
-      const int gm = m0 + mm, gk = k0 + kk;
-      float v = 0.f;
-      if (gm < g.M && gk < g.K) v = to_f<T>(A_MN ? A[(long long)gk * g.lda + gm] : A[(long long)gm * g.lda + gk]);
-      As[kk][mm] = v;
-    }
-#pragma unroll
-    for (int i = 0; i < (BN * BK) / 256; ++i) {
-      const int idx = tid + i * 256;
-      int nn, kk;
+      const int gm = m0 + mm;
+      int gk = k0 + kk;
+      ra[i] = (gm < g.M && gk < g.K) ? to_f<T>(A_MN ? A[(long long)gk * g.lda + gm] : A[(long long)gm * g.lda + gk]) : 0.f;
+      int nn;
       if (B_MN) { nn = idx % BN; kk = idx / BN; } else { kk = idx % BK; nn = idx / BK; }
-      const int gn = n0 + nn, gk = k0 + kk;
-      float v = 0.f;
-      if (gn < g.N && gk < g.K) v = to_f<T>(B_MN ? B[(long long)gk * g.ldb + gn] : B[(long long)gn * g.ldb + gk]);
-      Bs[kk][nn] = v;
+      const int gn = n0 + nn;
+      gk = k0 + kk;
+      rb[i] = (gn < g.N && gk < g.K) ? to_f<T>(B_MN ? B[(long long)gk * g.ldb + gn] : B[(long long)gn * g.ldb + gk]) : 0.f;
     }
-    __syncthreads();
+  };
+  auto store_slab = [&](int buf) {
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) {
+      const int idx = tid + i * 256;
+      int mm, kk;
+      if (A_MN) { mm = idx % BM; kk = idx / BM; } else { kk = idx % BK; mm = idx / BK; }
+      As[buf][kk][mm] = ra[i];
+      int nn;
+      if (B_MN) { nn = idx % BN; kk = idx / BN; } else { kk = idx % BK; nn = idx / BK; }
+      Bs[buf][kk][nn] = rb[i];
+    }
+  };
+
+  if (g.K > 0) {
+    load_slab(0);
+    store_slab(0);
+  }
+  __syncthreads();
+  int buf = 0;
+  for (int k0 = 0; k0 < g.K; k0 += BK, buf ^= 1) {
+    const bool more = k0 + BK < g.K;
+    if (more) load_slab(k0 + BK);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
-      const float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * TM]);
-      const float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][tx * TN]);
+      const float4 a4 = *reinterpret_cast<const float4*>(&As[buf][kk][ty * TM]);
+      const float4 b4 = *reinterpret_cast<const float4*>(&Bs[buf][kk][tx * TN]);
       const float a[TM] = {a4.x, a4.y, a4.z, a4.w};
       const float b[TN] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
@@ -67,6 +86,7 @@ __global__ void __launch_bounds__(256) k_gemm_simt(GemmArgs g) {
 #pragma unroll
         for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
     }
+    if (more) store_slab(buf ^ 1);
     __syncthreads();
   }
 
