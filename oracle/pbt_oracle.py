@@ -21,6 +21,9 @@ What it follows
 * `explore`: perturb (Section 4.1.1 (a)): every hyperparameter of a member
   that copied is multiplied by 0.8 or 1.2 independently (0.5 / 2.0 in Section
   4.3.1 are the same operator with other factors).
+* The other operators the paper lists: binary tournament (Section 4.3.1 (b)),
+  t-test selection on the last 10 scores (Section 4.1.1, exploit (a)), and
+  resampling from the prior (Section 4.1.1, explore (b)).
 * The guard of Algorithm 1 (explore and re-evaluate only when the weights
   changed) and the population update.
 
@@ -38,7 +41,10 @@ Pins (tests/test_oracle_*.py): toy closed form and the paper's printed Q ~ 0.4
 N = 2..5; donor uniformity; copy / explore / lineage invariants; member
 isolation with exploit off; finite-difference gradients; least-squares special
 case; hand-computed optimiser trajectories; energy-distance special cases;
-Philox known-answer vectors.  `Population.run` over a whole neural-network
+Philox known-answer vectors; Welch's test against printed critical values, the
+closed-form t distributions with 1 and 2 degrees of freedom and an independent
+library routine; resampling against the prior's range, rate and quantiles.
+`Population.run` over a whole neural-network
 config has no external truth to compare with: parity unpinned beyond the pins
 of its parts.
 """
@@ -137,6 +143,73 @@ def tournament_select(fitness, seed: int, rnd: int) -> np.ndarray:
     return src
 
 
+HISTORY = 10  # evaluations kept per member for the t-test (Section 4.1.1, exploit (a): the last 10 scores)
+
+
+def welch_t_test(a, b):
+    """Welch's unequal-variance t-test of sample b against sample a.  Returns (t, df, p): the statistic
+    (mean_b - mean_a) / sqrt(s_a^2/n_a + s_b^2/n_b) with unbiased variances, the Welch-Satterthwaite degrees
+    of freedom, and the two-sided p-value P(|T_df| >= |t|) = I_{df/(df+t^2)}(df/2, 1/2) (the regularised
+    incomplete beta function is the library primitive of this step)."""
+    from scipy.special import betainc
+    a = [float(x) for x in a]
+    b = [float(x) for x in b]
+    na, nb = len(a), len(b)
+    ma = sum(a) / na
+    mb = sum(b) / nb
+    va = sum((x - ma) ** 2 for x in a) / (na - 1)
+    vb = sum((x - mb) ** 2 for x in b) / (nb - 1)
+    qa, qb = va / na, vb / nb
+    se2 = qa + qb
+    t = (mb - ma) / math.sqrt(se2)
+    df = se2 * se2 / (qa * qa / (na - 1) + qb * qb / (nb - 1))
+    p = float(betainc(df / 2.0, 0.5, df / (df + t * t)))
+    return t, df, p
+
+
+def ttest_better(hist_self, hist_other, alpha: float) -> bool:
+    """Section 4.1.1, exploit (a): the other member replaces this one if its mean score over its recorded
+    evaluations is higher and Welch's t-test rejects equal means at level alpha (two-sided).  Readings: NaN
+    scores count as -inf; fewer than two recorded scores on either side -> no test, no copy; a member whose own
+    mean is -inf is replaced by any member with a larger mean; if both samples have zero variance the larger mean
+    wins outright (the statistic is unbounded); any other non-finite statistic -> no copy."""
+    clean = lambda h: [(-math.inf if math.isnan(float(x)) else float(x)) for x in h]
+    a, b = clean(hist_self), clean(hist_other)
+    if len(a) < 2 or len(b) < 2:
+        return False
+    ma, mb = sum(a) / len(a), sum(b) / len(b)
+    if not (mb > ma):
+        return False
+    if ma == -math.inf:
+        return True
+    if not math.isfinite(mb):
+        return False
+    va = sum((x - ma) ** 2 for x in a) / (len(a) - 1)
+    vb = sum((x - mb) ** 2 for x in b) / (len(b) - 1)
+    if va / len(a) + vb / len(b) == 0.0:
+        return True
+    _, _, p = welch_t_test(a, b)
+    return bool(p < alpha)
+
+
+def ttest_select(histories, seed: int, rnd: int, alpha: float) -> np.ndarray:
+    """T-test selection (Section 4.1.1, exploit (a)): every member draws one OTHER member uniformly and copies it
+    if `ttest_better` holds for the two score histories (oldest first, at most HISTORY entries each).
+    src[i] == i where nothing is copied.  All decisions use the histories as they stand before any copy."""
+    n = len(histories)
+    src = np.arange(n, dtype=np.int32)
+    if n < 2:
+        return src
+    for i in range(n):
+        word = px.draw(seed, i, rnd, px.STREAM_EXPLOIT, 2)[0]
+        j = donor_index(word, n - 1)
+        if j >= i:
+            j += 1
+        if ttest_better(histories[i], histories[j], alpha):
+            src[i] = j
+    return src
+
+
 def explore_bits(seed: int, member: int, rnd: int, nh: int) -> List[int]:
     """One bit per hyperparameter slot: 1 -> multiply by the high factor, 0 -> low."""
     bits = []
@@ -156,6 +229,40 @@ def perturb(h_row: np.ndarray, bits, mask, factor_lo, factor_hi, lo, hi) -> np.n
             continue
         f = dt(factor_hi) if bits[k] else dt(factor_lo)
         v = dt(out[k] * f)
+        v = max(v, dt(lo[k]))
+        v = min(v, dt(hi[k]))
+        out[k] = v
+    return out
+
+
+def resample_threshold(q: float) -> int:
+    """Probability q as a 32-bit threshold: a slot is resampled when its Philox word is below it."""
+    return min(max(int(q * 4294967296.0), 0), 0xFFFFFFFF)
+
+
+def resample(h_row: np.ndarray, seed: int, member: int, rnd: int, mask, priors, q: float, lo, hi) -> np.ndarray:
+    """Section 4.1.1, explore (b): each hyperparameter of a member that copied is, with probability q, drawn
+    afresh from its prior; otherwise the copied value is kept.  Slot k uses Philox block 16 + k of the explore
+    stream: word 0 decides (word < q * 2^32), word 1 gives u = (word + 1/2) / 2^32, and the value is
+    lo + u (hi - lo) for a uniform prior, exp(log lo + u (log hi - log lo)) for a log-uniform one -- computed in
+    float64, rounded once to h's dtype, then clamped like a perturbed value."""
+    dt = h_row.dtype.type
+    out = h_row.copy()
+    thr = resample_threshold(q)
+    for k in range(len(out)):
+        kind, plo, phi = priors[k]
+        if not mask[k] or kind == "fixed":
+            continue
+        words = px.draw(seed, member, rnd, px.STREAM_EXPLORE, 16 + k)
+        if not (words[0] < thr):
+            continue
+        u = (float(words[1]) + 0.5) / 4294967296.0
+        if kind == "logu":
+            la, lb = math.log(plo), math.log(phi)
+            v = math.exp(la + u * (lb - la))
+        else:
+            v = plo + u * (phi - plo)
+        v = dt(v)
         v = max(v, dt(lo[k]))
         v = min(v, dt(hi[k]))
         out[k] = v
@@ -279,6 +386,7 @@ class Population:
         self.round = 0
         self.H = np.array(inputs.init_hparams, dtype=np.float64).astype(self.master)
         self.fitness = np.zeros(self.N, dtype=self.master)
+        self.history = [[] for _ in range(self.N)]   # scores of the last HISTORY evaluations, oldest first
         self.src = np.arange(self.N, dtype=np.int32)
         self.last_loss = np.zeros((self.N, 2), dtype=np.float64)
         self.scalars = np.ones((self.N, N_SCALARS), dtype=np.float32)
@@ -501,19 +609,24 @@ class Population:
         members = self.members if members is None else members
         for m in members:
             self.fitness[m] = self.master(self.eval_member(m))
+            self.history[m] = (self.history[m] + [self.fitness[m]])[-HISTORY:]
         return self.fitness.copy()
 
     # ----- exploit + explore at a ready point ---------------------------------
     def exploit_explore(self):
         cfg = self.cfg
-        if getattr(cfg, "exploit", "truncation") == "tournament":
+        rule = getattr(cfg, "exploit", "truncation")
+        if rule == "tournament":
             src = tournament_select(self.fitness, self.seed, self.round)
+        elif rule == "ttest":
+            src = ttest_select(self.history, self.seed, self.round, cfg.ttest_alpha)
         else:
             src = truncation_select(self.fitness, self.seed, self.round, cfg.trunc_num, cfg.trunc_den)
         copied = [b for b in range(self.N) if src[b] != b]
         # every copy reads the donor's record as it was BEFORE this ready point (under the tournament rule a
         # donor may itself be a recipient), so the donors are snapshotted first
         old_H, old_fit = self.H.copy(), self.fitness.copy()
+        old_hist = [list(h) for h in self.history]
         snap = {int(src[b]): self._snapshot_member(int(src[b])) for b in copied} if cfg.flags & COPY_WEIGHTS else {}
         for b in copied:
             d = int(src[b])
@@ -523,6 +636,10 @@ class Population:
                 self.H[b] = old_H[d]
         if cfg.flags & EXPLORE:
             for b in copied:
+                if getattr(cfg, "explore", "perturb") == "resample":
+                    self.H[b] = resample(self.H[b], self.seed, b, self.round, cfg.perturb, cfg.priors,
+                                         cfg.resample_prob, cfg.clamp_lo, cfg.clamp_hi)
+                    continue
                 bits = explore_bits(self.seed, b, self.round, cfg.nh)
                 self.H[b] = perturb(self.H[b], bits, cfg.perturb, cfg.factor_lo, cfg.factor_hi,
                                     cfg.clamp_lo, cfg.clamp_hi)
@@ -530,6 +647,8 @@ class Population:
             for b in copied:
                 # eval depends on the weights only, so the copy's performance is the donor's
                 self.fitness[b] = old_fit[int(src[b])]
+                # ... and so are the scores recorded for it (the t-test compares like with like)
+                self.history[b] = list(old_hist[int(src[b])])
         self.src = src
         self.round += 1
         return src

@@ -77,7 +77,10 @@ class PBTConfig:
     factor_lo: float = 0.8
     factor_hi: float = 1.2
     flags: int = COPY_WEIGHTS | COPY_HPARAMS | EXPLORE
-    exploit: str = "truncation"   # or "tournament" (Section 4.3.1 (b))
+    exploit: str = "truncation"   # or "tournament" (Section 4.3.1 (b)), "ttest" (Section 4.1.1, exploit (a))
+    ttest_alpha: float = 0.05     # significance level of the t-test (not stated in the paper)
+    explore: str = "perturb"      # or "resample" (Section 4.1.1, explore (b))
+    resample_prob: float = 0.25   # probability that a slot is redrawn from its prior (not stated in the paper)
     ready_interval: int = 1
     total_steps: int = 0
     seed: int = 0
@@ -182,6 +185,11 @@ CONFIGS: Dict[str, PBTConfig] = {
     "c3_mini_rms": _c3(n=6, widths=(72, 136, 200, 10), batch=40, eval_batch=96, pool=640, interval=3, steps=6,
                        name="c3_mini_rms").replace(optimizer=OPT_RMSPROP, slots=("lr",), priors=(("logu", 1e-5, 1e-3),),
                                                    perturb=(True,), clamp_lo=(-INF,), clamp_hi=(INF,), beta2=0.99),
+    # t-test selection and resample-from-prior on the same small shapes
+    "c2_mini_ttest": _c2(n=7, widths=(40, 72, 56, 1), batch=24, eval_batch=40, pool=512, interval=2, steps=12,
+                         name="c2_mini_ttest").replace(exploit="ttest"),
+    "c3_mini_resample": _c3(n=6, widths=(72, 136, 200, 10), batch=40, eval_batch=96, pool=640, interval=3, steps=9,
+                            name="c3_mini_resample").replace(explore="resample", resample_prob=0.5),
     # mid-size: every big layer is a multiple of the tensor-core tile so the
     # tcgen05 path is exercised, still seconds on a CPU
     "c3_mid": _c3(n=4, widths=(784, 1024, 1024, 10), batch=256, eval_batch=512, pool=2048,
