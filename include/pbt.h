@@ -37,6 +37,7 @@ extern "C" {
 
 #define PBT_MAX_LAYERS 8   /* weight layers per stack */
 #define PBT_MAX_NH 8       /* hyperparameter slots per member */
+#define PBT_HISTORY 10     /* scores kept per member for t-test selection (Section 4.1.1, exploit (a)) */
 #define PBT_N_SCALARS 4    /* Adam running beta products: c1,c2 of stack 0; c1,c2 of stack 1 */
 
 typedef enum pbt_status {
@@ -71,6 +72,9 @@ typedef enum pbt_optimizer {
   PBT_OPT_ADAM = 2,
   PBT_OPT_RMSPROP = 3 /* ms <- rho ms + (1-rho) g^2, theta <- theta - lr g / (sqrt(ms) + eps); rho = const_beta2; ms in opt1 */
 } pbt_optimizer;
+
+/* prior of a hyperparameter slot, used by the resample explore rule (Section 4.1.1, explore (b)) */
+typedef enum pbt_prior { PBT_PRIOR_FIXED = 0, PBT_PRIOR_UNIFORM = 1, PBT_PRIOR_LOG_UNIFORM = 2 } pbt_prior;
 
 /* exploit / explore switches ("PBT targets" ablation, Section 4.4) */
 #define PBT_COPY_WEIGHTS 1u  /* exploit copies weights and optimiser state */
@@ -118,12 +122,22 @@ typedef struct pbt_spec {
                         layers never goes to HBM); 0: weight gradients are written once and one streaming pass over
                         the slabs applies the update.  Results are bit-identical; only the traffic pattern differs. */
   int32_t exploit_rule; /* 0: truncation selection (Section 4.1.1 (b)); 1: binary tournament (Section 4.3.1 (b)): every
-                           member draws one other member uniformly and copies it if its fitness is strictly higher */
+                           member draws one other member uniformly and copies it if its fitness is strictly higher;
+                           2: t-test selection (Section 4.1.1, exploit (a)): one other member drawn uniformly is
+                           copied if its mean over its last PBT_HISTORY scores is higher and Welch's t-test rejects
+                           equal means at level ttest_alpha (two-sided).  pbt_eval records the scores. */
+  int32_t explore_rule; /* 0: perturb (Section 4.1.1, explore (a)); 1: resample (Section 4.1.1, explore (b)): each
+                           slot of perturb_mask whose prior is not PBT_PRIOR_FIXED is redrawn from its prior with
+                           probability resample_prob, else the copied value is kept; clamped either way */
+  int32_t prior_kind[PBT_MAX_NH]; /* pbt_prior of each slot (resample only) */
   double const_lr, const_momentum, const_beta1, const_beta2, const_eps, const_wd;
   double toy_eta;                 /* toy step size */
   double toy_theta0[PBT_MAX_NH];  /* toy initial theta (same for all members) */
   double factor_lo, factor_hi;    /* perturbation factors, 0.8 / 1.2 */
   double clamp_lo[PBT_MAX_NH], clamp_hi[PBT_MAX_NH]; /* applied after perturbation; +-inf = none */
+  double ttest_alpha;    /* significance level of the t-test (the paper states none; 0.05 is customary) */
+  double resample_prob;  /* probability that explore redraws a slot (the paper states none) */
+  double prior_lo[PBT_MAX_NH], prior_hi[PBT_MAX_NH]; /* range of each slot's prior; log-uniform needs 0 < lo <= hi */
 } pbt_spec;
 
 /*
@@ -207,11 +221,12 @@ int pbt_eval(pbt_t* p);
 
 /*
  * One ready point for the whole population (Algorithm 1: exploit, the
- * theta != theta' guard, explore, population update): truncation selection on
- * the current fitness vector (Section 4.1.1 (b)), slab copy donor -> recipient of
- * weights, optimiser state and (flag) hyperparameters, perturbation of the
- * recipients' h by factor_lo / factor_hi (Section 4.1.1 (a)), p[b] <- p[src[b]],
- * round <- round + 1.
+ * theta != theta' guard, explore, population update): selection by
+ * exploit_rule on the current fitness vector (or score histories), slab copy
+ * donor -> recipient of weights, optimiser state and (flag) hyperparameters,
+ * explore_rule applied to the recipients' h, p[b] <- p[src[b]] (and the score
+ * history with it), round <- round + 1.  Every copy reads the donor's record
+ * as it was before this ready point.
  */
 int pbt_exploit_explore(pbt_t* p);
 
@@ -223,6 +238,16 @@ int pbt_set_state(pbt_t* p, int member, const pbt_state_view* in_host);
  * fitness vector so that selection can be compared bit for bit. */
 int pbt_get_fitness(pbt_t* p, double* out_host);
 int pbt_set_fitness(pbt_t* p, const double* in_host);
+
+/*
+ * Score history used by t-test selection (Section 4.1.1, exploit (a)): hist[n_members][PBT_HISTORY] doubles, oldest
+ * first, the first count[m] entries of row m valid (the rest read as 0); count[n_members] int32.  Both host.
+ * pbt_eval appends to it when exploit_rule == 2 (dropping the oldest of PBT_HISTORY); a copy at a ready point
+ * moves the donor's history with its weights.  set lets a test inject histories so that the decisions can be
+ * compared bit for bit; counts outside [0, PBT_HISTORY] are PBT_ERR_INVALID_ARG.  Either pointer may be NULL in get.
+ */
+int pbt_get_history(pbt_t* p, double* hist_out_host, int32_t* count_out_host);
+int pbt_set_history(pbt_t* p, const double* hist_in_host, const int32_t* count_in_host);
 
 /* h[n_members][nh] as doubles (host). */
 int pbt_get_hparams(pbt_t* p, double* out_host);

@@ -17,6 +17,7 @@ import numpy as np
 PBT_MAX_LAYERS = 8
 PBT_MAX_NH = 8
 PBT_N_SCALARS = 4
+PBT_HISTORY = 10
 
 _DTYPE = {"fp64_toy": 0, "fp32": 1, "bf16_fp32master": 2}
 _MODEL = {"toy_quadratic": 0, "mlp": 1, "gan_pair": 2}
@@ -38,11 +39,14 @@ class PbtSpec(C.Structure):
         ("slot_beta1", C.c_int32), ("slot_wd", C.c_int32),
         ("perturb_mask", C.c_uint32), ("flags", C.c_uint32),
         ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("exploit_rule", C.c_int32),
+        ("explore_rule", C.c_int32), ("prior_kind", C.c_int32 * PBT_MAX_NH),
         ("const_lr", C.c_double), ("const_momentum", C.c_double), ("const_beta1", C.c_double),
         ("const_beta2", C.c_double), ("const_eps", C.c_double), ("const_wd", C.c_double),
         ("toy_eta", C.c_double), ("toy_theta0", C.c_double * PBT_MAX_NH),
         ("factor_lo", C.c_double), ("factor_hi", C.c_double),
         ("clamp_lo", C.c_double * PBT_MAX_NH), ("clamp_hi", C.c_double * PBT_MAX_NH),
+        ("ttest_alpha", C.c_double), ("resample_prob", C.c_double),
+        ("prior_lo", C.c_double * PBT_MAX_NH), ("prior_hi", C.c_double * PBT_MAX_NH),
     ]
 
 
@@ -73,6 +77,7 @@ class PbtGemmDesc(C.Structure):
 EXPORTS = [
     "pbt_query_workspace", "pbt_param_count", "pbt_create", "pbt_destroy", "pbt_step", "pbt_eval",
     "pbt_exploit_explore", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
+    "pbt_get_history", "pbt_set_history",
     "pbt_get_hparams", "pbt_set_hparams", "pbt_get_copy_map", "pbt_get_best", "pbt_get_last_loss",
     "pbt_set_batch", "pbt_step_host", "pbt_prefetch_host_batch", "pbt_step_prefetched", "pbt_get_launch_count", "pbt_profile_begin", "pbt_profile_end", "pbt_profile_get",
     "pbt_grouped_gemm", "pbt_energy_fitness_static", "pbt_last_error",
@@ -166,7 +171,13 @@ def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True) -> Pb
     s.flags = cfg.flags
     s.trunc_num, s.trunc_den = cfg.trunc_num, cfg.trunc_den
     s.keep_grad = 1 if keep_grad else 0
-    s.exploit_rule = {"truncation": 0, "tournament": 1}[getattr(cfg, "exploit", "truncation")]
+    s.exploit_rule = {"truncation": 0, "tournament": 1, "ttest": 2}[getattr(cfg, "exploit", "truncation")]
+    s.explore_rule = {"perturb": 0, "resample": 1}[getattr(cfg, "explore", "perturb")]
+    s.ttest_alpha = getattr(cfg, "ttest_alpha", 0.05)
+    s.resample_prob = getattr(cfg, "resample_prob", 0.25)
+    for k, (kind, lo, hi) in enumerate(cfg.priors[:cfg.nh]):
+        s.prior_kind[k] = {"fixed": 0, "u": 1, "logu": 2}[kind]
+        s.prior_lo[k], s.prior_hi[k] = lo, hi
     s.fuse_adam = 1 if fuse_adam else 0
     s.const_lr = 0.0
     s.const_momentum = cfg.momentum
@@ -383,6 +394,21 @@ class Population:
         f = np.zeros(self.N, dtype=np.float64)
         self._check(self.lib.pbt_get_fitness(self.handle, f.ctypes.data_as(C.POINTER(C.c_double))))
         return f
+
+    def history(self):
+        """(scores [N][PBT_HISTORY] oldest first, counts [N]) used by t-test selection."""
+        h = np.zeros((self.N, PBT_HISTORY), dtype=np.float64)
+        c = np.zeros(self.N, dtype=np.int32)
+        self._check(self.lib.pbt_get_history(self.handle, h.ctypes.data_as(C.POINTER(C.c_double)),
+                                             c.ctypes.data_as(C.POINTER(C.c_int32))))
+        return h, c
+
+    def set_history(self, h, c):
+        h = np.ascontiguousarray(h, dtype=np.float64)
+        c = np.ascontiguousarray(c, dtype=np.int32)
+        assert h.shape == (self.N, PBT_HISTORY) and c.shape == (self.N,)
+        self._check(self.lib.pbt_set_history(self.handle, h.ctypes.data_as(C.POINTER(C.c_double)),
+                                             c.ctypes.data_as(C.POINTER(C.c_int32))))
 
     def set_fitness(self, f):
         f = np.ascontiguousarray(f, dtype=np.float64)

@@ -59,6 +59,8 @@ struct pbt_handle {
   void* fitness;  // [N] float (double for the toy)
   int* src;
   int* level;        // [N] copy pass of each recipient at the last ready point
+  void* hist;        // [N][PBT_HISTORY] scores for t-test selection, same type as fitness
+  int* hist_n;       // [N]
   Counters* counters;
   float* last_loss;  // [N][2]
   double* theta;     // toy: [N][nh]
@@ -125,7 +127,19 @@ int validate(const pbt_spec* s) {
   if (s->n_members < 1 || s->n_members > 1024) return fail(nullptr, PBT_ERR_INVALID_ARG, "n_members must be in [1, 1024]");
   if (s->nh < 0 || s->nh > PBT_MAX_NH) return fail(nullptr, PBT_ERR_INVALID_ARG, "nh must be in [0, %d]", PBT_MAX_NH);
   if (s->trunc_num < 0 || s->trunc_den < 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "bad truncation fraction");
-  if (s->exploit_rule != 0 && s->exploit_rule != 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "unknown exploit rule");
+  if (s->exploit_rule < 0 || s->exploit_rule > 2) return fail(nullptr, PBT_ERR_INVALID_ARG, "unknown exploit rule");
+  if (s->explore_rule != 0 && s->explore_rule != 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "unknown explore rule");
+  if (s->exploit_rule == 2 && !(s->ttest_alpha > 0.0 && s->ttest_alpha < 1.0))
+    return fail(nullptr, PBT_ERR_INVALID_ARG, "ttest_alpha must lie in (0, 1)");
+  if (s->explore_rule == 1) {
+    if (!(s->resample_prob >= 0.0 && s->resample_prob <= 1.0)) return fail(nullptr, PBT_ERR_INVALID_ARG, "resample_prob must lie in [0, 1]");
+    for (int k = 0; k < s->nh; ++k) {
+      const int kind = s->prior_kind[k];
+      if (kind < PBT_PRIOR_FIXED || kind > PBT_PRIOR_LOG_UNIFORM) return fail(nullptr, PBT_ERR_INVALID_ARG, "unknown prior kind");
+      if (kind != PBT_PRIOR_FIXED && !(s->prior_lo[k] <= s->prior_hi[k])) return fail(nullptr, PBT_ERR_INVALID_ARG, "prior range is empty");
+      if (kind == PBT_PRIOR_LOG_UNIFORM && !(s->prior_lo[k] > 0.0)) return fail(nullptr, PBT_ERR_INVALID_ARG, "log-uniform prior needs lo > 0");
+    }
+  }
   const int slots[5] = {s->slot_lr, s->slot_lr_d, s->slot_momentum, s->slot_beta1, s->slot_wd};
   for (int i = 0; i < 5; ++i)
     if (slots[i] < -1 || slots[i] >= s->nh) return fail(nullptr, PBT_ERR_INVALID_ARG, "hyperparameter slot out of range");
@@ -185,6 +199,8 @@ size_t plan(pbt_handle* h, char* base) {
   h->level = (int*)take(N * sizeof(int));
   h->H = take(N * PBT_MAX_NH * sizeof(double));
   h->fitness = take(N * sizeof(double));
+  h->hist = take(N * PBT_HISTORY * sizeof(double));
+  h->hist_n = (int*)take(N * sizeof(int));
   h->last_loss = (float*)take(N * 2 * sizeof(float));
   h->scalars = (float*)take(N * PBT_N_SCALARS * sizeof(float));
   if (h->toy) {
@@ -741,13 +757,20 @@ int pbt_step(pbt_t* p, int k) {
   return PBT_OK;
 }
 
+// t-test selection compares the last PBT_HISTORY scores of two members: every evaluation is appended
+static int record_scores(pbt_t* p) {
+  if (p->spec.exploit_rule != 2) return PBT_OK;
+  LAUNCH(p, kOther, launch_history_push(p->fitness, p->hist, p->hist_n, p->N, p->toy ? 1 : 0, p->stream));
+  return PBT_OK;
+}
+
 int pbt_eval(pbt_t* p) {
   if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
   p->launches = 0;
   const pbt_spec& s = p->spec;
   if (p->toy) {
     LAUNCH(p, kLoss, launch_toy_eval(p->theta, (double*)p->fitness, p->N, p->nh, p->stream));
-    return PBT_OK;
+    return record_scores(p);
   }
   int rc = forward(p, 0, s.eval_batch, p->data.x_eval, 0);
   if (rc) return rc;
@@ -755,7 +778,7 @@ int pbt_eval(pbt_t* p) {
     LAUNCH(p, kLoss, launch_energy_distance(p->logits[0], logits_stride(p, 0), s.eval_batch, p->N, p->ed_partial,
                                             (float*)p->fitness, p->stream));
     p->launches++;  // the launcher issues two kernels
-    return PBT_OK;
+    return record_scores(p);
   }
   LossArgs a;
   memset(&a, 0, sizeof(a));
@@ -768,7 +791,7 @@ int pbt_eval(pbt_t* p) {
   a.dz = nullptr; a.row_loss = p->row_loss;
   LAUNCH(p, kLoss, launch_loss_rows(a, p->stream));
   LAUNCH(p, kLoss, launch_reduce_rows(p->row_loss, s.eval_batch, p->N, -1.0f / (float)s.eval_batch, p->fitness, 0, 1, p->stream));
-  return PBT_OK;
+  return record_scores(p);
 }
 
 int pbt_exploit_explore(pbt_t* p) {
@@ -789,16 +812,28 @@ int pbt_exploit_explore(pbt_t* p) {
   a.h_is_double = p->toy ? 1 : 0;
   a.H = p->H; a.fitness = p->fitness; a.src = p->src; a.level = p->level; a.counters = p->counters; a.seed = p->seed;
   a.rule = s.exploit_rule;
+  a.hist = p->hist; a.hist_n = p->hist_n; a.alpha = s.ttest_alpha;
+  a.explore_rule = s.explore_rule;
+  if (s.explore_rule == 1) {
+    long long thr = (long long)(s.resample_prob * 4294967296.0);
+    a.resample_thr = (uint32_t)(thr < 0 ? 0 : (thr > 0xFFFFFFFFll ? 0xFFFFFFFFll : thr));
+    for (int k = 0; k < PBT_MAX_NH; ++k) {
+      a.prior_kind[k] = k < p->nh ? s.prior_kind[k] : PBT_PRIOR_FIXED;
+      const bool lg = a.prior_kind[k] == PBT_PRIOR_LOG_UNIFORM;
+      a.prior_a[k] = lg ? log(s.prior_lo[k]) : s.prior_lo[k];
+      a.prior_b[k] = lg ? log(s.prior_hi[k]) : s.prior_hi[k];
+    }
+  }
   a.perturb_mask = s.perturb_mask; a.flags = s.flags;
   a.factor_lo = s.factor_lo; a.factor_hi = s.factor_hi;
   for (int k = 0; k < PBT_MAX_NH; ++k) { a.clamp_lo[k] = s.clamp_lo[k]; a.clamp_hi[k] = s.clamp_hi[k]; }
   LAUNCH(p, kSelect, launch_select_explore(a, p->stream));
   if (!(s.flags & PBT_COPY_WEIGHTS) || p->N < 2 || (s.exploit_rule == 0 && n_cut == 0)) return PBT_OK;
-  // Truncation: donors are never recipients, one parallel copy pass.  Tournament: a donor may be a recipient
+  // Truncation: donors are never recipients, one parallel copy pass.  Tournament, t-test: a donor may be a recipient
   // too; recipients are copied in passes (deepest readers first) so that every copy reads the donor's record
   // as it was before this ready point.  The number of passes is read back from the device.
   int passes = 1;
-  if (s.exploit_rule == 1) {
+  if (s.exploit_rule != 0) {
     Counters cnt;
     CU(p, cudaMemcpyAsync(&cnt, p->counters, sizeof(cnt), cudaMemcpyDeviceToHost, p->stream));
     CU(p, cudaStreamSynchronize(p->stream));
@@ -807,7 +842,7 @@ int pbt_exploit_explore(pbt_t* p) {
   CopyArgs c;
   memset(&c, 0, sizeof(c));
   c.n = p->N; c.src = p->src;
-  c.level = s.exploit_rule == 1 ? p->level : nullptr;
+  c.level = s.exploit_rule != 0 ? p->level : nullptr;
   auto add = [&](void* base, long long stride, long long bytes) {
     if (!base) return;
     c.base[c.n_arrays] = (char*)base; c.stride_bytes[c.n_arrays] = stride; c.copy_bytes[c.n_arrays] = bytes;
@@ -961,6 +996,41 @@ int pbt_set_fitness(pbt_t* p, const double* in) {
     CU(p, cudaMemcpyAsync(p->fitness, f.data(), (size_t)p->N * 4, cudaMemcpyHostToDevice, p->stream));
     CU(p, cudaStreamSynchronize(p->stream));
   }
+  return PBT_OK;
+}
+
+int pbt_get_history(pbt_t* p, double* hist, int32_t* count) {
+  if (!p) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  const size_t n = (size_t)p->N * PBT_HISTORY;
+  std::vector<int32_t> c(p->N);
+  CU(p, cudaMemcpyAsync(c.data(), p->hist_n, (size_t)p->N * 4, cudaMemcpyDeviceToHost, p->stream));
+  std::vector<double> hd(n);
+  std::vector<float> hf(n);
+  if (p->toy) CU(p, cudaMemcpyAsync(hd.data(), p->hist, n * 8, cudaMemcpyDeviceToHost, p->stream));
+  else CU(p, cudaMemcpyAsync(hf.data(), p->hist, n * 4, cudaMemcpyDeviceToHost, p->stream));
+  CU(p, cudaStreamSynchronize(p->stream));
+  for (int m = 0; m < p->N; ++m) {
+    if (count) count[m] = c[m];
+    if (hist)
+      for (int k = 0; k < PBT_HISTORY; ++k) {
+        const size_t i = (size_t)m * PBT_HISTORY + k;
+        hist[i] = k < c[m] ? (p->toy ? hd[i] : (double)hf[i]) : 0.0;
+      }
+  }
+  return PBT_OK;
+}
+
+int pbt_set_history(pbt_t* p, const double* hist, const int32_t* count) {
+  if (!p || !hist || !count) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  for (int m = 0; m < p->N; ++m)
+    if (count[m] < 0 || count[m] > PBT_HISTORY) return fail(p, PBT_ERR_INVALID_ARG, "history count out of range");
+  const size_t n = (size_t)p->N * PBT_HISTORY;
+  std::vector<float> hf(n);
+  for (size_t i = 0; i < n; ++i) hf[i] = (float)hist[i];
+  if (p->toy) CU(p, cudaMemcpyAsync(p->hist, hist, n * 8, cudaMemcpyHostToDevice, p->stream));
+  else CU(p, cudaMemcpyAsync(p->hist, hf.data(), n * 4, cudaMemcpyHostToDevice, p->stream));
+  CU(p, cudaMemcpyAsync(p->hist_n, count, (size_t)p->N * 4, cudaMemcpyHostToDevice, p->stream));
+  CU(p, cudaStreamSynchronize(p->stream));
   return PBT_OK;
 }
 

@@ -151,7 +151,14 @@ struct SelectArgs {
   void* fitness;      // [n] float or double
   int* src;           // [n]
   int* level;         // [n] copy pass of each recipient (0 unless its donor chain is longer)
-  int rule;           // 0 truncation selection, 1 binary tournament
+  int rule;           // 0 truncation selection, 1 binary tournament, 2 t-test selection
+  void* hist;         // [n][PBT_HISTORY] scores, oldest first (same type as fitness); t-test only
+  int* hist_n;        // [n] valid entries per row
+  double alpha;       // t-test significance level
+  int explore_rule;   // 0 perturb, 1 resample from the prior
+  uint32_t resample_thr;            // a slot is redrawn when its Philox word is below this
+  int prior_kind[PBT_MAX_NH];
+  double prior_a[PBT_MAX_NH], prior_b[PBT_MAX_NH];   // uniform: lo, hi; log-uniform: log lo, log hi
   Counters* counters;
   uint64_t seed;
   uint32_t perturb_mask, flags;
@@ -159,6 +166,8 @@ struct SelectArgs {
   double clamp_lo[PBT_MAX_NH], clamp_hi[PBT_MAX_NH];
 };
 cudaError_t launch_select_explore(const SelectArgs& a, cudaStream_t s);
+// append fitness[i] to row i of the score history (drop the oldest of PBT_HISTORY)
+cudaError_t launch_history_push(const void* fitness, void* hist, int* hist_n, int n, int is_double, cudaStream_t s);
 
 struct CopyArgs {
   int n;

@@ -10,7 +10,7 @@ from oracle import pbt_oracle as O
 from workloads import configs as C
 from workloads import get_config, make_inputs
 
-from util import TOL, assert_state_close, push_oracle_state, rel_err
+from util import TOL, assert_state_close, oracle_history_arrays, push_oracle_state, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -226,7 +226,7 @@ def _check_optimizer_arithmetic(cfg, s0, s1, h):
 # step / eval parity, step by step, re-seeding the GPU from the oracle at ready points
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("name", ["c2_mini", "c3_mini", "c4_mini", "c5_mini", "c3_mid", "c5_mid", "c4_mid", "c2_mini_rms",
-                                  "c3_mini_rms"])
+                                  "c3_mini_rms", "c2_mini_ttest", "c3_mini_resample"])
 def test_step_eval_exploit_parity(pkg, name):
     cfg = get_config(name)
     inp = make_inputs(cfg)
@@ -254,12 +254,20 @@ def test_step_eval_exploit_parity(pkg, name):
             gpu.eval()
             cpu.eval()
             np.testing.assert_allclose(gpu.fitness(), cpu.fitness, rtol=ftol, atol=2e-5)
-            # selection is compared on identical fitness vectors
+            # selection is compared on identical fitness vectors (and score histories)
             gpu.set_fitness(cpu.fitness.astype(np.float64))
+            if cfg.exploit == "ttest":
+                (gh, gc), (ch, cc) = gpu.history(), oracle_history_arrays(cpu)
+                assert np.array_equal(gc, cc)
+                np.testing.assert_allclose(gh[:, -1 if cc[0] == 10 else cc[0] - 1], cpu.fitness, rtol=ftol, atol=2e-5)
+                gpu.set_history(ch, cc)
             gpu.exploit_explore()
             src = cpu.exploit_explore()
             assert np.array_equal(gpu.copy_map(), src)
             assert np.array_equal(gpu.hparams(), cpu.H.astype(np.float64))
+            if cfg.exploit == "ttest":
+                (gh, gc), (ch, cc) = gpu.history(), oracle_history_arrays(cpu)
+                assert np.array_equal(gc, cc) and np.array_equal(gh, ch)
         # every step starts from identical state: training is chaotic, parity is per step
         push_oracle_state(gpu, cpu)
     gpu.close()

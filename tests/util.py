@@ -72,3 +72,13 @@ def push_oracle_state(gpu, cpu):
             gpu.set_state(m, w=f["w"], opt1=f["opt1"], opt2=f["opt2"], scalars=f["scalars"],
                           hparams=cpu.H[m].astype(np.float64), fitness=float(cpu.fitness[m]),
                           step=cpu.step_count, round=cpu.round)
+
+
+def oracle_history_arrays(cpu, depth=10):
+    """The oracle's score histories as the dense (scores [N][depth], counts [N]) pair of the interface."""
+    h = np.zeros((cpu.N, depth), dtype=np.float64)
+    c = np.zeros(cpu.N, dtype=np.int32)
+    for m in range(cpu.N):
+        c[m] = len(cpu.history[m])
+        h[m, :c[m]] = [float(x) for x in cpu.history[m]]
+    return h, c
