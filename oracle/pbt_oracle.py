@@ -545,6 +545,79 @@ class Population:
         gW, gb, _ = self.backward(m, 0, acts, self.q(dz))
         self._apply(m, 0, gW, gb, self._hp(m, "lr", 0.0))
 
+    def _interp_eps(self, m, j, B):
+        """Interpolation coefficient of row b in discriminator update j of this step: word b mod 4 of Philox
+        block j * 65536 + b div 4 of the interpolation stream; eps = ((word >> 9) + 1/2) / 2^23, which float32
+        holds exactly."""
+        eps = np.empty(B, dtype=np.float64)
+        for b in range(B):
+            w = px.draw(self.seed, m, self.step_count, px.STREAM_INTERP, j * 65536 + (b >> 2))[b & 3]
+            eps[b] = ((int(w) >> 9) + 0.5) / 8388608.0
+        return eps
+
+    def wgan_gp_critic(self, m, real, fake, eps, lam):
+        """The critic's WGAN-GP objective (Section 4.3.1) and its gradient for member m:
+            L_D = mean D(fake) - mean D(real) + lam * mean_b (||grad_x D(xhat_b)||_2 - 1)^2,
+            xhat_b = eps_b real_b + (1 - eps_b) fake_b.
+        The critic is a ReLU MLP, so its input gradient is a chain of matrix products gated by the activation
+        masks of the forward pass on xhat (u_L = 1; u_{l-1} = (u_l W_l) * [a_l > 0]; grad_x D = u_0 W_0), and the
+        penalty's gradient with respect to W_l follows by differentiating that chain (the masks are piecewise
+        constant): with r_b = (2 lam / B)(n_b - 1) / n_b * grad_x D(xhat_b), n_b the norm (r_b = 0 where n_b = 0),
+            dv_0 = r,  dv_{l+1} = (dv_l W_l^T) * [a_{l+1} > 0],  dL/dW_l += u_l^T dv_l.
+        Biases get no gradient from the penalty.  Operands of every product are rounded like all GEMM operands
+        (`self.q`); the input gradient itself is not rounded.  Returns (L_D, gW, gb, xhat)."""
+        B = real.shape[0]
+        ts = self._tensors_of_stack(1)
+        nl = len(ts)
+        xhat = self.q(eps[:, None] * real + (1.0 - eps[:, None]) * fake)
+        acts, d = self.forward(m, 1, np.concatenate([real, fake, xhat], axis=0))
+        d = d.reshape(-1)
+        W = [self.q(self.W[m][t]) for t in ts]
+        u = [None] * nl
+        u[nl - 1] = np.ones((B, 1), dtype=np.float64)
+        for l in range(nl - 1, 0, -1):
+            u[l - 1] = self.q((u[l] @ W[l]) * (acts[l][2 * B:] > 0.0))
+        gx = u[0] @ W[0]
+        nrm = np.sqrt((gx * gx).sum(axis=1))
+        pen = lam * np.mean((nrm - 1.0) ** 2)
+        loss = d[B:2 * B].mean() - d[:B].mean() + pen
+        scale = np.where(nrm > 0.0, (2.0 * lam / B) * (nrm - 1.0) / np.where(nrm > 0.0, nrm, 1.0), 0.0)
+        dv = [None] * nl
+        dv[0] = self.q(scale[:, None] * gx)
+        for l in range(nl - 1):
+            dv[l + 1] = self.q((dv[l] @ W[l].T) * (acts[l + 1][2 * B:] > 0.0))
+        dl = np.concatenate([np.full(B, -1.0 / B), np.full(B, 1.0 / B)]).reshape(-1, 1)
+        gW, gb, _ = self.backward(m, 1, [a[:2 * B] for a in acts], self.q(dl))
+        for l, t in enumerate(ts):
+            gW[t] = gW[t] + u[l].T @ dv[l]
+        return loss, gW, gb, xhat
+
+    def _step_wgan_gp(self, m):
+        """Section 4.3.1: K critic updates on the WGAN-GP objective, then one generator update on
+        L_G = -mean D(G(z))."""
+        cfg = self.cfg
+        B = cfg.batch
+        for j in range(cfg.gan_d_steps):
+            offr = self._window(m, j, 0, cfg.pool_rows, B)
+            offz = self._window(m, j, 1, cfg.pool_rows, B)
+            real = self.q(self.inp.x_pool[offr:offr + B])
+            zz = self.q(self.inp.z_pool[offz:offz + B])
+            _, gout = self.forward(m, 0, zz)
+            fake = self.q(gout)
+            loss, gW, gb, _ = self.wgan_gp_critic(m, real, fake, self._interp_eps(m, j, B), cfg.gp_lambda)
+            self.last_loss[m, 1] = loss
+            self._apply(m, 1, gW, gb, self._hp(m, "lr_d", 0.0))
+        offz = self._window(m, cfg.gan_d_steps, 1, cfg.pool_rows, B)
+        zz = self.q(self.inp.z_pool[offz:offz + B])
+        gacts, gout = self.forward(m, 0, zz)
+        fake = self.q(gout)
+        dacts, d = self.forward(m, 1, fake)
+        self.last_loss[m, 0] = -d.reshape(-1).mean()
+        dl = np.full((B, 1), -1.0 / B)
+        _, _, dfake = self.backward(m, 1, dacts, self.q(dl), need_wgrad=False, need_input_grad=True)
+        gW, gb, _ = self.backward(m, 0, gacts, dfake)
+        self._apply(m, 0, gW, gb, self._hp(m, "lr", 0.0))
+
     def _step_gan(self, m):
         """Section 4.3.1: K discriminator updates, then one generator update.
         Non-saturating logistic losses: L_D = mean softplus(-D(x)) + mean
@@ -584,6 +657,8 @@ class Population:
             for m in members:
                 if self.toy:
                     self._step_toy(m)
+                elif self.gan and self.cfg.loss == "wgan_gp":
+                    self._step_wgan_gp(m)
                 elif self.gan:
                     self._step_gan(m)
                 else:

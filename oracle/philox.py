@@ -30,6 +30,7 @@ STREAM_EXPLOIT = 0
 STREAM_EXPLORE = 1
 STREAM_BATCH = 2
 STREAM_INIT = 3
+STREAM_INTERP = 4  # interpolation coefficients of the gradient penalty
 
 
 def philox4x32_10(counter, key):

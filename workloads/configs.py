@@ -31,6 +31,7 @@ LOSS_MSE = "mse"
 LOSS_CE_HARD = "ce_hard"
 LOSS_CE_SOFT = "ce_soft"
 LOSS_GAN = "gan_logistic"
+LOSS_WGAN_GP = "wgan_gp"   # Section 4.3.1: Wasserstein critic with gradient penalty
 
 OPT_SGD = "sgd_plain"
 OPT_SGDM = "sgdm"
@@ -81,6 +82,7 @@ class PBTConfig:
     ttest_alpha: float = 0.05     # significance level of the t-test (not stated in the paper)
     explore: str = "perturb"      # or "resample" (Section 4.1.1, explore (b))
     resample_prob: float = 0.25   # probability that a slot is redrawn from its prior (not stated in the paper)
+    gp_lambda: float = 10.0       # weight of the gradient penalty (the value of the paper that introduced WGAN-GP)
     ready_interval: int = 1
     total_steps: int = 0
     seed: int = 0
@@ -185,6 +187,12 @@ CONFIGS: Dict[str, PBTConfig] = {
     "c3_mini_rms": _c3(n=6, widths=(72, 136, 200, 10), batch=40, eval_batch=96, pool=640, interval=3, steps=6,
                        name="c3_mini_rms").replace(optimizer=OPT_RMSPROP, slots=("lr",), priors=(("logu", 1e-5, 1e-3),),
                                                    perturb=(True,), clamp_lo=(-INF,), clamp_hi=(INF,), beta2=0.99),
+    # the paper's own GAN objective (WGAN-GP) on the GAN shapes
+    "c4_mini_wgan": _c4(n=5, g=(16, 72, 136, 2), d=(2, 136, 72, 1), batch=48, eval_batch=160,
+                        pool=512, interval=2, steps=4, name="c4_mini_wgan").replace(loss=LOSS_WGAN_GP),
+    "c4_mid_wgan": _c4(n=3, g=(64, 512, 512, 2), d=(2, 512, 512, 1), batch=512, eval_batch=512,
+                       pool=2048, interval=1, steps=2, name="c4_mid_wgan").replace(loss=LOSS_WGAN_GP),
+    "c4_wgan": _c4(name="c4_wgan_gp_bf16").replace(loss=LOSS_WGAN_GP),
     # t-test selection and resample-from-prior on the same small shapes
     "c2_mini_ttest": _c2(n=7, widths=(40, 72, 56, 1), batch=24, eval_batch=40, pool=512, interval=2, steps=12,
                          name="c2_mini_ttest").replace(exploit="ttest"),
