@@ -145,6 +145,13 @@ def _algorithmic_work(cfg):
         K = cfg.gan_d_steps
         # K discriminator updates: G forward (B rows), D forward + wgrad on 2B rows, D dgrad above layer 0
         flops = K * (2 * B * wg + 2 * (2 * B) * wd * 2 + 2 * (2 * B) * (wd - d[0] * d[1]))
+        rows_d = 2 * B
+        if cfg.loss == "wgan_gp":
+            # critic update on real, generated and interpolated rows: forward, data-gradient chain and weight gradient
+            # over 3B rows; input gradient of the interpolates; the penalty's second chain up to the last hidden layer
+            rows_d = 3 * B
+            flops = K * (2 * B * wg + 2 * (3 * B) * wd * 2 + 2 * (3 * B) * (wd - d[0] * d[1]) + 2 * B * d[0] * d[1]
+                         + 2 * B * (wd - d[-2] * d[-1]))
         # generator update: G fwd, D fwd, D dgrad to the input, G dgrad + wgrad
         flops += 2 * B * wg + 2 * B * wd + 2 * B * wd + 2 * B * (wg - g[0] * g[1]) + 2 * B * wg
         opt_params = (wg + sum(g[1:])) + K * (wd + sum(d[1:]))
@@ -154,9 +161,9 @@ def _algorithmic_work(cfg):
                     fused_params += g[i] * g[i + 1]
                     fused_flops += 2 * B * g[i] * g[i + 1]
             for i in range(len(d) - 1):
-                if _tc_layer(d[i], d[i + 1], 2 * B):
+                if _tc_layer(d[i], d[i + 1], rows_d):
                     fused_params += K * d[i] * d[i + 1]
-                    fused_flops += K * 2 * (2 * B) * d[i] * d[i + 1]
+                    fused_flops += K * 2 * rows_d * d[i] * d[i + 1]
     else:
         w = cfg.widths[0]
         W = sum(w[i] * w[i + 1] for i in range(len(w) - 1))

@@ -63,7 +63,10 @@ typedef enum pbt_loss {
   PBT_LOSS_MSE = 1,        /* mean_i sum_j (z_ij - y_ij)^2 */
   PBT_LOSS_CE_HARD = 2,    /* softmax cross-entropy, int32 class labels */
   PBT_LOSS_CE_SOFT = 3,    /* cross-entropy against a target distribution */
-  PBT_LOSS_GAN_LOGISTIC = 4 /* non-saturating logistic GAN losses */
+  PBT_LOSS_GAN_LOGISTIC = 4, /* non-saturating logistic GAN losses */
+  PBT_LOSS_WGAN_GP = 5       /* Section 4.3.1: Wasserstein critic with gradient penalty,
+                                L_D = mean D(G(z)) - mean D(x) + gp_lambda mean_b (||grad_x D(xhat_b)||_2 - 1)^2,
+                                xhat_b = eps_b x_b + (1 - eps_b) G(z_b);  L_G = -mean D(G(z)) */
 } pbt_loss;
 
 typedef enum pbt_optimizer {
@@ -138,6 +141,7 @@ typedef struct pbt_spec {
   double ttest_alpha;    /* significance level of the t-test (the paper states none; 0.05 is customary) */
   double resample_prob;  /* probability that explore redraws a slot (the paper states none) */
   double prior_lo[PBT_MAX_NH], prior_hi[PBT_MAX_NH]; /* range of each slot's prior; log-uniform needs 0 < lo <= hi */
+  double gp_lambda;      /* PBT_LOSS_WGAN_GP: weight of the gradient penalty (10 in the paper that introduced it) */
 } pbt_spec;
 
 /*
@@ -207,7 +211,11 @@ int pbt_destroy(pbt_t* p);
  * theta <- step(theta | h) for every member, k times in lockstep (Eq. 2, chained
  * as in Eq. 3).  MLP: forward, loss, backward, optimiser update with the member's
  * own h.  GAN: K discriminator updates then one generator update per step
- * (Section 4.3.1).  Toy: one gradient-ascent step on the surrogate objective.
+ * (Section 4.3.1), on the logistic losses or on the WGAN-GP objective; for the
+ * latter, row b of discriminator update j of a step interpolates with
+ * eps_b = ((w >> 9) + 1/2) / 2^23, w = word b mod 4 of Philox block
+ * j * 65536 + b div 4 of stream 4 at counter (member, step).
+ * Toy: one gradient-ascent step on the surrogate objective.
  */
 int pbt_step(pbt_t* p, int k);
 

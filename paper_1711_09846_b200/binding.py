@@ -21,7 +21,7 @@ PBT_HISTORY = 10
 
 _DTYPE = {"fp64_toy": 0, "fp32": 1, "bf16_fp32master": 2}
 _MODEL = {"toy_quadratic": 0, "mlp": 1, "gan_pair": 2}
-_LOSS = {"toy": 0, "mse": 1, "ce_hard": 2, "ce_soft": 3, "gan_logistic": 4}
+_LOSS = {"toy": 0, "mse": 1, "ce_hard": 2, "ce_soft": 3, "gan_logistic": 4, "wgan_gp": 5}
 _OPT = {"sgd_plain": 0, "sgdm": 1, "adam": 2, "rmsprop": 3}
 
 STATUS = {0: "PBT_OK", 1: "PBT_ERR_INVALID_ARG", 2: "PBT_ERR_UNSUPPORTED", 3: "PBT_ERR_WORKSPACE",
@@ -47,6 +47,7 @@ class PbtSpec(C.Structure):
         ("clamp_lo", C.c_double * PBT_MAX_NH), ("clamp_hi", C.c_double * PBT_MAX_NH),
         ("ttest_alpha", C.c_double), ("resample_prob", C.c_double),
         ("prior_lo", C.c_double * PBT_MAX_NH), ("prior_hi", C.c_double * PBT_MAX_NH),
+        ("gp_lambda", C.c_double),
     ]
 
 
@@ -179,6 +180,7 @@ def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True) -> Pb
         s.prior_kind[k] = {"fixed": 0, "u": 1, "logu": 2}[kind]
         s.prior_lo[k], s.prior_hi[k] = lo, hi
     s.fuse_adam = 1 if fuse_adam else 0
+    s.gp_lambda = getattr(cfg, "gp_lambda", 10.0)
     s.const_lr = 0.0
     s.const_momentum = cfg.momentum
     s.const_beta1, s.const_beta2, s.const_eps, s.const_wd = cfg.beta1, cfg.beta2, cfg.eps, cfg.weight_decay

@@ -202,6 +202,13 @@ __global__ void k_loss_rows(LossArgs a) {
           store_from_float(a.dz, a.dz_dtype, dz_base + c, (p * tsum - t) * a.inv_batch);
         }
     }
+  } else if (a.kind == PBT_LOSS_WGAN_GP) {  // one critic value per row
+    const float d = z[0];
+    const int cls = row < a.n_real_rows ? 0 : (row < 2 * a.n_real_rows ? 1 : 2);
+    if (a.dz && lane == 0)
+      store_from_float(a.dz, a.dz_dtype, dz_base, cls == 0 ? -a.inv_batch : (cls == 1 ? a.inv_batch : 1.f));
+    if (cls == 2) return;  // interpolate: its loss is the penalty, written once the input gradient is known
+    loss = cls == 0 ? -d : d;
   } else {  // PBT_LOSS_GAN_LOGISTIC: one logit per row
     const float d = z[0];
     const bool real = row < a.n_real_rows;
@@ -396,6 +403,72 @@ cudaError_t launch_energy_distance(const float* x, long long stride, int n, int 
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   k_energy_final<<<n_members, 1, 0, s>>>(partial, nblocks, n, fitness);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// WGAN-GP (Section 4.3.1): interpolates between real and generated rows, and the
+// penalty on the norm of the critic's input gradient with its derivative.
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void k_gp_interp(T* __restrict__ x, long long stride, int B, int dim, int j, uint64_t seed,
+                            const Counters* __restrict__ counters) {
+  const int m = blockIdx.y;
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const U4 r = philox4x32_10((uint32_t)m, (uint32_t)counters->step, kStreamInterp, (uint32_t)(j * 65536 + (b >> 2)), seed);
+  // (w >> 9) + 1/2 has 24 significant bits, and so has its complement: both are exact in float
+  const float e = ((float)(r.x[b & 3] >> 9) + 0.5f) * 1.1920928955078125e-07f;
+  const float ome = 1.0f - e;
+  T* xm = x + m * stride;
+  for (int c = 0; c < dim; ++c) {
+    float re, fa;
+    if constexpr (sizeof(T) == 2) {
+      re = __bfloat162float(xm[(long long)b * dim + c]);
+      fa = __bfloat162float(xm[(long long)(B + b) * dim + c]);
+      xm[(long long)(2 * B + b) * dim + c] = __float2bfloat16_rn(fmaf(e, re, ome * fa));
+    } else {
+      re = xm[(long long)b * dim + c];
+      fa = xm[(long long)(B + b) * dim + c];
+      xm[(long long)(2 * B + b) * dim + c] = fmaf(e, re, ome * fa);
+    }
+  }
+}
+
+cudaError_t launch_gp_interp(void* x, int dtype, long long stride, int B, int dim, int j, int n_members, uint64_t seed,
+                             const Counters* counters, cudaStream_t s) {
+  dim3 grid((B + 127) / 128, n_members);
+  if (dtype == kBF16) k_gp_interp<bf16><<<grid, 128, 0, s>>>((bf16*)x, stride, B, dim, j, seed, counters);
+  else k_gp_interp<float><<<grid, 128, 0, s>>>((float*)x, stride, B, dim, j, seed, counters);
+  return cudaGetLastError();
+}
+
+// one warp per (member, row)
+__global__ void k_gp_penalty(const float* __restrict__ gx, long long gx_stride, int B, int dim, float lam,
+                             float inv_batch, float* __restrict__ row_loss, int rows_total, int row_off, void* dv,
+                             int dv_dtype, long long dv_stride) {
+  const int lane = threadIdx.x & 31;
+  const int m = blockIdx.y;
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (b >= B) return;
+  const float* g = gx + m * gx_stride + (long long)b * dim;
+  float ss = 0.f;
+  for (int c = lane; c < dim; c += 32) ss = fmaf(g[c], g[c], ss);
+  ss = warp_sum(ss);
+  const float nrm = sqrtf(ss);
+  const float dev = nrm - 1.0f;
+  if (lane == 0) row_loss[(long long)m * rows_total + row_off + b] = lam * dev * dev;
+  const float scale = nrm > 0.f ? (2.0f * lam * inv_batch) * dev / nrm : 0.f;
+  for (int c = lane; c < dim; c += 32) store_from_float(dv, dv_dtype, m * dv_stride + (long long)b * dim + c, scale * g[c]);
+}
+
+cudaError_t launch_gp_penalty(const float* gx, long long gx_stride, int B, int dim, float lam, float inv_batch,
+                              float* row_loss, int rows_total, int row_off, void* dv, int dv_dtype,
+                              long long dv_stride, int n_members, cudaStream_t s) {
+  const int warps = 8;
+  dim3 grid((B + warps - 1) / warps, n_members);
+  k_gp_penalty<<<grid, warps * 32, 0, s>>>(gx, gx_stride, B, dim, lam, inv_batch, row_loss, rows_total, row_off, dv,
+                                           dv_dtype, dv_stride);
   return cudaGetLastError();
 }
 

@@ -67,6 +67,11 @@ struct pbt_handle {
   void* act[2][PBT_MAX_LAYERS];  // input of layer l of stack s: [N][rows_cap][in_l]
   float* logits[2];              // [N][rows_cap][out_last]
   void* dz[2];                   // ping-pong deltas [N][dz_rows_cap][max_width]
+  // WGAN-GP only: the critic's deltas of every layer are kept until its weight gradients, which need the
+  // penalty's second chain, can be formed: gp_dz[l] is [N][3 batch][out_l]; gp_gx is the input gradient [N][batch][d]
+  void* gp_dz[PBT_MAX_LAYERS];
+  float* gp_gx;
+  bool wgan;
   void* ybatch;
   long long ybatch_stride;  // elements of the target type per member
   // second copy of the training-row buffers: host batches are uploaded here on a copy stream while the step
@@ -162,7 +167,9 @@ int validate(const pbt_spec* s) {
   if (s->batch < 1 || s->eval_batch < 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "batch sizes must be positive");
   if (s->pool_rows < s->batch) return fail(nullptr, PBT_ERR_INVALID_ARG, "pool smaller than one batch");
   if (s->model == PBT_GAN_PAIR) {
-    if (s->loss != PBT_LOSS_GAN_LOGISTIC) return fail(nullptr, PBT_ERR_UNSUPPORTED, "GAN pairs use the logistic loss");
+    if (s->loss != PBT_LOSS_GAN_LOGISTIC && s->loss != PBT_LOSS_WGAN_GP)
+      return fail(nullptr, PBT_ERR_UNSUPPORTED, "GAN pairs use the logistic losses or WGAN-GP");
+    if (s->loss == PBT_LOSS_WGAN_GP && !(s->gp_lambda >= 0.0)) return fail(nullptr, PBT_ERR_INVALID_ARG, "gp_lambda must be >= 0");
     if (s->widths[1][0] != s->widths[0][s->n_layers[0]]) return fail(nullptr, PBT_ERR_INVALID_ARG, "discriminator input != generator output");
     if (s->widths[1][s->n_layers[1]] != 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "discriminator must end in one logit");
     if (s->widths[0][s->n_layers[0]] != 2) return fail(nullptr, PBT_ERR_UNSUPPORTED, "GAN evaluation (energy distance to the ring) is two-dimensional");
@@ -187,6 +194,7 @@ size_t plan(pbt_handle* h, char* base) {
   h->cdt = h->is_bf16 ? kBF16 : kF32;
   h->esz = h->is_bf16 ? 2 : 4;
   h->ns = h->toy ? 0 : (h->gan ? 2 : 1);
+  h->wgan = h->gan && s.loss == PBT_LOSS_WGAN_GP;
   size_t off = 0;
   auto take = [&](size_t bytes) -> char* {
     char* p = base ? base + off : nullptr;
@@ -234,13 +242,14 @@ size_t plan(pbt_handle* h, char* base) {
   h->P_pad = p;
   if (h->gan) {
     h->st[0].rows_cap = s.batch > s.eval_batch ? s.batch : s.eval_batch;
-    h->st[1].rows_cap = 2 * s.batch;
+    h->st[1].rows_cap = (h->wgan ? 3 : 2) * s.batch;   // real, generated (and interpolated) rows
     h->dz_rows_cap = 2 * s.batch;
   } else {
     h->st[0].rows_cap = s.batch > s.eval_batch ? s.batch : s.eval_batch;
     h->dz_rows_cap = s.batch;
   }
   h->rowloss_cap = h->dz_rows_cap > s.eval_batch ? h->dz_rows_cap : s.eval_batch;
+  if (h->wgan && h->rowloss_cap < 3 * s.batch) h->rowloss_cap = 3 * s.batch;
   const size_t slab = (size_t)h->P_pad * sizeof(float);
   h->W32 = (float*)take(N * slab);
   h->O1 = (float*)take(N * slab);
@@ -257,6 +266,11 @@ size_t plan(pbt_handle* h, char* base) {
     h->logits[k] = (float*)take(N * (size_t)st.rows_cap * st.L[st.nl - 1].out * sizeof(float));
   }
   for (int i = 0; i < 2; ++i) h->dz[i] = take(N * (size_t)h->dz_rows_cap * h->max_width * h->esz);
+  h->gp_gx = nullptr;
+  if (h->wgan) {
+    for (int l = 0; l < h->st[1].nl; ++l) h->gp_dz[l] = take(N * (size_t)3 * s.batch * h->st[1].L[l].out * h->esz);
+    h->gp_gx = (float*)take(N * (size_t)s.batch * h->st[1].L[0].in * sizeof(float));
+  }
   if (!h->gan) {
     const int out = h->st[0].L[h->st[0].nl - 1].out;
     if (s.loss == PBT_LOSS_MSE) h->ybatch_stride = (long long)s.batch * out;
@@ -388,60 +402,53 @@ void fill_opt_args(pbt_handle* h, OptArgs* a, int slot_lr, int scalar_base) {
   a->scalars = h->scalars; a->scalar_base = scalar_base;
 }
 
-// dW_l = dZ_l^T a_{l-1}, db_l = column sums of dZ_l, dZ_{l-1} = (dZ_l W_l) * [a_{l-1} > 0].
-// dZ of the last layer is in h->dz[*cur]; on return *cur names the buffer written last.
-// With need_wgrad the optimiser update of the stack is part of this pass: layers whose weight
-// gradient runs on the tensor cores get their Adam update inside that GEMM's epilogue (after the
-// layer's data gradient has read the old weights); everything else (biases, skinny layers,
-// SGD-momentum) is updated by the element-wise kernel over the remaining slab ranges.
-int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride, bool need_wgrad,
-             bool need_input_grad, int* cur, int slot_lr, int scalar_base) {
-  const Stack& st = h->st[k];
+// dC = (dZ_l W_l) [* (mask > 0)]: the data gradient of layer l of stack k for `rows` rows per member.
+int dgrad(pbt_handle* h, int k, int l, int rows, const void* dz, long long dz_stride, void* out, long long out_stride,
+          int out_dtype, const void* mask, long long mask_stride) {
+  const Layer& L = h->st[k].L[l];
+  GemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.M = rows; g.N = L.in; g.K = L.out; g.batch = h->N;
+  g.in_dtype = h->cdt; g.out_dtype = out_dtype;
+  g.A = dz; g.lda = L.out; g.strideA = dz_stride;
+  g.B = weights(h, L.w_off); g.ldb = L.in; g.strideB = h->P_pad; g.b_mn = 1;
+  g.C = out; g.ldc = L.in; g.strideC = out_stride;
+  if (mask) { g.mask = mask; g.ldmask = L.in; g.strideMask = mask_stride; }
+  return gemm(h, g);
+}
+
+// dW_l = dZ_l^T a_{l-1} over `rows` rows and db_l = column sums of the first `bias_rows` rows of dZ_l.
+// Layers whose weight gradient runs on the tensor cores get their Adam update inside that GEMM's epilogue
+// (the caller must have finished every read of the layer's old weights); fused[l] records it.
+int wgrad_layer(pbt_handle* h, int k, int l, int rows, int bias_rows, const void* dz, long long dz_stride,
+                const void* in, long long in_stride, const OptArgs& opt, bool* fused) {
   const pbt_spec& s = h->spec;
-  const long long dzs = dz_stride(h);
-  OptArgs opt;
-  fill_opt_args(h, &opt, slot_lr, scalar_base);
-  bool fused[PBT_MAX_LAYERS] = {false};
-  for (int l = st.nl - 1; l >= 0; --l) {
-    const Layer& L = st.L[l];
-    const void* dz = h->dz[*cur];
-    bool wrote_dgrad = false;
-    if (l > 0 || need_input_grad) {
-      GemmArgs g;
-      memset(&g, 0, sizeof(g));
-      g.M = rows; g.N = L.in; g.K = L.out; g.batch = h->N;
-      g.in_dtype = h->cdt; g.out_dtype = h->cdt;
-      g.A = dz; g.lda = L.out; g.strideA = dzs;
-      g.B = weights(h, L.w_off); g.ldb = L.in; g.strideB = h->P_pad; g.b_mn = 1;
-      g.C = h->dz[1 - *cur]; g.ldc = L.in; g.strideC = dzs;
-      if (l > 0) { g.mask = h->act[k][l]; g.ldmask = L.in; g.strideMask = act_stride(h, k, l); }
-      int rc = gemm(h, g);
-      if (rc) return rc;
-      wrote_dgrad = true;
-    }
-    if (need_wgrad) {
-      GemmArgs g;
-      memset(&g, 0, sizeof(g));
-      g.M = L.out; g.N = L.in; g.K = rows; g.batch = h->N;
-      g.in_dtype = h->cdt; g.out_dtype = kF32;
-      g.A = dz; g.lda = L.out; g.strideA = dzs; g.a_mn = 1;
-      g.B = l == 0 ? in : h->act[k][l]; g.ldb = L.in; g.strideB = l == 0 ? in_stride : act_stride(h, k, l); g.b_mn = 1;
-      g.C = h->G + L.w_off; g.ldc = L.in; g.strideC = h->P_pad;
-      OptArgs lopt = opt;
-      if (s.fuse_adam && s.optimizer == PBT_OPT_ADAM && gemm_tc_supported(g)) {
-        lopt.begin = L.w_off; lopt.count = (long long)L.in * L.out;
-        g.adam = &lopt;
-        if (!s.keep_grad) g.C = nullptr;
-        fused[l] = true;
-      }
-      int rc = gemm(h, g);
-      if (rc) return rc;
-      LAUNCH(h, kLoss, launch_bias_grad(dz, h->cdt, L.out, dzs, rows, L.out, h->G + L.b_off, h->P_pad, h->N, h->stream));
-    }
-    if (wrote_dgrad) *cur = 1 - *cur;
+  const Layer& L = h->st[k].L[l];
+  GemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.M = L.out; g.N = L.in; g.K = rows; g.batch = h->N;
+  g.in_dtype = h->cdt; g.out_dtype = kF32;
+  g.A = dz; g.lda = L.out; g.strideA = dz_stride; g.a_mn = 1;
+  g.B = in; g.ldb = L.in; g.strideB = in_stride; g.b_mn = 1;
+  g.C = h->G + L.w_off; g.ldc = L.in; g.strideC = h->P_pad;
+  OptArgs lopt = opt;
+  if (s.fuse_adam && s.optimizer == PBT_OPT_ADAM && gemm_tc_supported(g)) {
+    lopt.begin = L.w_off; lopt.count = (long long)L.in * L.out;
+    g.adam = &lopt;
+    if (!s.keep_grad) g.C = nullptr;
+    fused[l] = true;
   }
-  if (!need_wgrad) return PBT_OK;
-  // element-wise optimiser over what the fused epilogues did not cover; adjacent ranges are merged
+  int rc = gemm(h, g);
+  if (rc) return rc;
+  LAUNCH(h, kLoss, launch_bias_grad(dz, h->cdt, L.out, dz_stride, bias_rows, L.out, h->G + L.b_off, h->P_pad, h->N, h->stream));
+  return PBT_OK;
+}
+
+// element-wise optimiser over what the fused epilogues did not cover (biases, skinny layers, SGD-momentum,
+// RMSProp); adjacent slab ranges are merged into one launch
+int finish_optimizer(pbt_handle* h, int k, const bool* fused, const OptArgs& opt) {
+  const pbt_spec& s = h->spec;
+  const Stack& st = h->st[k];
   long long rb = -1, re = -1;
   auto flush = [&]() -> int {
     if (rb < 0) return PBT_OK;
@@ -470,6 +477,37 @@ int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride
   if (rc) return rc;
   if (s.optimizer == PBT_OPT_ADAM) LAUNCH(h, kOther, launch_adam_advance(opt, h->stream));
   return PBT_OK;
+}
+
+// dW_l = dZ_l^T a_{l-1}, db_l = column sums of dZ_l, dZ_{l-1} = (dZ_l W_l) * [a_{l-1} > 0].
+// dZ of the last layer is in h->dz[*cur]; on return *cur names the buffer written last.
+// With need_wgrad the optimiser update of the stack is part of this pass: a layer's fused update runs
+// after the layer's data gradient has read the old weights.
+int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride, bool need_wgrad,
+             bool need_input_grad, int* cur, int slot_lr, int scalar_base) {
+  const Stack& st = h->st[k];
+  const long long dzs = dz_stride(h);
+  OptArgs opt;
+  fill_opt_args(h, &opt, slot_lr, scalar_base);
+  bool fused[PBT_MAX_LAYERS] = {false};
+  for (int l = st.nl - 1; l >= 0; --l) {
+    const void* dz = h->dz[*cur];
+    bool wrote_dgrad = false;
+    if (l > 0 || need_input_grad) {
+      int rc = dgrad(h, k, l, rows, dz, dzs, h->dz[1 - *cur], dzs, h->cdt, l > 0 ? h->act[k][l] : nullptr,
+                     l > 0 ? act_stride(h, k, l) : 0);
+      if (rc) return rc;
+      wrote_dgrad = true;
+    }
+    if (need_wgrad) {
+      int rc = wgrad_layer(h, k, l, rows, rows, dz, dzs, l == 0 ? in : h->act[k][l],
+                           l == 0 ? in_stride : act_stride(h, k, l), opt, fused);
+      if (rc) return rc;
+    }
+    if (wrote_dgrad) *cur = 1 - *cur;
+  }
+  if (!need_wgrad) return PBT_OK;
+  return finish_optimizer(h, k, fused, opt);
 }
 
 int loss_and_dz(pbt_handle* h, int k, int rows, int n_real, const void* target, long long target_stride,
@@ -555,10 +593,107 @@ int step_gan(pbt_handle* h) {
   return PBT_OK;
 }
 
+// Section 4.3.1 with the paper's own objective (WGAN-GP): K critic updates, then one generator update on
+// L_G = -mean D(G(z)).  A critic update sends three row blocks per member through the critic: real rows,
+// generated rows and their interpolates xhat.  Back-propagation of all three is one chain of data-gradient
+// GEMMs over 3B rows (the interpolates start from dD/dD = 1, so their deltas u_l are the factors of the input
+// gradient grad_x D(xhat) = u_0 W_0).  The penalty's gradient with respect to W_l is u_l^T dv_l with a second,
+// forward-running chain dv_0 = d(penalty)/d(grad_x D), dv_{l+1} = (dv_l W_l^T) * [a_{l+1}(xhat) > 0].  dv_l
+// overwrites the interpolates' rows of layer l's input, which nothing reads any more (each element is the
+// ReLU mask of exactly the element that replaces it, read by the thread that then writes it), so that ONE
+// weight-gradient GEMM over 3B rows gives  dZ_l^T a_{l-1} (real, generated rows) + u_l^T dv_l.
+int step_wgan(pbt_handle* h) {
+  const pbt_spec& s = h->spec;
+  const int B = s.batch;
+  const Stack& G = h->st[0];
+  const Stack& D = h->st[1];
+  const int zdim = G.L[0].in, xdim = D.L[0].in;
+  const long long d_in_stride = act_stride(h, 1, 0);
+  const float lam = (float)s.gp_lambda;
+  int rc;
+  for (int j = 0; j < s.gan_d_steps; ++j) {
+    LAUNCH(h, kCopy, launch_gather_window((char*)h->act[1][0], d_in_stride * h->esz, 0, (const char*)h->data.x_pool,
+                                          xdim * h->esz, B, s.pool_rows, h->N, j, 0, h->seed, h->counters, h->stream));
+    LAUNCH(h, kCopy, launch_gather_window((char*)h->act[0][0], act_stride(h, 0, 0) * h->esz, 0, (const char*)h->data.z_pool,
+                                          zdim * h->esz, B, s.pool_rows, h->N, j, 1, h->seed, h->counters, h->stream));
+    rc = forward(h, 0, B, h->act[0][0], act_stride(h, 0, 0));
+    if (rc) return rc;
+    LAUNCH(h, kCopy, launch_copy_rows((char*)h->act[1][0] + (size_t)B * xdim * h->esz, h->cdt, xdim, d_in_stride, h->logits[0],
+                                      xdim, logits_stride(h, 0), B, xdim, h->N, h->stream));
+    LAUNCH(h, kOther, launch_gp_interp(h->act[1][0], h->cdt, d_in_stride, B, xdim, j, h->N, h->seed, h->counters, h->stream));
+    rc = forward(h, 1, 3 * B, h->act[1][0], d_in_stride);
+    if (rc) return rc;
+    // deltas of the last layer for all 3B rows; losses of the real and generated rows
+    {
+      LossArgs a;
+      memset(&a, 0, sizeof(a));
+      a.kind = PBT_LOSS_WGAN_GP; a.n_members = h->N; a.rows = 3 * B; a.cols = 1;
+      a.n_real_rows = B; a.inv_batch = 1.0f / (float)B;
+      a.logits = h->logits[1]; a.ld_logits = 1; a.stride_logits = logits_stride(h, 1);
+      a.dz = h->gp_dz[D.nl - 1]; a.dz_dtype = h->cdt; a.ld_dz = 1; a.stride_dz = 3ll * B;
+      a.row_loss = h->row_loss;
+      LAUNCH(h, kLoss, launch_loss_rows(a, h->stream));
+    }
+    for (int l = D.nl - 1; l >= 1; --l) {
+      rc = dgrad(h, 1, l, 3 * B, h->gp_dz[l], 3ll * B * D.L[l].out, h->gp_dz[l - 1], 3ll * B * D.L[l].in, h->cdt,
+                 h->act[1][l], act_stride(h, 1, l));
+      if (rc) return rc;
+    }
+    // grad_x D(xhat) = u_0 W_0 (kept in fp32), then the penalty and the start of its chain, dv_0, over xhat
+    rc = dgrad(h, 1, 0, B, (const char*)h->gp_dz[0] + (size_t)2 * B * D.L[0].out * h->esz, 3ll * B * D.L[0].out, h->gp_gx,
+               (long long)B * xdim, kF32, nullptr, 0);
+    if (rc) return rc;
+    LAUNCH(h, kLoss, launch_gp_penalty(h->gp_gx, (long long)B * xdim, B, xdim, lam, 1.0f / (float)B, h->row_loss, 3 * B, 2 * B,
+                                       (char*)h->act[1][0] + (size_t)2 * B * xdim * h->esz, h->cdt, d_in_stride, h->N,
+                                       h->stream));
+    LAUNCH(h, kLoss, launch_reduce_rows(h->row_loss, 3 * B, h->N, 1.0f / (float)B, h->last_loss + 1, 0, 2, h->stream));
+    for (int l = 0; l + 1 < D.nl; ++l) {
+      const Layer& L = D.L[l];
+      GemmArgs g;
+      memset(&g, 0, sizeof(g));
+      g.M = B; g.N = L.out; g.K = L.in; g.batch = h->N;
+      g.in_dtype = h->cdt; g.out_dtype = h->cdt;
+      g.A = (const char*)h->act[1][l] + (size_t)2 * B * L.in * h->esz; g.lda = L.in; g.strideA = act_stride(h, 1, l);
+      g.B = weights(h, L.w_off); g.ldb = L.in; g.strideB = h->P_pad;
+      g.C = (char*)h->act[1][l + 1] + (size_t)2 * B * L.out * h->esz; g.ldc = L.out; g.strideC = act_stride(h, 1, l + 1);
+      g.mask = g.C; g.ldmask = L.out; g.strideMask = g.strideC;
+      rc = gemm(h, g);
+      if (rc) return rc;
+    }
+    OptArgs opt;
+    fill_opt_args(h, &opt, s.slot_lr_d, 2);
+    bool fused[PBT_MAX_LAYERS] = {false};
+    for (int l = D.nl - 1; l >= 0; --l) {
+      rc = wgrad_layer(h, 1, l, 3 * B, 2 * B, h->gp_dz[l], 3ll * B * D.L[l].out, h->act[1][l], act_stride(h, 1, l), opt, fused);
+      if (rc) return rc;
+    }
+    rc = finish_optimizer(h, 1, fused, opt);
+    if (rc) return rc;
+  }
+  // generator update
+  LAUNCH(h, kCopy, launch_gather_window((char*)h->act[0][0], act_stride(h, 0, 0) * h->esz, 0, (const char*)h->data.z_pool,
+                                        zdim * h->esz, B, s.pool_rows, h->N, s.gan_d_steps, 1, h->seed, h->counters, h->stream));
+  rc = forward(h, 0, B, h->act[0][0], act_stride(h, 0, 0));
+  if (rc) return rc;
+  LAUNCH(h, kCopy, launch_copy_rows(h->act[1][0], h->cdt, xdim, d_in_stride, h->logits[0], xdim, logits_stride(h, 0), B, xdim,
+                                    h->N, h->stream));
+  rc = forward(h, 1, B, h->act[1][0], d_in_stride);
+  if (rc) return rc;
+  rc = loss_and_dz(h, 1, B, B, nullptr, 0, true, 0, 1.0f / B, h->last_loss, 2);
+  if (rc) return rc;
+  int cur = 0;
+  rc = backward(h, 1, B, h->act[1][0], d_in_stride, false, true, &cur, s.slot_lr_d, 2);
+  if (rc) return rc;
+  return backward(h, 0, B, h->act[0][0], act_stride(h, 0, 0), true, false, &cur, s.slot_lr, 0);
+}
+
 int one_step(pbt_handle* h) {
   int rc;
   if (h->toy) {
     LAUNCH(h, kOpt, launch_toy_step(h->theta, (const double*)h->H, h->N, h->nh, h->spec.toy_eta, h->stream));
+  } else if (h->wgan) {
+    rc = step_wgan(h);
+    if (rc) return rc;
   } else if (h->gan) {
     rc = step_gan(h);
     if (rc) return rc;

@@ -15,7 +15,7 @@ typedef __nv_bfloat16 bf16;
 // Philox4x32-10 (Salmon et al., SC'11, Section 3.3), device + host.
 // counter = (member, round_or_step, stream, block), key = (seed_lo, seed_hi)
 // ---------------------------------------------------------------------------
-enum PhiloxStream : uint32_t { kStreamExploit = 0, kStreamExplore = 1, kStreamBatch = 2, kStreamInit = 3 };
+enum PhiloxStream : uint32_t { kStreamExploit = 0, kStreamExplore = 1, kStreamBatch = 2, kStreamInit = 3, kStreamInterp = 4 };
 
 struct U4 {
   uint32_t x[4];
@@ -202,7 +202,8 @@ cudaError_t launch_copy_rows(void* dst, int dst_dtype, long long dst_ld, long lo
 struct LossArgs {
   int kind;        // pbt_loss
   int n_members, rows, cols;
-  int n_real_rows; // GAN: rows < n_real_rows are labelled real
+  int n_real_rows; // GAN: rows < n_real_rows are labelled real; WGAN-GP: the next n_real_rows are generated rows and
+                   // any rows after those are interpolates (dL/dz = 1, their loss is written by launch_gp_penalty)
   float inv_batch; // 1 / B  (scale of dL/dz and of the mean)
   const float* logits; long long ld_logits, stride_logits;
   const void* target; long long stride_target;   // elements of the target type; 0 = shared by all members
@@ -222,6 +223,15 @@ cudaError_t launch_toy_eval(const double* theta, double* fitness, int n_members,
 cudaError_t launch_energy_distance(const float* x, long long stride, int n, int n_members, double* partial,
                                    float* fitness, cudaStream_t s);
 int energy_partial_count(int n);  // doubles of scratch per member
+// WGAN-GP (Section 4.3.1).  x holds, per member, rows [0,B) real, [B,2B) generated; writes rows [2B,3B):
+// xhat_b = eps_b real_b + (1 - eps_b) fake_b, eps_b from the interpolation stream at (member, step, block j*65536 + b/4)
+cudaError_t launch_gp_interp(void* x, int dtype, long long stride, int B, int dim, int j, int n_members, uint64_t seed,
+                             const Counters* counters, cudaStream_t s);
+// gx[m][b][dim] = grad_x D(xhat_b).  row_loss[m][row_off + b] = lam (||gx_b|| - 1)^2 (row stride rows_total) and
+// dv[m][b][:] = (2 lam / B)(||gx_b|| - 1) / ||gx_b|| * gx_b (zero where the norm is zero), in the operand type
+cudaError_t launch_gp_penalty(const float* gx, long long gx_stride, int B, int dim, float lam, float inv_batch,
+                              float* row_loss, int rows_total, int row_off, void* dv, int dv_dtype,
+                              long long dv_stride, int n_members, cudaStream_t s);
 cudaError_t launch_advance_step(Counters* c, cudaStream_t s);
 
 }  // namespace pbt

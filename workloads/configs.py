@@ -193,6 +193,11 @@ CONFIGS: Dict[str, PBTConfig] = {
     "c4_mid_wgan": _c4(n=3, g=(64, 512, 512, 2), d=(2, 512, 512, 1), batch=512, eval_batch=512,
                        pool=2048, interval=1, steps=2, name="c4_mid_wgan").replace(loss=LOSS_WGAN_GP),
     "c4_wgan": _c4(name="c4_wgan_gp_bf16").replace(loss=LOSS_WGAN_GP),
+    # fp32 compute, one critic update per step: every tensor is updated once per step, so the step's stored gradient
+    # says which elements Adam's sign-like early updates make ill-conditioned (the critic's exact +-1/B deltas cancel
+    # to zero in many bias-gradient sums)
+    "c4_mini_wgan_fp32": _c4(n=4, g=(16, 72, 136, 2), d=(2, 136, 72, 1), batch=48, eval_batch=160, pool=512, interval=2,
+                             steps=4, name="c4_mini_wgan_fp32").replace(loss=LOSS_WGAN_GP, dtype=FP32, gan_d_steps=1),
     # t-test selection and resample-from-prior on the same small shapes
     "c2_mini_ttest": _c2(n=7, widths=(40, 72, 56, 1), batch=24, eval_batch=40, pool=512, interval=2, steps=12,
                          name="c2_mini_ttest").replace(exploit="ttest"),
