@@ -317,7 +317,7 @@ def main():
     pop.step(3)
     pop.synchronize()
     probe_ms = (time.perf_counter() - t_probe0) / 3 * 1e3
-    two_pass = args.graph == 1 or (args.graph < 0 and probe_ms < 3.0)
+    two_pass = args.graph == 1 or (args.graph < 0 and probe_ms < 6.0)
 
     # ---- timed region: device-resident inputs, CUDA events on the library's stream ----
     sampler = ClockSampler(local)
