@@ -4,15 +4,22 @@
 // The gradient goes from tensor memory straight into the update: it is never written to HBM (unless the
 // caller asks for a copy), which removes 8 of the 34 bytes per parameter that a separate optimiser pass moves.
 //
+// The tile is computed TRANSPOSED, D[i][o] (128 inputs i x 256 outputs o, layer input as the A operand): a
+// tensor-memory lane is then an index i, which is the contiguous direction of W[out][in] in memory, so that a
+// warp's 32 lanes hold 32 consecutive floats of one weight row and a 32-column chunk of the accumulator is a box
+// of 32 weight rows x 512 contiguous bytes.  (With lanes = weight rows the same chunk was 128 rows x 128 bytes;
+// 128-byte pieces 8 KB apart cost about a tenth of the HBM bandwidth against 512-byte runs.)
+//
 // The update is HBM-bound (12 bytes in, 14 bytes out per parameter), so the kernel is organised around keeping
 // ~100 KB of that traffic in flight per SM without holding it in registers:
 //   warp 0       TMA producer for the GEMM operands (2-stage ring, the contraction over the batch is short)
 //   warp 1       tensor-memory allocation + tcgen05.mma issue (128 x 256 tile, accumulator double-buffered)
-//   warp 2       TMA loader for the optimiser state: per 32-column chunk of the tile one 128 x 32 fp32 box each of
-//                master weights, first and second moment into a ring of two slots (128-byte swizzle)
+//   warp 2       TMA loader for the optimiser state: per 32-column chunk of the tile one box of 32 weight rows x
+//                128 floats each of master weights, first and second moment into a ring of two slots (row-major,
+//                no swizzle: a warp reads and writes 128 consecutive bytes of a box row)
 //   warp 3       TMA storer: when the sixteen update warps are done with a slot, stores the three boxes back in
 //                place plus the bf16 shadow box, and hands the slot back to the loader once it has been read
-//   warps 4..19  update: tcgen05.ld of 8 gradient columns of the thread's row, Adam on the slot in shared memory
+//   warps 4..19  update: tcgen05.ld of 8 gradient columns (weight rows) of the thread's lane, Adam on the slot
 // All mbarrier waits are bounded; on expiry PBT_ERR_TIMEOUT is recorded and every role leaves its loop.
 #include <string.h>
 
@@ -27,7 +34,7 @@ using namespace tc;
 constexpr int kBM = 128, kBN = 256, kBK = 64;
 constexpr int kStages = 2, kSlots = 2, kChunk = 32, kUpdWarps = 16;
 constexpr int kColsPerWarp = kChunk / (kUpdWarps / 4);   // gradient columns one update thread handles per chunk
-static_assert(kColsPerWarp == 8 || kColsPerWarp == 16, "update warps per TMEM lane quadrant");
+static_assert(kColsPerWarp == 4 || kColsPerWarp == 8 || kColsPerWarp == 16, "update warps per TMEM lane quadrant");
 constexpr int kThreads = 32 * (4 + kUpdWarps);
 constexpr int kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2, kStageBytes = kABytes + kBBytes;
 constexpr int kBoxBytes = kBM * kChunk * 4;     // one fp32 state box
@@ -40,7 +47,7 @@ constexpr int kSmemTotal = kBarOffset + 256 + 1024;
 static_assert(kSmemTotal <= 232448, "shared memory budget of one CTA");
 
 struct FusedParams {
-  int M, N, K, batch;
+  int M, N, K, batch;   // of the transposed product: M = layer inputs (tile rows / lanes), N = layer outputs
   int tiles_m, tiles_n, num_tiles, k_blocks;
   float* gout; long long ldc, strideC;  // optional copy of the gradient (may be null)
   Counters* counters;
@@ -151,9 +158,9 @@ k_wgrad_adam(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           if (!mbar_wait(&sempty[slot], sphase ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* box = smem + kSlotOffset + slot * kSlotBytes;
           mbar_expect_tx(&sfull[slot], kSlotBytes);
-          tma_load_3d(box, &tmW, &sfull[slot], col, m0, member);
-          tma_load_3d(box + kBoxBytes, &tmM, &sfull[slot], col, m0, member);
-          tma_load_3d(box + 2 * kBoxBytes, &tmV, &sfull[slot], col, m0, member);
+          tma_load_3d(box, &tmW, &sfull[slot], m0, col, member);
+          tma_load_3d(box + kBoxBytes, &tmM, &sfull[slot], m0, col, member);
+          tma_load_3d(box + 2 * kBoxBytes, &tmV, &sfull[slot], m0, col, member);
           if (++slot == kSlots) { slot = 0; sphase ^= 1; }
         }
       }
@@ -172,10 +179,10 @@ k_wgrad_adam(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
           if (col >= p.N) break;
           if (!mbar_wait(&sdone[slot], sphase, abort_flag)) { ok = false; break; }
           const uint8_t* box = smem + kSlotOffset + slot * kSlotBytes;
-          tma_store_3d(&tmW, box, col, m0, member);
-          tma_store_3d(&tmM, box + kBoxBytes, col, m0, member);
-          tma_store_3d(&tmV, box + 2 * kBoxBytes, col, m0, member);
-          tma_store_3d(&tmW16, smem + kW16Offset + slot * kW16Bytes, col, m0, member);
+          tma_store_3d(&tmW, box, m0, col, member);
+          tma_store_3d(&tmM, box + kBoxBytes, m0, col, member);
+          tma_store_3d(&tmV, box + 2 * kBoxBytes, m0, col, member);
+          tma_store_3d(&tmW16, smem + kW16Offset + slot * kW16Bytes, m0, col, member);
           tma_store_commit();
           tma_store_wait_read();           // shared memory of the slot may be overwritten now
           mbar_arrive(&sempty[slot]);
@@ -210,7 +217,7 @@ k_wgrad_adam(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       const float omb1 = 1.f - b1, omb2 = 1.f - b2, lrwd = lr * wd;
       const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kBN + half * kColsPerWarp);
       uint32_t g[kColsPerWarp];
-      if (kColsPerWarp == 16) tmem_ld16(tacc, g); else tmem_ld8(tacc, g);
+      tmem_ld_cols<kColsPerWarp>(tacc, g);
 #pragma unroll 1
       for (int c = 0; c < kChunks; ++c) {
         const int col0 = n0 + c * kChunk;
@@ -222,44 +229,35 @@ k_wgrad_adam(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const bool last = (c + 1 == kChunks) || (col0 + kChunk >= p.N);
         if (!last) {
           // next chunk's gradient while this one is applied
-          if (kColsPerWarp == 16) tmem_ld16(tacc + (c + 1) * kChunk, g); else tmem_ld8(tacc + (c + 1) * kChunk, g);
+          tmem_ld_cols<kColsPerWarp>(tacc + (c + 1) * kChunk, g);
         } else {
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&tempty[acc]);   // the accumulator can be reused by the MMA warp
         }
         if (!mbar_wait(&sfull[slot], sphase, abort_flag)) { ok = false; break; }
-        uint8_t* box = smem + kSlotOffset + slot * kSlotBytes;
-        uint8_t* w16row = smem + kW16Offset + slot * kW16Bytes + rloc * (kChunk * 2) + half * (kColsPerWarp * 2);
+        // box row r (0..31) = weight row col0 + r, 128 floats = inputs m0 .. m0+127: this thread owns input rloc
+        float* box = reinterpret_cast<float*>(smem + kSlotOffset + slot * kSlotBytes) + (half * kColsPerWarp) * kBM + rloc;
+        bf16* w16 = reinterpret_cast<bf16*>(smem + kW16Offset + slot * kW16Bytes) + (half * kColsPerWarp) * kBM + rloc;
+        constexpr int kBoxFloats = kBoxBytes / 4;
 #pragma unroll
-        for (int j = 0; j < kColsPerWarp / 4; ++j) {
-          // 16-byte piece (half * kColsPerWarp/4 + j) of this thread's 128-byte row sits at position piece ^ (row & 7)
-          const int off = rloc * 128 + (((half * (kColsPerWarp / 4) + j) ^ (rloc & 7)) << 4);
-          float4 w = *reinterpret_cast<float4*>(box + off);
-          float4 m1 = *reinterpret_cast<float4*>(box + kBoxBytes + off);
-          float4 m2 = *reinterpret_cast<float4*>(box + 2 * kBoxBytes + off);
-          float4 nw;
-          nw.x = adam_one(w.x, m1.x, m2.x, gf[4 * j + 0], b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
-          nw.y = adam_one(w.y, m1.y, m2.y, gf[4 * j + 1], b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
-          nw.z = adam_one(w.z, m1.z, m2.z, gf[4 * j + 2], b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
-          nw.w = adam_one(w.w, m1.w, m2.w, gf[4 * j + 3], b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
-          *reinterpret_cast<float4*>(box + off) = nw;
-          *reinterpret_cast<float4*>(box + kBoxBytes + off) = m1;
-          *reinterpret_cast<float4*>(box + 2 * kBoxBytes + off) = m2;
-          __nv_bfloat162 lo = __floats2bfloat162_rn(nw.x, nw.y), hi = __floats2bfloat162_rn(nw.z, nw.w);
-          uint2 u;
-          u.x = *reinterpret_cast<uint32_t*>(&lo);
-          u.y = *reinterpret_cast<uint32_t*>(&hi);
-          *reinterpret_cast<uint2*>(w16row + j * 8) = u;
+        for (int j = 0; j < kColsPerWarp; ++j) {
+          const float w = box[j * kBM];
+          float m1 = box[kBoxFloats + j * kBM];
+          float m2 = box[2 * kBoxFloats + j * kBM];
+          const float nw = adam_one(w, m1, m2, gf[j], b1, omb1, b2, omb2, inv_bc1, inv_bc2, lr, eps, lrwd);
+          box[j * kBM] = nw;
+          box[kBoxFloats + j * kBM] = m1;
+          box[2 * kBoxFloats + j * kBM] = m2;
+          w16[j * kBM] = __float2bfloat16_rn(nw);
         }
         if (p.gout) {
-          const int row = m0 + rloc;
-          if (row < p.M) {
-            float* gp = p.gout + member * p.strideC + (long long)row * p.ldc;
+          const int in_idx = m0 + rloc;
+          if (in_idx < p.M) {
 #pragma unroll
             for (int j = 0; j < kColsPerWarp; ++j) {
-              const int col = col0 + half * kColsPerWarp + j;
-              if (col < p.N) gp[col] = gf[j];
+              const int out_idx = col0 + half * kColsPerWarp + j;
+              if (out_idx < p.N) p.gout[member * p.strideC + (long long)out_idx * p.ldc + in_idx] = gf[j];
             }
           }
         }
@@ -280,13 +278,14 @@ k_wgrad_adam(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
 // g describes the weight-gradient GEMM (A = dZ, B = layer input, both MN-major bf16, M = out, N = in,
 // K = batch rows); g.adam carries the slab pointers and the layer's offset; g.C, if not null, receives the gradient.
+// The kernel computes the transposed product, so g's B operand is its A operand and g.N its M.
 cudaError_t launch_wgrad_adam(const GemmArgs& g, Counters* counters, cudaStream_t s) {
   if (!g.adam || !g.a_mn || !g.b_mn || g.in_dtype != kBF16 || !g.adam->w16 || !g.adam->opt2) return cudaErrorInvalidValue;
   FusedParams p;
   memset(&p, 0, sizeof(p));
-  p.M = g.M; p.N = g.N; p.K = g.K; p.batch = g.batch;
-  p.tiles_m = (g.M + kBM - 1) / kBM;
-  p.tiles_n = (g.N + kBN - 1) / kBN;
+  p.M = g.N; p.N = g.M; p.K = g.K; p.batch = g.batch;
+  p.tiles_m = (p.M + kBM - 1) / kBM;
+  p.tiles_n = (p.N + kBN - 1) / kBN;
   p.num_tiles = p.tiles_m * p.tiles_n * g.batch;
   p.k_blocks = (g.K + kBK - 1) / kBK;
   p.gout = reinterpret_cast<float*>(g.C); p.ldc = g.ldc; p.strideC = g.strideC;
@@ -295,12 +294,13 @@ cudaError_t launch_wgrad_adam(const GemmArgs& g, Counters* counters, cudaStream_
   const OptArgs& o = *g.adam;
   CUtensorMap tmA, tmB, tmW, tmM, tmV, tmW16;
   const int ab = (g.batch > 1 && g.strideA != 0) ? g.batch : 1, bb = (g.batch > 1 && g.strideB != 0) ? g.batch : 1;
-  bool ok = make_map(&tmA, g.A, g.M, g.K, g.lda, ab, g.strideA, kBK) &&
-            make_map(&tmB, g.B, g.N, g.K, g.ldb, bb, g.strideB, kBK) &&
-            make_map(&tmW, o.w32 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kBM, 4, kChunk, 128) &&
-            make_map(&tmM, o.opt1 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kBM, 4, kChunk, 128) &&
-            make_map(&tmV, o.opt2 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kBM, 4, kChunk, 128) &&
-            make_map(&tmW16, o.w16 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kBM, 2, kChunk, 0);
+  // operand roles swapped (the layer input is the kernel's A); state boxes: kChunk weight rows x kBM inputs, row-major
+  bool ok = make_map(&tmA, g.B, g.N, g.K, g.ldb, bb, g.strideB, kBK) &&
+            make_map(&tmB, g.A, g.M, g.K, g.lda, ab, g.strideA, kBK) &&
+            make_map(&tmW, o.w32 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kChunk, 4, kBM, 0) &&
+            make_map(&tmM, o.opt1 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kChunk, 4, kBM, 0) &&
+            make_map(&tmV, o.opt2 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kChunk, 4, kBM, 0) &&
+            make_map(&tmW16, o.w16 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kChunk, 2, kBM, 0);
   if (!ok) return cudaErrorInvalidValue;
   if (g.batch > 1 && (g.strideA == 0 || g.strideB == 0)) return cudaErrorInvalidValue;  // operands are per member here
   static bool configured = false;
