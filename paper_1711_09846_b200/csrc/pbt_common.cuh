@@ -131,15 +131,17 @@ __device__ __forceinline__ void st_bf16x4(bf16* p, float4 v) {
   *reinterpret_cast<uint2*>(p) = u;
 }
 
+// Every operation is an explicitly rounded intrinsic: the compiler's choice of where to contract a multiply and an add
+// depends on the surrounding code, and the fused and the separate update must give identical bits.
 __device__ __forceinline__ float adam_one(float w, float& m1, float& m2, float g, float b1, float omb1, float b2,
                                           float omb2, float inv_bc1, float inv_bc2, float lr, float eps,
                                           float lrwd) {
-  m1 = __fmaf_rn(b1, m1, omb1 * g);
-  m2 = __fmaf_rn(b2, m2, omb2 * g * g);
-  const float mhat = m1 * inv_bc1;
-  const float vhat = m2 * inv_bc2;
-  const float upd = __fdividef(mhat, sqrtf(vhat) + eps);
-  return w - lr * upd - lrwd * w;
+  m1 = __fmaf_rn(b1, m1, __fmul_rn(omb1, g));
+  m2 = __fmaf_rn(b2, m2, __fmul_rn(__fmul_rn(omb2, g), g));
+  const float mhat = __fmul_rn(m1, inv_bc1);
+  const float vhat = __fmul_rn(m2, inv_bc2);
+  const float upd = __fdividef(mhat, __fadd_rn(__fsqrt_rn(vhat), eps));
+  return __fmaf_rn(-lrwd, w, __fmaf_rn(-lr, upd, w));
 }
 
 #endif  // __CUDACC__
