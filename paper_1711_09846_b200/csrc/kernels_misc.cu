@@ -288,8 +288,46 @@ __global__ void k_bias_grad(const T* __restrict__ dz, long long ld, long long st
   }
 }
 
+// bf16 deltas with 16-byte alignment: a lane reads 8 columns per row, a warp 512 contiguous bytes; warp w adds rows
+// w, w + 8, ... and the eight partial sums are combined in order, exactly like the scalar kernel above (same bits).
+__global__ void __launch_bounds__(256) k_bias_grad_bf16x8(const bf16* __restrict__ dz, long long ld, long long stride, int rows,
+                                                          int cols, float* __restrict__ out, long long out_stride) {
+  __shared__ float sh[8][256 + 8];
+  const int m = blockIdx.y, lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int c0 = blockIdx.x * 256 + lane * 8;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (c0 < cols) {
+    const bf16* p = dz + m * stride + c0;
+#pragma unroll 4
+    for (int r = w; r < rows; r += 8) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(p + (long long)r * ld));
+      const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        acc[2 * j] += __uint_as_float(u[j] << 16);
+        acc[2 * j + 1] += __uint_as_float(u[j] & 0xFFFF0000u);
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) sh[w][lane * 8 + j] = acc[j];
+  __syncthreads();
+  const int c = blockIdx.x * 256 + threadIdx.x;
+  if (c < cols) {
+    float t = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) t += sh[j][threadIdx.x];
+    out[m * out_stride + c] = t;
+  }
+}
+
 cudaError_t launch_bias_grad(const void* dz, int dz_dtype, long long ld, long long stride, int rows, int cols,
                              float* out, long long out_stride, int n_members, cudaStream_t s) {
+  if (dz_dtype == kBF16 && cols % 8 == 0 && cols >= 256 && ld % 8 == 0 && stride % 8 == 0 && ((uintptr_t)dz & 15) == 0) {
+    dim3 grid((cols + 255) / 256, n_members);
+    k_bias_grad_bf16x8<<<grid, 256, 0, s>>>((const bf16*)dz, ld, stride, rows, cols, out, out_stride);
+    return cudaGetLastError();
+  }
   dim3 grid((cols + 31) / 32, n_members), block(32, 8);
   if (dz_dtype == kBF16)
     k_bias_grad<bf16><<<grid, block, 0, s>>>((const bf16*)dz, ld, stride, rows, cols, out, out_stride);
