@@ -33,6 +33,52 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, float* buf, uin
   // neither latency sits on the warp's critical path.
   constexpr int kChunkStep = 32 * (NEPIW / 4);
   uint32_t r[32];
+  // Interior tiles with bf16 output (the bulk of the forward and data-gradient GEMMs) take a path with no bounds
+  // checks, pointers advanced by constant steps and the ReLU mask applied to the packed bf16 pairs: the epilogue
+  // warps are bound by instruction issue, two warps per scheduler, so the instruction count per element is what
+  // decides whether the epilogue hides behind a short main loop.
+  if (vec_ok && p.out_dtype == kBF16 && m0 + kBM <= p.M && n0 + BN <= p.N) {
+    const long long row0 = m0 + q * 32 + rsub;
+    bf16* crow = reinterpret_cast<bf16*>(p.C) + member * p.strideC + row0 * p.ldc + n0 + cc;
+    const bf16* mrow = p.mask ? p.mask + member * p.strideMask + row0 * p.ldmask + n0 + cc : nullptr;
+    const long long cstep = 4 * p.ldc, mstep = 4 * p.ldmask;
+    const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
+    tmem_ld32(tacc + half * 32, r);
+#pragma unroll 1
+    for (int c0 = half * 32; c0 < BN; c0 += kChunkStep) {
+      uint2 mk[8];
+      if (mrow) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mk[i] = __ldg(reinterpret_cast<const uint2*>(mrow + c0 + i * mstep));
+      }
+      tmem_ld_wait();
+      __syncwarp();  // the previous chunk's phase-2 reads of `buf` are complete
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        *reinterpret_cast<uint4*>(&buf[lane * kEpiPitch + j * 4]) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+      if (c0 + kChunkStep < BN) tmem_ld32(tacc + c0 + kChunkStep, r);
+      __syncwarp();
+      float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (bias) bv = __ldg(reinterpret_cast<const float4*>(bias + n0 + c0 + cc));
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float4 a4 = *reinterpret_cast<const float4*>(&buf[(i * 4 + rsub) * kEpiPitch + cc]);
+        if (bias) { a4.x += bv.x; a4.y += bv.y; a4.z += bv.z; a4.w += bv.w; }
+        if (p.relu) { a4.x = fmaxf(a4.x, 0.f); a4.y = fmaxf(a4.y, 0.f); a4.z = fmaxf(a4.z, 0.f); a4.w = fmaxf(a4.w, 0.f); }
+        __nv_bfloat162 t0 = __floats2bfloat162_rn(a4.x, a4.y);
+        __nv_bfloat162 t1 = __floats2bfloat162_rn(a4.z, a4.w);
+        uint2 o;
+        o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
+        if (mrow) {
+          // keep an element where its mask value is > 0 (all-ones half-word), clear it otherwise (zero, negative, NaN)
+          o.x &= __hgt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&mk[i].x), zero2);
+          o.y &= __hgt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&mk[i].y), zero2);
+        }
+        *reinterpret_cast<uint2*>(crow + c0 + i * cstep) = o;
+      }
+    }
+    return;
+  }
   if (n0 + half * 32 < p.N) tmem_ld32(tacc + half * 32, r);
 #pragma unroll 1
   for (int c0 = half * 32; c0 < BN; c0 += kChunkStep) {
