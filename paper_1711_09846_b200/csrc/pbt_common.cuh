@@ -140,7 +140,11 @@ __device__ __forceinline__ float adam_one(float w, float& m1, float& m2, float g
   m2 = __fmaf_rn(b2, m2, __fmul_rn(__fmul_rn(omb2, g), g));
   const float mhat = __fmul_rn(m1, inv_bc1);
   const float vhat = __fmul_rn(m2, inv_bc2);
-  const float upd = __fdividef(mhat, __fadd_rn(__fsqrt_rn(vhat), eps));
+  // square root and reciprocal by the special-function unit (relative error about 2^-23 each): the update warps of
+  // the fused kernel are bound by instruction issue, and the correctly rounded forms cost several times as many
+  float root;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(root) : "f"(vhat));
+  const float upd = __fdividef(mhat, __fadd_rn(root, eps));
   return __fmaf_rn(-lrwd, w, __fmaf_rn(-lr, upd, w));
 }
 
