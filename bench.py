@@ -109,8 +109,8 @@ class ClockSampler:
 
 # DRAM bytes per parameter of the fused weight-gradient + Adam kernel, from one `ncu --set full` capture of a
 # small case (profiles/k_wgrad_adam_c5_8members.md), valid for the source file with this sha1 only.
-_NCU_TRAFFIC = {"wgrad_adam": {"bytes_per_param": 25.48, "source": "paper_1711_09846_b200/csrc/wgrad_adam_tcgen05.cu",
-                               "sha1": "8e5c237a7aac9a20bd38b2f8e9693f2484a05f1d"}}
+_NCU_TRAFFIC = {"wgrad_adam": {"bytes_per_param": 25.40, "source": "paper_1711_09846_b200/csrc/wgrad_adam_tcgen05.cu",
+                               "sha1": "1a23ce01242513f201662b9397fbf935bc3d0339"}}
 
 
 def _ncu_traffic(name, params_per_launch):
