@@ -108,9 +108,24 @@ def donor_index(word: int, n_cut: int) -> int:
     return (int(word) * int(n_cut)) >> 32
 
 
-def truncation_select(fitness, seed: int, rnd: int, num: int = 1, den: int = 5) -> np.ndarray:
+def ready_members(step: int, interval: int, offsets=None, n: int = 0) -> np.ndarray:
+    """`ready` of Algorithm 1 for every member at optimisation step `step` (Section 3: enough steps have gone by
+    since the member was last ready).  Member m is ready when step - offsets[m] is a positive multiple of
+    `interval`; with no offsets all members are ready together (the lockstep schedule), with offsets the ready
+    points are staggered as they are when workers run at their own pace."""
+    if offsets is None or len(offsets) == 0:
+        return np.full(n, step > 0 and step % interval == 0, dtype=bool)
+    return np.array([(step - int(o)) > 0 and (step - int(o)) % interval == 0 for o in offsets], dtype=bool)
+
+
+def _is_ready(ready, i) -> bool:
+    return True if ready is None else bool(ready[i])
+
+
+def truncation_select(fitness, seed: int, rnd: int, num: int = 1, den: int = 5, ready=None) -> np.ndarray:
     """Copy map src[N]: src[i] == i for members that keep their state; a bottom
-    member b gets src[b] = a top member drawn uniformly (Section 4.1.1 (b))."""
+    member b gets src[b] = a top member drawn uniformly (Section 4.1.1 (b)).
+    Only members that are `ready` (Algorithm 1; None = all) exploit; the ranking is over the whole population."""
     n = len(fitness)
     src = np.arange(n, dtype=np.int32)
     c = n_cut_of(n, num, den)
@@ -119,12 +134,14 @@ def truncation_select(fitness, seed: int, rnd: int, num: int = 1, den: int = 5) 
     order = rank_members(fitness)
     top, bottom = order[:c], order[n - c:]
     for b in bottom:
+        if not _is_ready(ready, b):
+            continue
         word = px.draw(seed, b, rnd, px.STREAM_EXPLOIT, 0)[0]
         src[b] = top[donor_index(word, c)]
     return src
 
 
-def tournament_select(fitness, seed: int, rnd: int) -> np.ndarray:
+def tournament_select(fitness, seed: int, rnd: int, ready=None) -> np.ndarray:
     """Binary tournament (Section 4.3.1 (b)): every member draws one OTHER member uniformly and copies it if that
     member's score is strictly better (NaN counts as the worst score).  src[i] == i where nothing is copied.
     All decisions use the fitness vector as it stands before any copy."""
@@ -134,6 +151,8 @@ def tournament_select(fitness, seed: int, rnd: int) -> np.ndarray:
         return src
     f = [(-math.inf if math.isnan(float(x)) else float(x)) for x in fitness]
     for i in range(n):
+        if not _is_ready(ready, i):
+            continue
         word = px.draw(seed, i, rnd, px.STREAM_EXPLOIT, 1)[0]
         j = donor_index(word, n - 1)
         if j >= i:
@@ -192,7 +211,7 @@ def ttest_better(hist_self, hist_other, alpha: float) -> bool:
     return bool(p < alpha)
 
 
-def ttest_select(histories, seed: int, rnd: int, alpha: float) -> np.ndarray:
+def ttest_select(histories, seed: int, rnd: int, alpha: float, ready=None) -> np.ndarray:
     """T-test selection (Section 4.1.1, exploit (a)): every member draws one OTHER member uniformly and copies it
     if `ttest_better` holds for the two score histories (oldest first, at most HISTORY entries each).
     src[i] == i where nothing is copied.  All decisions use the histories as they stand before any copy."""
@@ -201,6 +220,8 @@ def ttest_select(histories, seed: int, rnd: int, alpha: float) -> np.ndarray:
     if n < 2:
         return src
     for i in range(n):
+        if not _is_ready(ready, i):
+            continue
         word = px.draw(seed, i, rnd, px.STREAM_EXPLOIT, 2)[0]
         j = donor_index(word, n - 1)
         if j >= i:
@@ -688,15 +709,17 @@ class Population:
         return self.fitness.copy()
 
     # ----- exploit + explore at a ready point ---------------------------------
-    def exploit_explore(self):
+    def exploit_explore(self, ready=None):
+        """One ready point.  `ready[m]` (Algorithm 1: `if ready(p, t, P)`; None = everybody) says which members
+        exploit and explore now; the others keep their record but are ranked and can be copied from."""
         cfg = self.cfg
         rule = getattr(cfg, "exploit", "truncation")
         if rule == "tournament":
-            src = tournament_select(self.fitness, self.seed, self.round)
+            src = tournament_select(self.fitness, self.seed, self.round, ready)
         elif rule == "ttest":
-            src = ttest_select(self.history, self.seed, self.round, cfg.ttest_alpha)
+            src = ttest_select(self.history, self.seed, self.round, cfg.ttest_alpha, ready)
         else:
-            src = truncation_select(self.fitness, self.seed, self.round, cfg.trunc_num, cfg.trunc_den)
+            src = truncation_select(self.fitness, self.seed, self.round, cfg.trunc_num, cfg.trunc_den, ready)
         copied = [b for b in range(self.N) if src[b] != b]
         # every copy reads the donor's record as it was BEFORE this ready point (under the tournament rule a
         # donor may itself be a recipient), so the donors are snapshotted first
@@ -759,13 +782,15 @@ class Population:
     def run(self, total_steps=None, on_ready=None):
         cfg = self.cfg
         total = cfg.total_steps if total_steps is None else total_steps
+        offsets = getattr(cfg, "ready_offsets", ())
         for _ in range(total):
             self.step(1)
-            if self.step_count % cfg.ready_interval == 0:
+            ready = ready_members(self.step_count, cfg.ready_interval, offsets, self.N)
+            if ready.any():
                 self.eval()
                 if on_ready is not None:
                     on_ready(self, "pre")
-                self.exploit_explore()
+                self.exploit_explore(None if ready.all() else ready)
                 if on_ready is not None:
                     on_ready(self, "post")
         return self.best()

@@ -109,3 +109,62 @@ def test_training_reduces_the_loss():
     p.step(30)
     p.eval()
     assert np.mean(p.fitness) > np.mean(before)
+
+
+@pytest.mark.parametrize("name", ["c2_mini_stagger", "c3_mini_stagger_tournament"])
+def test_staggered_ready_points_touch_only_ready_members(name):
+    """Algorithm 1 applies exploit / explore to the member that is ready: at a staggered ready point the record
+    (weights, optimiser state, h, p) of every member that is not ready is bit-unchanged, a ready member either keeps
+    its record or holds a copy of its donor's record as it was before the ready point, and the number of surviving
+    initial lineages never grows (Section 4.4)."""
+    cfg = get_config(name)
+    inp = make_inputs(cfg)
+    pop = O.Population(cfg, inp)
+    lineage = list(range(cfg.n_members))
+    ready_steps = {m: [] for m in range(cfg.n_members)}
+    state = {}
+
+    def on_ready(p, when):
+        nonlocal lineage
+        ready = O.ready_members(p.step_count, cfg.ready_interval, cfg.ready_offsets, p.N)
+        if when == "pre":
+            state["before"] = [p.get_flat(m) for m in range(p.N)]
+            state["H"] = p.H.copy()
+            state["fit"] = p.fitness.copy()
+            return
+        before, n_before = state["before"], len(set(lineage))
+        for m in range(p.N):
+            if ready[m]:
+                ready_steps[m].append(p.step_count)
+            d = int(p.src[m])
+            if not ready[m]:
+                assert d == m
+            now = p.get_flat(m)
+            for key in ("w", "opt1", "opt2", "scalars"):
+                assert np.array_equal(now[key], before[d][key]), (m, key)
+            if d == m:
+                assert np.array_equal(p.H[m], state["H"][m]) and p.fitness[m] == state["fit"][m]
+        lineage = [lineage[int(p.src[m])] for m in range(p.N)]
+        assert len(set(lineage)) <= n_before
+
+    pop.run(on_ready=on_ready)
+    for m in range(cfg.n_members):
+        want = [t for t in range(1, cfg.total_steps + 1)
+                if t > cfg.ready_offsets[m] and (t - cfg.ready_offsets[m]) % cfg.ready_interval == 0]
+        assert ready_steps[m] == want
+
+
+def test_all_ready_mask_is_the_lockstep_ready_point():
+    cfg = get_config("c2_mini")
+    inp = make_inputs(cfg)
+    a, b = O.Population(cfg, inp), O.Population(cfg, inp)
+    for p in (a, b):
+        p.step(2)
+        p.eval()
+    sa = a.exploit_explore()
+    sb = b.exploit_explore(np.ones(cfg.n_members, dtype=bool))
+    assert np.array_equal(sa, sb) and np.array_equal(a.H, b.H) and a.round == b.round
+    # nobody ready: nothing moves, but the ready point is counted (the draws of the next one differ)
+    H0, r0 = a.H.copy(), a.round
+    s = a.exploit_explore(np.zeros(cfg.n_members, dtype=bool))
+    assert np.array_equal(s, np.arange(cfg.n_members)) and np.array_equal(a.H, H0) and a.round == r0 + 1

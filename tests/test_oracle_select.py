@@ -215,3 +215,59 @@ def test_tournament_copies_read_the_state_before_the_ready_point():
                     assert p.H[i, k] in cands
         found = found or bool(chain)
     assert found
+
+
+# ---------------------------------------------------------------------------
+# per-member `ready` (Algorithm 1: `if ready(p, t, P)`): only ready members exploit
+# ---------------------------------------------------------------------------
+def test_ready_mask_truncation_brute_force():
+    """All fitness vectors over {0,1,2}^N, N = 2..5, ALL ready masks: a member copies iff it is ready and in the
+    definitional bottom set; its donor is the one its own draw picks from the definitional top set; a member that is
+    not ready keeps its state even when it ranks last."""
+    for n in range(2, 6):
+        c = O.n_cut_of(n, 2, 5)
+        for f in itertools.product((0.0, 1.0, 2.0), repeat=n):
+            top, bottom = _definitional_sets(f, c)
+            for mask in itertools.product((False, True), repeat=n):
+                src = O.truncation_select(f, seed=11, rnd=1, num=2, den=5, ready=mask)
+                for i in range(n):
+                    if mask[i] and i in bottom:
+                        w = px.draw(11, i, 1, px.STREAM_EXPLOIT, 0)[0]
+                        assert src[i] == top[(w * c) >> 32]
+                    else:
+                        assert src[i] == i
+
+
+def test_ready_mask_tournament_and_ttest():
+    rng = np.random.default_rng(5)
+    n = 9
+    f = rng.standard_normal(n)
+    hist = [list(rng.standard_normal(10) + (3.0 if i % 2 else 0.0)) for i in range(n)]
+    full_t = O.tournament_select(f, 3, 2)
+    full_w = O.ttest_select(hist, 3, 2, 0.05)
+    assert (full_t != np.arange(n)).any() and (full_w != np.arange(n)).any()
+    for mask in itertools.product((False, True), repeat=n):
+        if sum(mask) not in (0, 1, 4, n):
+            continue
+        st = O.tournament_select(f, 3, 2, ready=mask)
+        sw = O.ttest_select(hist, 3, 2, 0.05, ready=mask)
+        for i in range(n):
+            # a ready member decides exactly as it does when everybody is ready; the others keep their state
+            assert st[i] == (full_t[i] if mask[i] else i)
+            assert sw[i] == (full_w[i] if mask[i] else i)
+    assert np.array_equal(O.tournament_select(f, 3, 2, ready=None), full_t)
+
+
+def test_ready_schedule():
+    """Lockstep: everybody at multiples of the interval, never at step 0.  Staggered: each member once per interval,
+    first at offset + interval."""
+    assert not O.ready_members(0, 4, None, 3).any()
+    assert O.ready_members(8, 4, None, 3).all() and not O.ready_members(9, 4, None, 3).any()
+    offs = (0, 1, 3)
+    seen = {m: [] for m in range(3)}
+    for t in range(0, 13):
+        r = O.ready_members(t, 4, offs, 3)
+        for m in range(3):
+            if r[m]:
+                seen[m].append(t)
+    assert seen == {0: [4, 8, 12], 1: [5, 9], 2: [7, 11]}

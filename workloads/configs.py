@@ -84,6 +84,8 @@ class PBTConfig:
     resample_prob: float = 0.25   # probability that a slot is redrawn from its prior (not stated in the paper)
     gp_lambda: float = 10.0       # weight of the gradient penalty (the value of the paper that introduced WGAN-GP)
     ready_interval: int = 1
+    ready_offsets: Tuple[int, ...] = ()   # per member: ready when step - offset is a positive multiple of the interval
+                                          # (empty: everybody together); staggered ready points as under asynchrony
     total_steps: int = 0
     seed: int = 0
 
@@ -198,6 +200,12 @@ CONFIGS: Dict[str, PBTConfig] = {
     # to zero in many bias-gradient sums)
     "c4_mini_wgan_fp32": _c4(n=4, g=(16, 72, 136, 2), d=(2, 136, 72, 1), batch=48, eval_batch=160, pool=512, interval=2,
                              steps=4, name="c4_mini_wgan_fp32").replace(loss=LOSS_WGAN_GP, dtype=FP32, gan_d_steps=1),
+    # staggered ready points (Algorithm 1's per-member `ready`): members exploit at different steps
+    "c2_mini_stagger": _c2(n=6, widths=(40, 72, 56, 1), batch=24, eval_batch=40, pool=512, interval=3, steps=9,
+                           name="c2_mini_stagger").replace(ready_offsets=(0, 1, 2, 0, 1, 2)),
+    "c3_mini_stagger_tournament": _c3(n=6, widths=(72, 136, 200, 10), batch=40, eval_batch=96, pool=640, interval=3, steps=9,
+                                      name="c3_mini_stagger_tournament").replace(ready_offsets=(2, 1, 0, 0, 1, 2),
+                                                                                 exploit="tournament"),
     # t-test selection and resample-from-prior on the same small shapes
     "c2_mini_ttest": _c2(n=7, widths=(40, 72, 56, 1), batch=24, eval_batch=40, pool=512, interval=2, steps=12,
                          name="c2_mini_ttest").replace(exploit="ttest"),
