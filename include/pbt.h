@@ -238,6 +238,16 @@ int pbt_eval(pbt_t* p);
  */
 int pbt_exploit_explore(pbt_t* p);
 
+/*
+ * The same ready point for a population whose members are not all ready together (Algorithm 1 tests
+ * `ready(p, t, P)` member by member; under the asynchronous execution of Section 3 the ready points of the
+ * workers are staggered).  ready_host: n_members bytes of host memory, non-zero = this member is ready and may
+ * exploit and explore now; NULL = everybody (pbt_exploit_explore).  Members that are not ready keep their whole
+ * record, but they are ranked with the others and can be copied from.  The ready-point counter advances by
+ * one per call whatever the mask, so the random draws of successive calls differ.
+ */
+int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host);
+
 /* Read / overwrite one member's record.  get synchronises the stream. */
 int pbt_get_state(pbt_t* p, int member, pbt_state_view* out_host);
 int pbt_set_state(pbt_t* p, int member, const pbt_state_view* in_host);

@@ -77,7 +77,7 @@ class PbtGemmDesc(C.Structure):
 
 EXPORTS = [
     "pbt_query_workspace", "pbt_param_count", "pbt_create", "pbt_destroy", "pbt_step", "pbt_eval",
-    "pbt_exploit_explore", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
+    "pbt_exploit_explore", "pbt_exploit_explore_ready", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
     "pbt_get_history", "pbt_set_history",
     "pbt_get_hparams", "pbt_set_hparams", "pbt_get_copy_map", "pbt_get_best", "pbt_get_last_loss",
     "pbt_set_batch", "pbt_step_host", "pbt_prefetch_host_batch", "pbt_step_prefetched", "pbt_get_launch_count", "pbt_profile_begin", "pbt_profile_end", "pbt_profile_get",
@@ -110,6 +110,7 @@ def load_library() -> C.CDLL:
     lib.pbt_step.argtypes = [vp, C.c_int]
     lib.pbt_eval.argtypes = [vp]
     lib.pbt_exploit_explore.argtypes = [vp]
+    lib.pbt_exploit_explore_ready.argtypes = [vp, C.POINTER(C.c_uint8)]
     lib.pbt_get_state.argtypes = [vp, C.c_int, C.POINTER(PbtStateView)]
     lib.pbt_set_state.argtypes = [vp, C.c_int, C.POINTER(PbtStateView)]
     lib.pbt_get_fitness.argtypes = [vp, C.POINTER(C.c_double)]
@@ -335,8 +336,14 @@ class Population:
     def eval(self):
         self._check(self.lib.pbt_eval(self.handle))
 
-    def exploit_explore(self):
-        self._check(self.lib.pbt_exploit_explore(self.handle))
+    def exploit_explore(self, ready=None):
+        """One ready point; `ready` (bools, one per member; None = everybody) says which members may exploit now."""
+        if ready is None:
+            self._check(self.lib.pbt_exploit_explore(self.handle))
+            return
+        mask = np.ascontiguousarray(np.asarray(ready, dtype=bool).astype(np.uint8))
+        assert mask.shape == (self.cfg.n_members,)
+        self._check(self.lib.pbt_exploit_explore_ready(self.handle, mask.ctypes.data_as(C.POINTER(C.c_uint8))))
 
     # ----- state access ---------------------------------------------------
     def get_state(self, m: int) -> Dict[str, np.ndarray]:
@@ -491,6 +498,21 @@ class Population:
         cfg = self.cfg
         total = cfg.total_steps if total_steps is None else total_steps
         done = 0
+        offsets = tuple(getattr(cfg, "ready_offsets", ()))
+        if offsets:
+            # staggered ready points (Algorithm 1's `ready`, member by member): member m is ready when
+            # step - offsets[m] is a positive multiple of the interval; run to the next step at which anybody is
+            iv = cfg.ready_interval
+            while done < total:
+                nxt = min(o + iv * ((done - o) // iv + 1) if done >= o else o + iv for o in offsets)
+                k = min(nxt, total) - done
+                self.step(k)
+                done += k
+                ready = [(done - o) > 0 and (done - o) % iv == 0 for o in offsets]
+                if any(ready):
+                    self.eval()
+                    self.exploit_explore(None if all(ready) else ready)
+            return self.best()
         while done < total:
             k = min(cfg.ready_interval, total - done)
             self.step(k)

@@ -929,12 +929,16 @@ int pbt_eval(pbt_t* p) {
   return record_scores(p);
 }
 
-int pbt_exploit_explore(pbt_t* p) {
+int pbt_exploit_explore(pbt_t* p) { return pbt_exploit_explore_ready(p, nullptr); }
+
+int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host) {
   if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
   p->launches = 0;
   const pbt_spec& s = p->spec;
   SelectArgs a;
   memset(&a, 0, sizeof(a));
+  for (int i = 0; i < p->N; ++i)
+    if (!ready_host || ready_host[i]) a.ready_bits[i >> 5] |= 1u << (i & 31);
   a.n = p->N; a.nh = p->nh;
   int n_cut = 0;
   if (p->N >= 2) {

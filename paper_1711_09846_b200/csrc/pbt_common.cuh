@@ -167,6 +167,7 @@ struct SelectArgs {
   double prior_a[PBT_MAX_NH], prior_b[PBT_MAX_NH];   // uniform: lo, hi; log-uniform: log lo, log hi
   Counters* counters;
   uint64_t seed;
+  uint32_t ready_bits[32];          // bit i set: member i is ready (Algorithm 1) and may exploit at this ready point
   uint32_t perturb_mask, flags;
   double factor_lo, factor_hi;
   double clamp_lo[PBT_MAX_NH], clamp_hi[PBT_MAX_NH];

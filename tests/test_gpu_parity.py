@@ -179,6 +179,75 @@ def test_flag_variants_bit_exact(pkg, flags):
     gpu.close()
 
 
+@pytest.mark.parametrize("rule", ["truncation", "tournament", "ttest"])
+@pytest.mark.parametrize("n", [2, 5, 33, 80, 200])
+def test_ready_mask_bit_exact(pkg, n, rule):
+    """Algorithm 1's per-member `ready`: with a mask only ready members copy and explore; copy map, copied records,
+    hyperparameters, fitness and (t-test) score histories against the oracle, bit for bit, for random masks, the
+    empty mask and the full mask."""
+    cfg = _tiny_cfg(n, C.FP32).replace(exploit=rule)
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    rng = np.random.default_rng(100 + n)
+    gpu.step(1)
+    cpu.step(1)
+    push_oracle_state(gpu, cpu)
+    masks = [rng.random(n) < 0.5, np.zeros(n, dtype=bool), rng.random(n) < 0.2, np.ones(n, dtype=bool), rng.random(n) < 0.8]
+    for rnd, mask in enumerate(masks):
+        f = rng.standard_normal(n).astype(np.float32)
+        cpu.fitness[:] = f
+        gpu.set_fitness(f.astype(np.float64))
+        if rule == "ttest":
+            for m in range(n):
+                cnt = int(rng.integers(0, 11))
+                cpu.history[m] = [np.float32(x) for x in rng.standard_normal(cnt) + (2.0 if m % 3 == 0 else 0.0)]
+            ch, cc = oracle_history_arrays(cpu)
+            gpu.set_history(ch, cc)
+        before = [gpu.get_state(m) for m in range(n)]
+        h_before = gpu.hparams()
+        gpu.exploit_explore(mask)
+        src = cpu.exploit_explore(mask)
+        assert np.array_equal(gpu.copy_map(), src)
+        assert all(src[m] == m for m in range(n) if not mask[m])
+        assert np.array_equal(gpu.hparams(), cpu.H.astype(np.float64))
+        assert np.array_equal(gpu.fitness(), cpu.fitness.astype(np.float64))
+        if rule == "ttest":
+            (gh, gc), (ch, cc) = gpu.history(), oracle_history_arrays(cpu)
+            assert np.array_equal(gc, cc) and np.array_equal(gh, ch)
+        for m in range(n):
+            now = gpu.get_state(m)
+            assert now["round"] == cpu.round
+            for key in ("w", "opt1", "opt2", "scalars"):
+                assert np.array_equal(now[key], before[int(src[m])][key]), (rnd, m, key)
+            if not mask[m]:
+                assert np.array_equal(gpu.hparams()[m], h_before[m])
+    gpu.close()
+
+
+def test_staggered_run_matches_the_oracle_schedule(pkg):
+    """Population.run with staggered ready points: the host schedule (which members are ready at which step) is the
+    binding's own; the copy maps it produces must be the oracle's when both see the same fitness."""
+    cfg = get_config("c2_mini_stagger")
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    seen = []
+    orig = gpu.exploit_explore
+
+    def spy(ready=None):
+        seen.append((None if ready is None else tuple(bool(r) for r in ready)))
+        orig(ready)
+    gpu.exploit_explore = spy
+    gpu.run()
+    want = []
+    for t in range(1, cfg.total_steps + 1):
+        r = O.ready_members(t, cfg.ready_interval, cfg.ready_offsets, cfg.n_members)
+        if r.any():
+            want.append(None if r.all() else tuple(bool(x) for x in r))
+    assert seen == want
+    assert gpu.get_state(0)["step"] == cfg.total_steps and gpu.get_state(0)["round"] == len(want)
+    gpu.close()
+
+
 # ---------------------------------------------------------------------------
 # initial population
 # ---------------------------------------------------------------------------
@@ -227,7 +296,7 @@ def _check_optimizer_arithmetic(cfg, s0, s1, h):
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("name", ["c2_mini", "c3_mini", "c4_mini", "c5_mini", "c3_mid", "c5_mid", "c4_mid", "c2_mini_rms",
                                   "c3_mini_rms", "c2_mini_ttest", "c3_mini_resample", "c4_mini_wgan", "c4_mini_wgan_fp32",
-                                  "c4_mid_wgan"])
+                                  "c4_mid_wgan", "c2_mini_stagger", "c3_mini_stagger_tournament"])
 def test_step_eval_exploit_parity(pkg, name):
     cfg = get_config(name)
     inp = make_inputs(cfg)
@@ -254,7 +323,9 @@ def test_step_eval_exploit_parity(pkg, name):
             got[0] += critic_offset(cfg, g)
             want[0] += critic_offset(cfg, c)
             np.testing.assert_allclose(got, want, rtol=ftol, atol=1e-5)
-        if t % cfg.ready_interval == 0:
+        ready = O.ready_members(t, cfg.ready_interval, cfg.ready_offsets, cfg.n_members)
+        if ready.any():
+            mask = None if ready.all() else ready
             gpu.eval()
             cpu.eval()
             np.testing.assert_allclose(gpu.fitness(), cpu.fitness, rtol=ftol, atol=2e-5)
@@ -265,8 +336,8 @@ def test_step_eval_exploit_parity(pkg, name):
                 assert np.array_equal(gc, cc)
                 np.testing.assert_allclose(gh[:, -1 if cc[0] == 10 else cc[0] - 1], cpu.fitness, rtol=ftol, atol=2e-5)
                 gpu.set_history(ch, cc)
-            gpu.exploit_explore()
-            src = cpu.exploit_explore()
+            gpu.exploit_explore(mask)
+            src = cpu.exploit_explore(mask)
             assert np.array_equal(gpu.copy_map(), src)
             assert np.array_equal(gpu.hparams(), cpu.H.astype(np.float64))
             if cfg.exploit == "ttest":
