@@ -494,7 +494,32 @@ class Population:
         return out
 
     # ----- Algorithm 1 in partial synchrony ---------------------------------
-    def run(self, total_steps: Optional[int] = None) -> int:
+    def _ready_point(self, step, ready, log):
+        """eval, exploit / explore and, if asked, one record of the ready point (Section 4.4's analyses are made
+        from such records: score and hyperparameter traces, who copied whom)."""
+        self.eval()
+        if log is None:
+            self.exploit_explore(ready)
+            return
+        rec = {"step": step, "ready": None if ready is None else [bool(r) for r in ready],
+               "fitness": self.fitness(), "hparams_before": self.hparams()}
+        self.exploit_explore(ready)
+        rec["src"] = self.copy_map()
+        rec["hparams_after"] = self.hparams()
+        log.append(rec)
+
+    @staticmethod
+    def ancestors(log, n_members):
+        """Initial member each current member descends from, following the copy maps of a ready-point log."""
+        anc = list(range(n_members))
+        for rec in log:
+            anc = [anc[int(d)] for d in rec["src"]]
+        return anc
+
+    def run(self, total_steps: Optional[int] = None, log=None) -> int:
+        """Algorithm 1 in partial synchrony: steps, and a ready point whenever `ready` holds.  `log`: a list (or a
+        bounded collections.deque) that receives one record per ready point; each record costs four small
+        device-to-host reads."""
         cfg = self.cfg
         total = cfg.total_steps if total_steps is None else total_steps
         done = 0
@@ -510,14 +535,12 @@ class Population:
                 done += k
                 ready = [(done - o) > 0 and (done - o) % iv == 0 for o in offsets]
                 if any(ready):
-                    self.eval()
-                    self.exploit_explore(None if all(ready) else ready)
+                    self._ready_point(done, None if all(ready) else ready, log)
             return self.best()
         while done < total:
             k = min(cfg.ready_interval, total - done)
             self.step(k)
             done += k
             if done % cfg.ready_interval == 0:
-                self.eval()
-                self.exploit_explore()
+                self._ready_point(done, None, log)
         return self.best()

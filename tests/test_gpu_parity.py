@@ -248,6 +248,30 @@ def test_staggered_run_matches_the_oracle_schedule(pkg):
     gpu.close()
 
 
+def test_ready_point_log_and_lineages(pkg):
+    """The ready-point records of a run: one per ready point, copy maps consistent with the hyperparameter traces
+    (only members that copied change h), and the number of surviving initial lineages never grows (Section 4.4)."""
+    cfg = get_config("c3_mini").replace(total_steps=12)
+    inp = make_inputs(cfg)
+    gpu = pkg.Population(cfg, inp)
+    log = []
+    gpu.run(log=log)
+    assert [r["step"] for r in log] == list(range(cfg.ready_interval, 13, cfg.ready_interval))
+    alive = cfg.n_members
+    for k, rec in enumerate(log):
+        n_cut = O.n_cut_of(cfg.n_members, cfg.trunc_num, cfg.trunc_den)
+        assert np.array_equal(rec["src"], O.truncation_select(rec["fitness"].astype(np.float32), cfg.seed, k,
+                                                              cfg.trunc_num, cfg.trunc_den))
+        assert (rec["src"] != np.arange(cfg.n_members)).sum() == n_cut
+        for m in range(cfg.n_members):
+            if rec["src"][m] == m:
+                assert np.array_equal(rec["hparams_after"][m], rec["hparams_before"][m])
+        now = len(set(pkg.Population.ancestors(log[:k + 1], cfg.n_members)))
+        assert now <= alive
+        alive = now
+    gpu.close()
+
+
 # ---------------------------------------------------------------------------
 # initial population
 # ---------------------------------------------------------------------------
