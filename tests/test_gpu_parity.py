@@ -180,7 +180,7 @@ def test_flag_variants_bit_exact(pkg, flags):
 
 
 @pytest.mark.parametrize("rule", ["truncation", "tournament", "ttest"])
-@pytest.mark.parametrize("n", [2, 5, 33, 80, 200])
+@pytest.mark.parametrize("n", [2, 5, 33, 80, 200, 1024])
 def test_ready_mask_bit_exact(pkg, n, rule):
     """Algorithm 1's per-member `ready`: with a mask only ready members copy and explore; copy map, copied records,
     hyperparameters, fitness and (t-test) score histories against the oracle, bit for bit, for random masks, the
