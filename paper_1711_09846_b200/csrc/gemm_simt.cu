@@ -202,21 +202,34 @@ __global__ void __launch_bounds__(512) k_gemm_colacc(GemmArgs g) {
   }
 }
 
-// K <= 16: every output element is a short dot product; block = 256 consecutive n of one row m.
+// K <= 16: every output element is a short dot product.  A thread owns one column n: it keeps B(n, 0..K-1) in
+// registers and walks kSmallKRows rows of A, whose values every thread of the block reads alike (broadcast).
+constexpr int kSmallKRows = 32;
 template <typename T>
 __global__ void __launch_bounds__(256) k_gemm_smallk(GemmArgs g) {
-  const int member = blockIdx.z, m = blockIdx.y;
+  const int member = blockIdx.z, m0 = blockIdx.y * kSmallKRows;
   const int n = blockIdx.x * 256 + threadIdx.x;
-  if (n >= g.N) return;
+  __shared__ float As[kSmallKRows][kSkinny];
   const T* __restrict__ A = reinterpret_cast<const T*>(g.A) + member * g.strideA;
   const T* __restrict__ B = reinterpret_cast<const T*>(g.B) + member * g.strideB;
-  float v = 0.f;
-  for (int k = 0; k < g.K; ++k) {
-    const float a = to_f<T>(g.a_mn ? A[(long long)k * g.lda + m] : A[(long long)m * g.lda + k]);
-    const float b = to_f<T>(g.b_mn ? B[(long long)k * g.ldb + n] : B[(long long)n * g.ldb + k]);
-    v = fmaf(a, b, v);
+  for (int i = threadIdx.x; i < kSmallKRows * g.K; i += 256) {
+    const int r = i / g.K, k = i % g.K, m = m0 + r;
+    As[r][k] = m < g.M ? to_f<T>(g.a_mn ? A[(long long)k * g.lda + m] : A[(long long)m * g.lda + k]) : 0.f;
   }
-  store_one(g, member, m, n, epilogue_one(g, member, m, n, v, sizeof(T) == 2));
+  __syncthreads();
+  if (n >= g.N) return;
+  float b[kSkinny];
+#pragma unroll
+  for (int k = 0; k < kSkinny; ++k)
+    b[k] = k < g.K ? to_f<T>(g.b_mn ? B[(long long)k * g.ldb + n] : B[(long long)n * g.ldb + k]) : 0.f;
+  const int rows = min(kSmallKRows, g.M - m0);
+  for (int r = 0; r < rows; ++r) {
+    float v = 0.f;
+#pragma unroll
+    for (int k = 0; k < kSkinny; ++k)
+      if (k < g.K) v = fmaf(As[r][k], b[k], v);
+    store_one(g, member, m0 + r, n, epilogue_one(g, member, m0 + r, n, v, sizeof(T) == 2));
+  }
 }
 
 template <typename T, bool B_MN>
@@ -241,8 +254,8 @@ static void launch_colacc(const GemmArgs& g, cudaStream_t s) {
 
 template <typename T>
 static bool launch_skinny(const GemmArgs& g, cudaStream_t s) {
-  if (g.K <= kSkinny && g.K > 0 && g.M <= 65535 && g.batch <= 65535) {
-    k_gemm_smallk<T><<<dim3((g.N + 255) / 256, g.M, g.batch), 256, 0, s>>>(g);
+  if (g.K <= kSkinny && g.K > 0 && (g.M + kSmallKRows - 1) / kSmallKRows <= 65535 && g.batch <= 65535) {
+    k_gemm_smallk<T><<<dim3((g.N + 255) / 256, (g.M + kSmallKRows - 1) / kSmallKRows, g.batch), 256, 0, s>>>(g);
     return true;
   }
   if (g.N <= kSkinny && !g.a_mn) {

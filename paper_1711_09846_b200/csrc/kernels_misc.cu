@@ -402,7 +402,9 @@ __global__ void __launch_bounds__(256) k_bias_grad_bf16x8(const bf16* __restrict
 
 cudaError_t launch_bias_grad(const void* dz, int dz_dtype, long long ld, long long stride, int rows, int cols,
                              float* out, long long out_stride, int n_members, cudaStream_t s) {
-  if (dz_dtype == kBF16 && cols % 8 == 0 && cols >= 256 && ld % 8 == 0 && stride % 8 == 0 && ((uintptr_t)dz & 15) == 0) {
+  // the wide kernel has one block per 256 columns and member: only when that fills the GPU twice over
+  if (dz_dtype == kBF16 && cols % 8 == 0 && (long long)((cols + 255) / 256) * n_members >= 296 && ld % 8 == 0 &&
+      stride % 8 == 0 && ((uintptr_t)dz & 15) == 0) {
     dim3 grid((cols + 255) / 256, n_members);
     k_bias_grad_bf16x8<<<grid, 256, 0, s>>>((const bf16*)dz, ld, stride, rows, cols, out, out_stride);
     return cudaGetLastError();
