@@ -232,6 +232,83 @@ __global__ void __launch_bounds__(256) k_gemm_smallk(GemmArgs g) {
   }
 }
 
+// The same for bf16 operands and output with K <= 4 and N a multiple of 8: a thread produces 8 consecutive columns
+// of a row (16-byte loads of the weights and of the ReLU mask, one 16-byte store), the block's threads are spread
+// over the 32 rows x N / 8 column groups of its slab.  Same multiply-add order per element as the kernel above.
+template <bool B_MN>
+__global__ void __launch_bounds__(256) k_gemm_smallk_bf16x8(GemmArgs g) {
+  constexpr int KV = 4;
+  const int member = blockIdx.z, m0 = blockIdx.y * kSmallKRows;
+  __shared__ float As[kSmallKRows][KV];
+  const bf16* __restrict__ A = reinterpret_cast<const bf16*>(g.A) + member * g.strideA;
+  const bf16* __restrict__ B = reinterpret_cast<const bf16*>(g.B) + member * g.strideB;
+  for (int i = threadIdx.x; i < kSmallKRows * KV; i += 256) {
+    const int r = i / KV, k = i % KV, m = m0 + r;
+    As[r][k] = (m < g.M && k < g.K) ? __bfloat162float(g.a_mn ? A[(long long)k * g.lda + m] : A[(long long)m * g.lda + k]) : 0.f;
+  }
+  __syncthreads();
+  const int groups = g.N >> 3;
+  const int rows = min(kSmallKRows, g.M - m0);
+  const float* bias = g.bias ? g.bias + member * g.strideBias : nullptr;
+  const bf16* mask = g.mask ? reinterpret_cast<const bf16*>(g.mask) + member * g.strideMask : nullptr;
+  bf16* C = reinterpret_cast<bf16*>(g.C) + member * g.strideC;
+  const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
+#pragma unroll 2
+  for (int idx = blockIdx.x * 256 + threadIdx.x; idx < rows * groups; idx += gridDim.x * 256) {
+    const int r = idx / groups, n = (idx % groups) << 3;
+    const int m = m0 + r;
+    float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int k = 0; k < KV; ++k) {
+      if (k < g.K) {
+        float b[8];
+        if (B_MN) {
+          const uint4 w = __ldg(reinterpret_cast<const uint4*>(B + (long long)k * g.ldb + n));
+          const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) { b[2 * j] = __uint_as_float(u[j] << 16); b[2 * j + 1] = __uint_as_float(u[j] & 0xFFFF0000u); }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) b[j] = __bfloat162float(B[(long long)(n + j) * g.ldb + k]);
+        }
+        const float a = As[r][k];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = fmaf(a, b[j], v[j]);
+      }
+    }
+    if (bias) {
+      const float4 b0 = __ldg(reinterpret_cast<const float4*>(bias + n)), b1 = __ldg(reinterpret_cast<const float4*>(bias + n + 4));
+      v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w; v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+    }
+    if (g.relu) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = fmaxf(v[j], 0.f);
+    }
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      __nv_bfloat162 t = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+      o[j] = *reinterpret_cast<uint32_t*>(&t);
+    }
+    if (mask) {
+      const uint4 mk = __ldg(reinterpret_cast<const uint4*>(mask + (long long)m * g.ldmask + n));
+      const uint32_t mu[4] = {mk.x, mk.y, mk.z, mk.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) o[j] &= __hgt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&mu[j]), zero2);
+    }
+    *reinterpret_cast<uint4*>(C + (long long)m * g.ldc + n) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+static bool smallk_vec_ok(const GemmArgs& g) {
+  if (g.in_dtype != kBF16 || g.out_dtype != kBF16 || g.K < 1 || g.K > 4 || g.N % 8 != 0) return false;
+  if (g.ldc % 8 || g.strideC % 8 || ((uintptr_t)g.C & 15)) return false;
+  if (g.b_mn && (g.ldb % 8 || g.strideB % 8 || ((uintptr_t)g.B & 15))) return false;
+  if (g.mask && (g.ldmask % 8 || g.strideMask % 8 || ((uintptr_t)g.mask & 15))) return false;
+  if (g.bias && (g.strideBias % 4 || ((uintptr_t)g.bias & 15))) return false;
+  return (g.M + kSmallKRows - 1) / kSmallKRows <= 65535 && g.batch <= 65535;
+}
+
 template <typename T, bool B_MN>
 static void launch_rowdot(const GemmArgs& g, cudaStream_t s) {
   dim3 grid((g.M + 7) / 8, g.batch);
@@ -254,6 +331,13 @@ static void launch_colacc(const GemmArgs& g, cudaStream_t s) {
 
 template <typename T>
 static bool launch_skinny(const GemmArgs& g, cudaStream_t s) {
+  if (smallk_vec_ok(g)) {
+    const int per_slab = kSmallKRows * (g.N / 8);
+    const dim3 grid((per_slab + 255) / 256 > 8 ? 8 : (per_slab + 255) / 256, (g.M + kSmallKRows - 1) / kSmallKRows, g.batch);
+    if (g.b_mn) k_gemm_smallk_bf16x8<true><<<grid, 256, 0, s>>>(g);
+    else k_gemm_smallk_bf16x8<false><<<grid, 256, 0, s>>>(g);
+    return true;
+  }
   if (g.K <= kSkinny && g.K > 0 && (g.M + kSmallKRows - 1) / kSmallKRows <= 65535 && g.batch <= 65535) {
     k_gemm_smallk<T><<<dim3((g.N + 255) / 256, (g.M + kSmallKRows - 1) / kSmallKRows, g.batch), 256, 0, s>>>(g);
     return true;
