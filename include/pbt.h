@@ -354,6 +354,18 @@ typedef struct pbt_gemm_desc {
 int pbt_grouped_gemm(const pbt_gemm_desc* desc, void* stream);
 
 /*
+ * Failure-detection self-test.  Every wait inside the tensor-core kernels (on a TMA transfer, an MMA commit, a
+ * partner CTA) is bounded: when its poll limit runs out the kernel stores PBT_ERR_TIMEOUT in the status word, every
+ * role leaves its loop, and the kernel returns normally, so the context stays usable and the next pbt_get_* call
+ * reports the error (a population's workers being lost or pre-empted is part of the paper's setting, Appendix A.1;
+ * here the only thing that can go missing is a signal inside a kernel).  This call runs that same wait in a
+ * one-CTA kernel on a barrier that nothing signals, with `polls` polls (1..100000; a few thousand last well under
+ * a second), so the expiry path can be exercised without provoking a fault: afterwards the int32 at byte offset 16
+ * of status_device (32 zeroed bytes of device memory, as for pbt_grouped_gemm) holds PBT_ERR_TIMEOUT.
+ */
+int pbt_selftest_bounded_wait(void* status_device, int polls, void* stream);
+
+/*
  * Allocation-free scorer (no counterpart in the paper: it exists for callers that are not
  * allowed to allocate device memory, e.g. a plug-in inside an application that owns the
  * whole device through its own arena, and so cannot provide the workspace pbt_create wants).

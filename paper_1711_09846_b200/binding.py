@@ -81,7 +81,7 @@ EXPORTS = [
     "pbt_get_history", "pbt_set_history",
     "pbt_get_hparams", "pbt_set_hparams", "pbt_get_copy_map", "pbt_get_best", "pbt_get_last_loss",
     "pbt_set_batch", "pbt_step_host", "pbt_prefetch_host_batch", "pbt_step_prefetched", "pbt_get_launch_count", "pbt_profile_begin", "pbt_profile_end", "pbt_profile_get",
-    "pbt_grouped_gemm", "pbt_energy_fitness_static", "pbt_last_error",
+    "pbt_grouped_gemm", "pbt_selftest_bounded_wait", "pbt_energy_fitness_static", "pbt_last_error",
 ]
 
 _LIB = None
@@ -130,6 +130,7 @@ def load_library() -> C.CDLL:
     lib.pbt_profile_get.argtypes = [vp, C.c_char_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.pbt_grouped_gemm.argtypes = [C.POINTER(PbtGemmDesc), vp]
     lib.pbt_energy_fitness_static.argtypes = [vp, C.c_int, C.c_int, vp, vp]
+    lib.pbt_selftest_bounded_wait.argtypes = [vp, C.c_int, vp]
     lib.pbt_last_error.argtypes = [vp]
     lib.pbt_last_error.restype = C.c_char_p
     for name in EXPORTS:
@@ -231,6 +232,16 @@ def grouped_gemm(A, B, C_out, a_mn=False, b_mn=False, bias=None, relu=False, mas
     if status is not None:
         d.status_device = status.data_ptr()
     rc = lib.pbt_grouped_gemm(C.byref(d), C.c_void_p(stream.cuda_stream if stream is not None else None))
+    if rc:
+        raise PbtError(rc, lib.pbt_last_error(None).decode())
+
+
+def selftest_bounded_wait(status, polls: int = 2000, stream=None) -> None:
+    """Run the kernels' bounded barrier wait on a barrier nothing signals (see pbt_selftest_bounded_wait);
+    status: >= 8 zeroed int32 on the device, status[4] becomes PBT_ERR_TIMEOUT."""
+    lib = load_library()
+    rc = lib.pbt_selftest_bounded_wait(C.c_void_p(status.data_ptr()), int(polls),
+                                       C.c_void_p(stream.cuda_stream if stream is not None else None))
     if rc:
         raise PbtError(rc, lib.pbt_last_error(None).decode())
 

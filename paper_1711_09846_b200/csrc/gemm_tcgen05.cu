@@ -206,6 +206,30 @@ cudaError_t launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, TcParams&
 
 }  // namespace
 
+// Self-test of the bounded wait every tensor-core kernel relies on: one CTA waits on a barrier that nothing ever
+// signals; when the limit runs out it records PBT_ERR_TIMEOUT like the real kernels do and returns normally.
+__global__ void k_selftest_bounded_wait(Counters* counters, uint32_t limit) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (!mbar_wait(&bar, 0, &abort_flag, limit)) {
+      atomicCAS(&counters->status, 0, PBT_ERR_TIMEOUT);
+      counters->status_info = 99;
+    }
+  }
+}
+
+cudaError_t launch_selftest_bounded_wait(Counters* counters, uint32_t limit, cudaStream_t s) {
+  k_selftest_bounded_wait<<<1, 32, 0, s>>>(counters, limit);
+  return cudaGetLastError();
+}
+
 bool gemm_tc_supported(const GemmArgs& g) {
   if (g.in_dtype != kBF16) return false;
   if (g.M < 128 || g.N < 128 || g.K < 64 || g.batch < 1) return false;  // every TMA box fits inside its tensor

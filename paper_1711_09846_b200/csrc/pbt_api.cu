@@ -1352,6 +1352,14 @@ int pbt_grouped_gemm(const pbt_gemm_desc* d, void* stream) {
   return PBT_OK;
 }
 
+int pbt_selftest_bounded_wait(void* status_device, int polls, void* stream) {
+  if (!status_device) return fail(nullptr, PBT_ERR_INVALID_ARG, "status_device is NULL");
+  if (polls < 1 || polls > 100000) return fail(nullptr, PBT_ERR_INVALID_ARG, "polls must lie in [1, 100000]");
+  cudaError_t e = launch_selftest_bounded_wait((Counters*)status_device, (uint32_t)polls, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail(nullptr, PBT_ERR_CUDA, "self-test launch: %s", cudaGetErrorString(e));
+  return PBT_OK;
+}
+
 int pbt_get_launch_count(const pbt_t* p, int64_t* count) {
   if (!p || !count) return fail(nullptr, PBT_ERR_INVALID_ARG, "NULL argument");
   *count = p->launches;

@@ -84,6 +84,8 @@ cudaError_t launch_gemm_simt(const GemmArgs& g, cudaStream_t s);
 // tensor-core path; returns cudaErrorNotSupported when the shape does not qualify
 bool gemm_tc_supported(const GemmArgs& g);
 cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s);
+// one CTA runs the kernels' bounded barrier wait on a barrier nobody signals, with `limit` polls
+cudaError_t launch_selftest_bounded_wait(Counters* counters, uint32_t limit, cudaStream_t s);
 // CTA-pair variant (256 x 256 tiles shared by two CTAs of a cluster) for shapes with M, N >= 256
 bool gemm_tc_pair_supported(const GemmArgs& g);
 cudaError_t launch_gemm_tc_pair(const GemmArgs& g, Counters* counters, cudaStream_t s);

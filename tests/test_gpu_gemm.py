@@ -132,3 +132,17 @@ def test_tensor_core_cta_pairs_many_tiles(env):
     # 2 x 4 x 12 = 96 pair tiles on 74 CTA pairs: the persistent loop and both accumulator buffers cycle
     _run(pkg, torch, 512, 1024, 256, 12, False, False, engine=3, epilogue="bias_relu", out_bf16=True, seed=19)
     _run(pkg, torch, 512, 1024, 256, 12, False, True, engine=3, epilogue="mask", out_bf16=True, seed=20)
+
+
+def test_bounded_wait_expires_with_a_status_and_leaves_the_context_usable(env):
+    """Failure detection without a fault: the kernels' bounded barrier wait, run on a barrier that nothing
+    signals, gives up after its poll limit, reports PBT_ERR_TIMEOUT through the status word and returns; the
+    next kernels on the same stream run normally."""
+    pkg, torch = env
+    status = torch.zeros(8, dtype=torch.int32, device="cuda")
+    pkg.selftest_bounded_wait(status, polls=2000)
+    torch.cuda.synchronize()
+    assert int(status[4]) == 5 and int(status[5]) == 99          # PBT_ERR_TIMEOUT, recorded by the self-test
+    with pytest.raises(pkg.PbtError):
+        pkg.selftest_bounded_wait(status, polls=0)
+    _run(pkg, torch, 256, 256, 128, 2, False, False, engine=2, epilogue="bias_relu", out_bf16=True)
