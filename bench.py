@@ -393,7 +393,9 @@ def main():
     def add(name, bound, amount, unit, peak, src):
         if prof[name]["launches"] and amount > 0:
             ach = amount * args.steps / (prof[name]["ms"] * 1e-3) / (1e12 if unit == "TFLOP/s" else 1e9)
-            kern[name] = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak, "traffic": None,
+            nominal = {"TFLOP/s": 2250.0 if bound == "tensor" else None, "GB/s": 8000.0}[unit]
+            kern[name] = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                          "frac_of_nominal": (ach / nominal) if nominal else None, "nominal_peak": nominal, "traffic": None,
                           "ms_per_step": prof[name]["ms"] / args.steps,
                           "launches_per_step": prof[name]["launches"] / args.steps, "peak_source": src}
 
