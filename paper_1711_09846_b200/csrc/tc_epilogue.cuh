@@ -37,6 +37,32 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, float* buf, uin
   // checks, pointers advanced by constant steps and the ReLU mask applied to the packed bf16 pairs: the epilogue
   // warps are bound by instruction issue, two warps per scheduler, so the instruction count per element is what
   // decides whether the epilogue hides behind a short main loop.
+  if (vec_ok && p.out_dtype != kBF16 && !p.mask && m0 + kBM <= p.M && n0 + BN <= p.N) {
+    // the same for fp32 output without a mask (logits, stored weight gradients)
+    float* crow = reinterpret_cast<float*>(p.C) + member * p.strideC + (long long)(m0 + q * 32 + rsub) * p.ldc + n0 + cc;
+    const long long cstep = 4 * p.ldc;
+    tmem_ld32(tacc + half * 32, r);
+#pragma unroll 1
+    for (int c0 = half * 32; c0 < BN; c0 += kChunkStep) {
+      tmem_ld_wait();
+      __syncwarp();
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        *reinterpret_cast<uint4*>(&buf[lane * kEpiPitch + j * 4]) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+      if (c0 + kChunkStep < BN) tmem_ld32(tacc + c0 + kChunkStep, r);
+      __syncwarp();
+      float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (bias) bv = __ldg(reinterpret_cast<const float4*>(bias + n0 + c0 + cc));
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float4 a4 = *reinterpret_cast<const float4*>(&buf[(i * 4 + rsub) * kEpiPitch + cc]);
+        if (bias) { a4.x += bv.x; a4.y += bv.y; a4.z += bv.z; a4.w += bv.w; }
+        if (p.relu) { a4.x = fmaxf(a4.x, 0.f); a4.y = fmaxf(a4.y, 0.f); a4.z = fmaxf(a4.z, 0.f); a4.w = fmaxf(a4.w, 0.f); }
+        *reinterpret_cast<float4*>(crow + c0 + i * cstep) = a4;
+      }
+    }
+    return;
+  }
   if (vec_ok && p.out_dtype == kBF16 && m0 + kBM <= p.M && n0 + BN <= p.N) {
     const long long row0 = m0 + q * 32 + rsub;
     bf16* crow = reinterpret_cast<bf16*>(p.C) + member * p.strideC + row0 * p.ldc + n0 + cc;
