@@ -505,6 +505,40 @@ class Population:
         return out
 
     # ----- Algorithm 1 in partial synchrony ---------------------------------
+    # ----- checkpoint / resume (Appendix A.1: members checkpoint themselves; here the whole population record) -----
+    def state_dict(self) -> Dict[str, np.ndarray]:
+        """The population record (theta, h, p, t) of every member plus optimiser state, score histories and the
+        ready-point counter, as host arrays: enough to continue a run bit for bit with load_state_dict."""
+        n = self.cfg.n_members
+        members = [self.get_state(m) for m in range(n)]
+        out = {"step": np.int64(members[0]["step"]), "round": np.int64(members[0]["round"]),
+               "hparams": self.hparams(), "fitness": self.fitness(),
+               "scalars": np.stack([s["scalars"] for s in members]),
+               "w": np.stack([s["w"] for s in members])}
+        if not self.toy:
+            out["opt1"] = np.stack([s["opt1"] for s in members])
+            out["opt2"] = np.stack([s["opt2"] for s in members])
+        hist, count = self.history()
+        out["history"], out["history_count"] = hist, count
+        return out
+
+    def load_state_dict(self, sd) -> None:
+        n = self.cfg.n_members
+        assert sd["w"].shape[0] == n and sd["hparams"].shape == (n, self.nh)
+        for m in range(n):
+            self.set_state(m, w=sd["w"][m], opt1=None if self.toy else sd["opt1"][m],
+                           opt2=None if self.toy else sd["opt2"][m], scalars=sd["scalars"][m],
+                           hparams=sd["hparams"][m], fitness=float(sd["fitness"][m]),
+                           step=int(sd["step"]), round=int(sd["round"]))
+        self.set_history(np.asarray(sd["history"], dtype=np.float64), np.asarray(sd["history_count"], dtype=np.int32))
+
+    def save(self, path: str) -> None:
+        np.savez(path, **self.state_dict())
+
+    def load(self, path: str) -> None:
+        with np.load(path) as z:
+            self.load_state_dict({k: z[k] for k in z.files})
+
     def _ready_point(self, step, ready, log):
         """eval, exploit / explore and, if asked, one record of the ready point (Section 4.4's analyses are made
         from such records: score and hyperparameter traces, who copied whom)."""

@@ -248,6 +248,33 @@ def test_staggered_run_matches_the_oracle_schedule(pkg):
     gpu.close()
 
 
+@pytest.mark.parametrize("name", ["c1", "c2_mini_ttest", "c3_mini", "c4_mini_wgan", "c3_mini_stagger_tournament"])
+def test_checkpoint_resume_is_bit_exact(pkg, name, tmp_path):
+    """Appendix A.1: members are restored from checkpoints.  A population saved after some ready points and loaded
+    into a fresh handle continues exactly like the one that kept running: records, score histories, counters and
+    the decisions of the following ready points, bit for bit."""
+    cfg = get_config(name)
+    inp = make_inputs(cfg)
+    a = pkg.Population(cfg, inp)
+    a.run(2 * cfg.ready_interval)
+    path = str(tmp_path / "pop.npz")
+    a.save(path)
+    b = pkg.Population(cfg, inp)
+    b.load(path)
+    for pop in (a, b):
+        for _ in range(2):
+            pop.step(cfg.ready_interval)
+            pop.eval()
+            pop.exploit_explore()
+    sa, sb = a.state_dict(), b.state_dict()
+    assert set(sa) == set(sb)
+    for key in sa:
+        assert np.array_equal(sa[key], sb[key], equal_nan=True), (name, key)
+    assert np.array_equal(a.copy_map(), b.copy_map())
+    a.close()
+    b.close()
+
+
 def test_ready_point_log_and_lineages(pkg):
     """The ready-point records of a run: one per ready point, copy maps consistent with the hyperparameter traces
     (only members that copied change h), and the number of surviving initial lineages never grows (Section 4.4)."""
