@@ -266,7 +266,7 @@ class Population:
     """One population living on one GPU.  Thin wrapper over the pbt_* calls."""
 
     def __init__(self, cfg, inputs, seed: Optional[int] = None, device: str = "cuda:0", keep_grad: bool = False,
-                 fuse_adam: bool = True):
+                 fuse_adam: bool = True, guard_bytes: int = 0):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -304,8 +304,12 @@ class Population:
         nbytes = C.c_size_t(0)
         self._check(self.lib.pbt_query_workspace(C.byref(self.spec), C.byref(nbytes)), None)
         self.workspace_bytes = nbytes.value
-        self.workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
-        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        # optional guard bands on both sides of the workspace (a debugging aid: guards_intact() tells whether any
+        # kernel wrote outside the memory the library was given)
+        self.guard_bytes = (int(guard_bytes) + 255) // 256 * 256
+        self.workspace = torch.full((nbytes.value + 256 + 2 * self.guard_bytes,), 0xA5, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + self.guard_bytes + 255) // 256 * 256
+        self._ws_off = base - self.workspace.data_ptr()
         h0 = np.ascontiguousarray(inputs.init_hparams, dtype=np.float64)
         assert h0.shape == (self.N, self.nh)
         self.handle = C.c_void_p(None)
@@ -339,6 +343,13 @@ class Population:
 
     def synchronize(self):
         self.stream.synchronize()
+
+    def guards_intact(self) -> bool:
+        """True if the guard bands around the workspace (guard_bytes at construction) still hold their fill."""
+        self.synchronize()
+        lo = self.workspace[:self._ws_off]
+        hi = self.workspace[self._ws_off + self.workspace_bytes:]
+        return bool((lo == 0xA5).all().item()) and bool((hi == 0xA5).all().item())
 
     # ----- the hot path ---------------------------------------------------
     def step(self, k: int = 1):

@@ -275,6 +275,23 @@ def test_checkpoint_resume_is_bit_exact(pkg, name, tmp_path):
     b.close()
 
 
+@pytest.mark.parametrize("name", ["c2_mini", "c3_mini", "c4_mini", "c4_mini_wgan", "c5_mini", "c3_mid", "c5_mid", "c4_mid_wgan",
+                                  "c2_mini_ttest", "c3_mini_stagger_tournament"])
+def test_no_kernel_writes_outside_the_workspace(pkg, name):
+    """Every kernel of a run (steps, evaluations, ready points; ragged and tile-sized shapes) stays inside the
+    workspace it was given: 1 MiB guard bands on both sides keep their fill, and the device status word stays 0."""
+    cfg = get_config(name)
+    inp = make_inputs(cfg)
+    for kw in ({"keep_grad": True, "fuse_adam": False}, {}):
+        gpu = pkg.Population(cfg, inp, guard_bytes=1 << 20, **kw)
+        assert gpu.guards_intact()
+        gpu.run(2 * cfg.ready_interval)
+        gpu.eval()
+        assert np.isfinite(gpu.fitness()).all()       # also reads the status word
+        assert gpu.guards_intact(), (name, kw)
+        gpu.close()
+
+
 def test_ready_point_log_and_lineages(pkg):
     """The ready-point records of a run: one per ready point, copy maps consistent with the hyperparameter traces
     (only members that copied change h), and the number of surviving initial lineages never grows (Section 4.4)."""
