@@ -73,6 +73,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         const int rem = tile % (p.tiles_m * p.tiles_n);
         const int m0 = (rem / p.tiles_n) * kBM, n0 = (rem % p.tiles_n) * BN;
         const int ca = p.a_batched ? member : 0, cb = p.b_batched ? member : 0;
+        // a windowed operand is one shared matrix: the problem's rows start at its offset (slow coordinate)
+        const int ra = p.a_rowoff ? p.a_rowoff[member] : 0, rb = p.b_rowoff ? p.b_rowoff[member] : 0;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + stage * L::kStageBytes;
@@ -80,16 +82,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           mbar_expect_tx(&full[stage], L::kStageBytes);
           const int k0 = kb * kBK;
           if (!p.a_mn) {
-            tma_load_3d(sa, &tmA, &full[stage], k0, m0, ca);
+            tma_load_3d(sa, &tmA, &full[stage], k0, m0 + ra, ca);
           } else {
 #pragma unroll
-            for (int j = 0; j < kBM / 64; ++j) tma_load_3d(sa + j * 8192, &tmA, &full[stage], m0 + j * 64, k0, ca);
+            for (int j = 0; j < kBM / 64; ++j) tma_load_3d(sa + j * 8192, &tmA, &full[stage], m0 + j * 64, k0 + ra, ca);
           }
           if (!p.b_mn) {
-            tma_load_3d(sb, &tmB, &full[stage], k0, n0, cb);
+            tma_load_3d(sb, &tmB, &full[stage], k0, n0 + rb, cb);
           } else {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j) tma_load_3d(sb + j * 8192, &tmB, &full[stage], n0 + j * 64, k0, cb);
+            for (int j = 0; j < BN / 64; ++j) tma_load_3d(sb + j * 8192, &tmB, &full[stage], n0 + j * 64, k0 + rb, cb);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -245,8 +247,9 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s
   p.tiles_m = (g.M + kBM - 1) / kBM;
   p.k_blocks = (g.K + kBK - 1) / kBK;
   p.a_mn = g.a_mn; p.b_mn = g.b_mn;
-  p.a_batched = (g.batch > 1 && g.strideA != 0) ? 1 : 0;
-  p.b_batched = (g.batch > 1 && g.strideB != 0) ? 1 : 0;
+  p.a_batched = (g.batch > 1 && g.strideA != 0 && !g.a_rowoff) ? 1 : 0;
+  p.b_batched = (g.batch > 1 && g.strideB != 0 && !g.b_rowoff) ? 1 : 0;
+  p.a_rowoff = g.a_rowoff; p.b_rowoff = g.b_rowoff;
   p.C = g.C; p.ldc = g.ldc; p.strideC = g.strideC; p.out_dtype = g.out_dtype;
   p.bias = g.bias; p.strideBias = g.strideBias; p.relu = g.relu;
   p.mask = reinterpret_cast<const bf16*>(g.mask); p.ldmask = g.ldmask; p.strideMask = g.strideMask;
@@ -255,11 +258,14 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s
   CUtensorMap tmA, tmB;
   bool ok;
   // K-major operand: rows = M (or N), cols = K.  MN-major operand: rows = K, cols = M (or N), boxes of 64 x 64.
-  if (!g.a_mn) ok = make_map(&tmA, g.A, g.K, g.M, g.lda, p.a_batched ? g.batch : 1, g.strideA, kBM);
-  else ok = make_map(&tmA, g.A, g.M, g.K, g.lda, p.a_batched ? g.batch : 1, g.strideA, kBK);
+  // A windowed operand's map covers the whole shared matrix (its rows_total rows).
+  const long long a_rows = g.a_rowoff ? g.a_rows_total : (g.a_mn ? g.K : g.M);
+  const long long b_rows = g.b_rowoff ? g.b_rows_total : (g.b_mn ? g.K : g.N);
+  if (!g.a_mn) ok = make_map(&tmA, g.A, g.K, a_rows, g.lda, p.a_batched ? g.batch : 1, g.strideA, kBM);
+  else ok = make_map(&tmA, g.A, g.M, a_rows, g.lda, p.a_batched ? g.batch : 1, g.strideA, kBK);
   if (!ok) return cudaErrorInvalidValue;
-  if (!g.b_mn) ok = make_map(&tmB, g.B, g.K, g.N, g.ldb, p.b_batched ? g.batch : 1, g.strideB, BN);
-  else ok = make_map(&tmB, g.B, g.N, g.K, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kBK);
+  if (!g.b_mn) ok = make_map(&tmB, g.B, g.K, b_rows, g.ldb, p.b_batched ? g.batch : 1, g.strideB, BN);
+  else ok = make_map(&tmB, g.B, g.N, b_rows, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kBK);
   if (!ok) return cudaErrorInvalidValue;
   if (g.adam) return cudaErrorInvalidValue;  // the fused weight-gradient + Adam kernel has its own launcher
   // 8 epilogue warps (two per TMEM lane quadrant) keep the tile write-out and the ReLU-mask reads off the critical

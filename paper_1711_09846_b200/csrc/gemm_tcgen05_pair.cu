@@ -123,6 +123,7 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int m0 = (rem / p.tiles_n) * (2 * kBM) + (int)rank * kBM;
         const int n0 = (rem % p.tiles_n) * kPN + (int)rank * (kPN / 2);
         const int ca = p.a_batched ? member : 0, cb = p.b_batched ? member : 0;
+        const int ra = p.a_rowoff ? p.a_rowoff[member] : 0, rb = p.b_rowoff ? p.b_rowoff[member] : 0;   // row windows
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + stage * kPStageBytes;
@@ -133,16 +134,16 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (rank == 0) mbar_expect_tx(&full[stage], 2 * kPStageBytes);
           const int k0 = kb * kBK;
           if (!p.a_mn) {
-            tma_load_3d_pair(sa, &tmA, lbar, k0, m0, ca);
+            tma_load_3d_pair(sa, &tmA, lbar, k0, m0 + ra, ca);
           } else {
 #pragma unroll
-            for (int j = 0; j < kBM / 64; ++j) tma_load_3d_pair(sa + j * 8192, &tmA, lbar, m0 + j * 64, k0, ca);
+            for (int j = 0; j < kBM / 64; ++j) tma_load_3d_pair(sa + j * 8192, &tmA, lbar, m0 + j * 64, k0 + ra, ca);
           }
           if (!p.b_mn) {
-            tma_load_3d_pair(sb, &tmB, lbar, k0, n0, cb);
+            tma_load_3d_pair(sb, &tmB, lbar, k0, n0 + rb, cb);
           } else {
 #pragma unroll
-            for (int j = 0; j < kPN / 128; ++j) tma_load_3d_pair(sb + j * 8192, &tmB, lbar, n0 + j * 64, k0, cb);
+            for (int j = 0; j < kPN / 128; ++j) tma_load_3d_pair(sb + j * 8192, &tmB, lbar, n0 + j * 64, k0 + rb, cb);
           }
           if (++stage == kPStages) { stage = 0; phase ^= 1; }
         }
@@ -249,19 +250,22 @@ cudaError_t launch_gemm_tc_pair(const GemmArgs& g, Counters* counters, cudaStrea
   p.num_tiles = p.tiles_m * p.tiles_n * g.batch;
   p.k_blocks = (g.K + kBK - 1) / kBK;
   p.a_mn = g.a_mn; p.b_mn = g.b_mn;
-  p.a_batched = (g.batch > 1 && g.strideA != 0) ? 1 : 0;
-  p.b_batched = (g.batch > 1 && g.strideB != 0) ? 1 : 0;
+  p.a_batched = (g.batch > 1 && g.strideA != 0 && !g.a_rowoff) ? 1 : 0;
+  p.b_batched = (g.batch > 1 && g.strideB != 0 && !g.b_rowoff) ? 1 : 0;
+  p.a_rowoff = g.a_rowoff; p.b_rowoff = g.b_rowoff;
   p.C = g.C; p.ldc = g.ldc; p.strideC = g.strideC; p.out_dtype = g.out_dtype;
   p.bias = g.bias; p.strideBias = g.strideBias; p.relu = g.relu;
   p.mask = reinterpret_cast<const bf16*>(g.mask); p.ldmask = g.ldmask; p.strideMask = g.strideMask;
   p.counters = counters;
   CUtensorMap tmA, tmB;
   bool ok;
-  if (!g.a_mn) ok = make_map(&tmA, g.A, g.K, g.M, g.lda, p.a_batched ? g.batch : 1, g.strideA, kBM);
-  else ok = make_map(&tmA, g.A, g.M, g.K, g.lda, p.a_batched ? g.batch : 1, g.strideA, kBK);
+  const long long a_rows = g.a_rowoff ? g.a_rows_total : (g.a_mn ? g.K : g.M);   // a windowed operand: the whole pool
+  const long long b_rows = g.b_rowoff ? g.b_rows_total : (g.b_mn ? g.K : g.N);
+  if (!g.a_mn) ok = make_map(&tmA, g.A, g.K, a_rows, g.lda, p.a_batched ? g.batch : 1, g.strideA, kBM);
+  else ok = make_map(&tmA, g.A, g.M, a_rows, g.lda, p.a_batched ? g.batch : 1, g.strideA, kBK);
   if (!ok) return cudaErrorInvalidValue;
-  if (!g.b_mn) ok = make_map(&tmB, g.B, g.K, g.N, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kPN / 2);
-  else ok = make_map(&tmB, g.B, g.N, g.K, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kBK);
+  if (!g.b_mn) ok = make_map(&tmB, g.B, g.K, b_rows, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kPN / 2);
+  else ok = make_map(&tmB, g.B, g.N, b_rows, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kBK);
   if (!ok) return cudaErrorInvalidValue;
   static bool configured = false;
   if (!configured) {

@@ -79,6 +79,21 @@ __global__ void k_gather_window(char* __restrict__ dst, long long dst_stride_byt
   }
 }
 
+__global__ void k_window_offsets(int* __restrict__ off, int rows, int pool_rows, int n_members, int block, int word_index,
+                                 uint64_t seed, const Counters* __restrict__ counters) {
+  const int m = blockIdx.x * blockDim.x + threadIdx.x;
+  if (m >= n_members) return;
+  const U4 r = philox4x32_10((uint32_t)m, (uint32_t)counters->step, kStreamBatch, (uint32_t)block, seed);
+  const uint32_t n_win = (uint32_t)((pool_rows - rows) / 128 + 1);
+  off[m] = (int)(128ll * (long long)(((uint64_t)r.x[word_index] * n_win) >> 32));
+}
+
+cudaError_t launch_window_offsets(int* off, int rows, int pool_rows, int n_members, int block, int word_index,
+                                  uint64_t seed, const Counters* counters, cudaStream_t s) {
+  k_window_offsets<<<(n_members + 127) / 128, 128, 0, s>>>(off, rows, pool_rows, n_members, block, word_index, seed, counters);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_gather_window(char* dst, long long dst_stride_bytes, long long dst_offset_bytes,
                                  const char* pool, int row_bytes, int rows, int pool_rows, int n_members,
                                  int block, int word_index, uint64_t seed, const Counters* counters,
@@ -157,10 +172,11 @@ __global__ void k_loss_rows(LossArgs a) {
   const int row = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
   if (row >= a.rows) return;
   const float* z = a.logits + m * a.stride_logits + (long long)row * a.ld_logits;
+  const long long trow = (long long)row + (a.target_rowoff ? a.target_rowoff[m] : 0);   // row of the target matrix
   const long long dz_base = m * a.stride_dz + (long long)row * a.ld_dz;
   float loss = 0.f;
   if (a.kind == PBT_LOSS_MSE) {
-    const float* y = reinterpret_cast<const float*>(a.target) + m * a.stride_target + (long long)row * a.cols;
+    const float* y = reinterpret_cast<const float*>(a.target) + m * a.stride_target + trow * a.cols;
     float acc = 0.f;
     for (int c = lane; c < a.cols; c += 32) {
       const float d = z[c] - y[c];
@@ -178,7 +194,7 @@ __global__ void k_loss_rows(LossArgs a) {
     const float lse = logf(se);
     const float inv_se = 1.f / se;
     if (a.kind == PBT_LOSS_CE_HARD) {
-      const int label = reinterpret_cast<const int*>(a.target)[m * a.stride_target + row];
+      const int label = reinterpret_cast<const int*>(a.target)[m * a.stride_target + trow];
       loss = lse - (z[label] - mx);
       if (a.dz)
         for (int c = lane; c < a.cols; c += 32) {
@@ -186,7 +202,7 @@ __global__ void k_loss_rows(LossArgs a) {
           store_from_float(a.dz, a.dz_dtype, dz_base + c, (p - (c == label ? 1.f : 0.f)) * a.inv_batch);
         }
     } else {
-      const long long tb = m * a.stride_target + (long long)row * a.cols;
+      const long long tb = m * a.stride_target + trow * a.cols;
       float tsum = 0.f, tl = 0.f;
       for (int c = lane; c < a.cols; c += 32) {
         const float t = load_as_float(a.target, a.target_dtype, tb + c);
@@ -230,8 +246,8 @@ __global__ void __launch_bounds__(256) k_loss_ce_soft_vec(LossArgs a) {
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
   if (row >= a.rows) return;
   const float4* z4 = reinterpret_cast<const float4*>(a.logits + m * a.stride_logits + (long long)row * a.ld_logits);
-  const uint2* t2 = reinterpret_cast<const uint2*>(reinterpret_cast<const bf16*>(a.target) + m * a.stride_target +
-                                                   (long long)row * a.cols);
+  const long long trow = (long long)row + (a.target_rowoff ? a.target_rowoff[m] : 0);
+  const uint2* t2 = reinterpret_cast<const uint2*>(reinterpret_cast<const bf16*>(a.target) + m * a.stride_target + trow * a.cols);
   float4 z[ITERS];
   uint2 tp[ITERS];
 #pragma unroll

@@ -72,6 +72,11 @@ struct pbt_handle {
   void* gp_dz[PBT_MAX_LAYERS];
   float* gp_gx;
   bool wgan;
+  // MLP populations whose first layer runs on the tensor cores read their training rows straight from the data
+  // pools (TMA row windows) instead of gathering them first: win_off[m] is member m's first pool row this step
+  int* win_off;
+  bool direct_pool;
+  bool supplied_next;   // the next step trains on rows the caller put into act[0][0] / ybatch
   void* ybatch;
   long long ybatch_stride;  // elements of the target type per member
   // second copy of the training-row buffers: host batches are uploaded here on a copy stream while the step
@@ -211,6 +216,8 @@ size_t plan(pbt_handle* h, char* base) {
   h->hist_n = (int*)take(N * sizeof(int));
   h->last_loss = (float*)take(N * 2 * sizeof(float));
   h->scalars = (float*)take(N * PBT_N_SCALARS * sizeof(float));
+  h->win_off = (int*)take(N * sizeof(int));
+  h->direct_pool = false;
   if (h->toy) {
     h->P = s.nh;
     h->P_pad = s.nh;
@@ -287,6 +294,12 @@ size_t plan(pbt_handle* h, char* base) {
     h->act0_alt = nullptr;
     h->ybatch_stride = 0;
   }
+  if (!h->gan && h->is_bf16) {
+    const Layer& L0 = h->st[0].L[0];
+    h->direct_pool = s.batch >= 128 && s.batch % 64 == 0 && L0.in >= 128 && L0.out >= 128 && L0.in % 8 == 0 &&
+                     L0.out % 8 == 0 && h->data.x_pool && (((uintptr_t)h->data.x_pool) & 15) == 0 &&
+                     h->data.y_pool && (((uintptr_t)h->data.y_pool) & 15) == 0;
+  }
   h->row_loss = (float*)take(N * (size_t)h->rowloss_cap * sizeof(float));
   h->ed_partial = h->gan ? (double*)take(N * (size_t)energy_partial_count(s.eval_batch) * sizeof(double)) : nullptr;
   h->workspace_bytes = off;
@@ -354,6 +367,7 @@ int gemm(pbt_handle* h, const GemmArgs& g) {
   } else if (gemm_tc_supported(g)) {
     LAUNCH(h, kGemm, launch_gemm_tc(g, h->counters, h->stream));
   } else {
+    if (g.a_rowoff || g.b_rowoff) return fail(h, PBT_ERR_UNSUPPORTED, "row-window operands need a tensor-core shape");
     LAUNCH(h, kGemm, launch_gemm_simt(g, h->stream));
   }
   return PBT_OK;
@@ -364,7 +378,9 @@ const void* weights(const pbt_handle* h, long long off) {
 }
 
 // z_l = a_{l-1} W_l^T + b_l, ReLU on hidden layers; the last layer's output goes to logits[k] in fp32
-int forward(pbt_handle* h, int k, int rows, const void* in, long long in_stride) {
+// With in_rowoff the input rows of member m are rows in_rowoff[m].. of `in`, a pool of in_rows_total rows.
+int forward(pbt_handle* h, int k, int rows, const void* in, long long in_stride, const int* in_rowoff = nullptr,
+            long long in_rows_total = 0) {
   const Stack& st = h->st[k];
   for (int l = 0; l < st.nl; ++l) {
     const Layer& L = st.L[l];
@@ -375,6 +391,7 @@ int forward(pbt_handle* h, int k, int rows, const void* in, long long in_stride)
     g.A = l == 0 ? in : h->act[k][l];
     g.lda = L.in;
     g.strideA = l == 0 ? in_stride : act_stride(h, k, l);
+    if (l == 0 && in_rowoff) { g.a_rowoff = in_rowoff; g.a_rows_total = in_rows_total; g.strideA = 0; }
     g.B = weights(h, L.w_off); g.ldb = L.in; g.strideB = h->P_pad;
     g.bias = h->W32 + L.b_off; g.strideBias = h->P_pad;
     if (l + 1 < st.nl) {
@@ -421,7 +438,8 @@ int dgrad(pbt_handle* h, int k, int l, int rows, const void* dz, long long dz_st
 // Layers whose weight gradient runs on the tensor cores get their Adam update inside that GEMM's epilogue
 // (the caller must have finished every read of the layer's old weights); fused[l] records it.
 int wgrad_layer(pbt_handle* h, int k, int l, int rows, int bias_rows, const void* dz, long long dz_stride,
-                const void* in, long long in_stride, const OptArgs& opt, bool* fused) {
+                const void* in, long long in_stride, const OptArgs& opt, bool* fused, const int* in_rowoff = nullptr,
+                long long in_rows_total = 0) {
   const pbt_spec& s = h->spec;
   const Layer& L = h->st[k].L[l];
   GemmArgs g;
@@ -430,6 +448,7 @@ int wgrad_layer(pbt_handle* h, int k, int l, int rows, int bias_rows, const void
   g.in_dtype = h->cdt; g.out_dtype = kF32;
   g.A = dz; g.lda = L.out; g.strideA = dz_stride; g.a_mn = 1;
   g.B = in; g.ldb = L.in; g.strideB = in_stride; g.b_mn = 1;
+  if (in_rowoff) { g.b_rowoff = in_rowoff; g.b_rows_total = in_rows_total; g.strideB = 0; }
   g.C = h->G + L.w_off; g.ldc = L.in; g.strideC = h->P_pad;
   OptArgs lopt = opt;
   if (s.fuse_adam && s.optimizer == PBT_OPT_ADAM && gemm_tc_supported(g)) {
@@ -484,7 +503,8 @@ int finish_optimizer(pbt_handle* h, int k, const bool* fused, const OptArgs& opt
 // With need_wgrad the optimiser update of the stack is part of this pass: a layer's fused update runs
 // after the layer's data gradient has read the old weights.
 int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride, bool need_wgrad,
-             bool need_input_grad, int* cur, int slot_lr, int scalar_base) {
+             bool need_input_grad, int* cur, int slot_lr, int scalar_base, const int* in_rowoff = nullptr,
+             long long in_rows_total = 0) {
   const Stack& st = h->st[k];
   const long long dzs = dz_stride(h);
   OptArgs opt;
@@ -501,7 +521,8 @@ int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride
     }
     if (need_wgrad) {
       int rc = wgrad_layer(h, k, l, rows, rows, dz, dzs, l == 0 ? in : h->act[k][l],
-                           l == 0 ? in_stride : act_stride(h, k, l), opt, fused);
+                           l == 0 ? in_stride : act_stride(h, k, l), opt, fused, l == 0 ? in_rowoff : nullptr,
+                           in_rows_total);
       if (rc) return rc;
     }
     if (wrote_dgrad) *cur = 1 - *cur;
@@ -511,7 +532,7 @@ int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride
 }
 
 int loss_and_dz(pbt_handle* h, int k, int rows, int n_real, const void* target, long long target_stride,
-                bool want_dz, int dz_buf, float scale, void* out, int out_stride) {
+                bool want_dz, int dz_buf, float scale, void* out, int out_stride, const int* target_rowoff = nullptr) {
   const pbt_spec& s = h->spec;
   const Stack& st = h->st[k];
   LossArgs a;
@@ -519,7 +540,7 @@ int loss_and_dz(pbt_handle* h, int k, int rows, int n_real, const void* target, 
   a.kind = s.loss; a.n_members = h->N; a.rows = rows; a.cols = st.L[st.nl - 1].out;
   a.n_real_rows = n_real; a.inv_batch = 1.0f / (float)s.batch;
   a.logits = h->logits[k]; a.ld_logits = a.cols; a.stride_logits = logits_stride(h, k);
-  a.target = target; a.stride_target = target_stride;
+  a.target = target; a.stride_target = target_stride; a.target_rowoff = target_rowoff;
   a.target_dtype = s.loss == PBT_LOSS_CE_SOFT ? h->cdt : kF32;
   a.dz = want_dz ? h->dz[dz_buf] : nullptr; a.dz_dtype = h->cdt; a.ld_dz = a.cols; a.stride_dz = dz_stride(h);
   a.row_loss = h->row_loss;
@@ -540,6 +561,16 @@ int step_mlp(pbt_handle* h) {
   const pbt_spec& s = h->spec;
   const Stack& st = h->st[0];
   const int in = st.L[0].in;
+  if (h->direct_pool && !h->supplied_next) {
+    // the first layer's forward and weight-gradient GEMMs and the loss read the window of each member in place
+    LAUNCH(h, kCopy, launch_window_offsets(h->win_off, s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, h->stream));
+    int rc = forward(h, 0, s.batch, h->data.x_pool, 0, h->win_off, s.pool_rows);
+    if (rc) return rc;
+    rc = loss_and_dz(h, 0, s.batch, s.batch, h->data.y_pool, 0, true, 0, 1.0f / s.batch, h->last_loss, 2, h->win_off);
+    if (rc) return rc;
+    int cur = 0;
+    return backward(h, 0, s.batch, h->data.x_pool, 0, true, false, &cur, s.slot_lr, 0, h->win_off, s.pool_rows);
+  }
   LAUNCH(h, kCopy, launch_gather_window((char*)h->act[0][0], act_stride(h, 0, 0) * h->esz, 0, (const char*)h->data.x_pool,
                                         in * h->esz, s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, h->stream));
   const size_t trb = target_row_bytes(h);
@@ -702,6 +733,7 @@ int one_step(pbt_handle* h) {
     if (rc) return rc;
   }
   LAUNCH(h, kOther, launch_advance_step(h->counters, h->stream));
+  h->supplied_next = false;
   return PBT_OK;
 }
 
@@ -857,6 +889,12 @@ int pbt_step(pbt_t* p, int k) {
   p->launches = 0;
   // Small populations are launch-bound: replay one captured step as a CUDA graph.  Capture needs a
   // non-default stream and no per-launch event records.
+  if (k > 0 && p->supplied_next && p->direct_pool) {
+    // the captured step reads the pools; the caller's rows are consumed by one step of the other form
+    int rc = one_step(p);
+    if (rc) return rc;
+    --k;
+  }
   const bool want_graph = !p->profiling && !p->graph_failed && p->stream != nullptr && k > 0;
   if (want_graph && !p->step_graph) {
     cudaGraph_t graph = nullptr;
@@ -1249,6 +1287,7 @@ int pbt_set_batch(pbt_t* p, const void* x, const void* y) {
   const int one = 1;
   CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &one, 4, cudaMemcpyHostToDevice, p->stream));
   CU(p, cudaStreamSynchronize(p->stream));
+  p->supplied_next = true;
   return PBT_OK;
 }
 
@@ -1264,6 +1303,7 @@ int pbt_step_host(pbt_t* p, const void* x_host, const void* y_host, double* loss
   CU(p, cudaMemcpy2DAsync(p->ybatch, p->ybatch_stride * tsz, y_host, trb, trb, p->N, cudaMemcpyHostToDevice, p->stream));
   const int one = 1;
   CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &one, 4, cudaMemcpyHostToDevice, p->stream));
+  p->supplied_next = true;
   int rc = one_step(p);
   if (rc) return rc;
   if (loss_out_host) {
@@ -1310,6 +1350,7 @@ int pbt_step_prefetched(pbt_t* p, double* loss_out_host) {
   if (p->step_graph) { cudaGraphExecDestroy(p->step_graph); p->step_graph = nullptr; }
   const int one = 1;
   CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &one, 4, cudaMemcpyHostToDevice, p->stream));
+  p->supplied_next = true;
   int rc = one_step(p);
   if (rc) return rc;
   CU(p, cudaEventRecord(p->ev_stepdone[p->pf_steps & 1], p->stream));

@@ -77,6 +77,12 @@ struct GemmArgs {
   // to the member's slab in place (C[m][n] is the gradient of element adam->begin + m*ldc + n) and stores the
   // gradient itself only if C is not null.
   const struct OptArgs* adam;
+  // Row windows (tensor-core kernels only): operand X is then ONE matrix of x_rows_total rows shared by all
+  // problems (a data pool) and problem b uses the rows that start at x_rowoff[b] (device array, one int per
+  // problem); strideX is ignored.  "Row" is the slow index of the stored matrix: m (or n) for a K-major operand,
+  // k for an MN-major one.
+  const int* a_rowoff; long long a_rows_total;
+  const int* b_rowoff; long long b_rows_total;
 };
 
 // launchers (each enqueues on `s` and returns the CUDA error of the launch)
@@ -199,6 +205,9 @@ cudaError_t launch_init_weights(float* w32, long long p_pad, int n_members, long
 cudaError_t launch_f32_to_bf16(const float* in, bf16* out, long long n, cudaStream_t s);
 // copy rows [off, off+rows) of a pool into dst + m*dst_stride_bytes (+ dst_offset_bytes) for every member;
 // off = 128 * ((word * n_win) >> 32), word = philox(seed; m, step, batch stream, block).x[word_index]
+// off[m] = first pool row of member m's training window for the current step (the rule of launch_gather_window)
+cudaError_t launch_window_offsets(int* off, int rows, int pool_rows, int n_members, int block, int word_index,
+                                  uint64_t seed, const Counters* counters, cudaStream_t s);
 cudaError_t launch_gather_window(char* dst, long long dst_stride_bytes, long long dst_offset_bytes,
                                  const char* pool, int row_bytes, int rows, int pool_rows, int n_members,
                                  int block, int word_index, uint64_t seed, const Counters* counters,
@@ -216,6 +225,8 @@ struct LossArgs {
   float inv_batch; // 1 / B  (scale of dL/dz and of the mean)
   const float* logits; long long ld_logits, stride_logits;
   const void* target; long long stride_target;   // elements of the target type; 0 = shared by all members
+  const int* target_rowoff;                      // optional (device, one int per member): the member's targets are the
+                                                 // rows of a shared pool that start here (stride_target is then 0)
   int target_dtype;                              // DType for MSE / CE_SOFT targets (MSE is always float)
   void* dz; int dz_dtype; long long ld_dz, stride_dz;   // may be null (eval)
   float* row_loss;   // [n_members][rows]

@@ -19,6 +19,8 @@ struct TcParams {
   const float* bias; long long strideBias; int relu;
   const bf16* mask; long long ldmask, strideMask;
   Counters* counters;
+  const int* a_rowoff;   // per-problem first row of the A / B operand inside a shared matrix (null: batched operand)
+  const int* b_rowoff;
 };
 
 

@@ -51,6 +51,7 @@ struct FusedParams {
   int tiles_m, tiles_n, num_tiles, k_blocks;
   float* gout; long long ldc, strideC;  // optional copy of the gradient (may be null)
   Counters* counters;
+  const int* in_rowoff;   // layer input taken from a shared pool: first batch row of each member (null: per-member buffer)
   OptArgs opt;
 };
 
@@ -102,13 +103,14 @@ k_wgrad_adam(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
         const int member = tile / tiles_per_member, rem = tile % tiles_per_member;
         const int m0 = (rem / p.tiles_n) * kBM, n0 = (rem % p.tiles_n) * kBN;
+        const int ra = p.in_rowoff ? p.in_rowoff[member] : 0, ca = p.in_rowoff ? 0 : member;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
           uint8_t* sa = smem + stage * kStageBytes;
           uint8_t* sb = sa + kABytes;
           mbar_expect_tx(&full[stage], kStageBytes);
 #pragma unroll
-          for (int j = 0; j < kBM / 64; ++j) tma_load_3d(sa + j * 8192, &tmA, &full[stage], m0 + j * 64, kb * kBK, member);
+          for (int j = 0; j < kBM / 64; ++j) tma_load_3d(sa + j * 8192, &tmA, &full[stage], m0 + j * 64, kb * kBK + ra, ca);
 #pragma unroll
           for (int j = 0; j < kBN / 64; ++j) tma_load_3d(sb + j * 8192, &tmB, &full[stage], n0 + j * 64, kb * kBK, member);
           if (++stage == kStages) { stage = 0; phase ^= 1; }
@@ -295,14 +297,16 @@ cudaError_t launch_wgrad_adam(const GemmArgs& g, Counters* counters, cudaStream_
   CUtensorMap tmA, tmB, tmW, tmM, tmV, tmW16;
   const int ab = (g.batch > 1 && g.strideA != 0) ? g.batch : 1, bb = (g.batch > 1 && g.strideB != 0) ? g.batch : 1;
   // operand roles swapped (the layer input is the kernel's A); state boxes: kChunk weight rows x kBM inputs, row-major
-  bool ok = make_map(&tmA, g.B, g.N, g.K, g.ldb, bb, g.strideB, kBK) &&
+  p.in_rowoff = g.b_rowoff;
+  bool ok = make_map(&tmA, g.B, g.N, g.b_rowoff ? g.b_rows_total : g.K, g.ldb, g.b_rowoff ? 1 : bb, g.strideB, kBK) &&
             make_map(&tmB, g.A, g.M, g.K, g.lda, ab, g.strideA, kBK) &&
             make_map(&tmW, o.w32 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kChunk, 4, kBM, 0) &&
             make_map(&tmM, o.opt1 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kChunk, 4, kBM, 0) &&
             make_map(&tmV, o.opt2 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kChunk, 4, kBM, 0) &&
             make_map(&tmW16, o.w16 + o.begin, g.N, g.M, g.ldc, g.batch, o.p_pad, kChunk, 2, kBM, 0);
   if (!ok) return cudaErrorInvalidValue;
-  if (g.batch > 1 && (g.strideA == 0 || g.strideB == 0)) return cudaErrorInvalidValue;  // operands are per member here
+  if (g.a_rowoff) return cudaErrorInvalidValue;   // only the layer input can come from a pool
+  if (g.batch > 1 && (g.strideA == 0 || (g.strideB == 0 && !g.b_rowoff))) return cudaErrorInvalidValue;  // operands are per member here
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(k_wgrad_adam, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
