@@ -109,8 +109,8 @@ class ClockSampler:
 
 # DRAM bytes per parameter of the fused weight-gradient + Adam kernel, from one `ncu --set full` capture of a
 # small case (profiles/k_wgrad_adam_c5_8members.md), valid for the source file with this sha1 only.
-_NCU_TRAFFIC = {"wgrad_adam": {"bytes_per_param": 25.40, "source": "paper_1711_09846_b200/csrc/wgrad_adam_tcgen05.cu",
-                               "sha1": "1a23ce01242513f201662b9397fbf935bc3d0339"}}
+_NCU_TRAFFIC = {"wgrad_adam": {"bytes_per_param": 25.41, "source": "paper_1711_09846_b200/csrc/wgrad_adam_tcgen05.cu",
+                               "sha1": "361db330e5ece7f9d58438bc88611d1a377a3299"}}
 
 
 def _ncu_traffic(name, params_per_launch):

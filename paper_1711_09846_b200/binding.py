@@ -307,9 +307,12 @@ class Population:
         # optional guard bands on both sides of the workspace (a debugging aid: guards_intact() tells whether any
         # kernel wrote outside the memory the library was given)
         self.guard_bytes = (int(guard_bytes) + 255) // 256 * 256
-        self.workspace = torch.full((nbytes.value + 256 + 2 * self.guard_bytes,), 0xA5, dtype=torch.uint8, device=self.device)
+        self.workspace = torch.empty(nbytes.value + 256 + 2 * self.guard_bytes, dtype=torch.uint8, device=self.device)
         base = (self.workspace.data_ptr() + self.guard_bytes + 255) // 256 * 256
         self._ws_off = base - self.workspace.data_ptr()
+        if self.guard_bytes:
+            self.workspace[:self._ws_off].fill_(0xA5)
+            self.workspace[self._ws_off + nbytes.value:].fill_(0xA5)
         h0 = np.ascontiguousarray(inputs.init_hparams, dtype=np.float64)
         assert h0.shape == (self.N, self.nh)
         self.handle = C.c_void_p(None)
@@ -346,6 +349,7 @@ class Population:
 
     def guards_intact(self) -> bool:
         """True if the guard bands around the workspace (guard_bytes at construction) still hold their fill."""
+        assert self.guard_bytes > 0, "construct the population with guard_bytes > 0"
         self.synchronize()
         lo = self.workspace[:self._ws_off]
         hi = self.workspace[self._ws_off + self.workspace_bytes:]
