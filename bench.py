@@ -433,6 +433,25 @@ def main():
         if pr["copy"]["ms"] > 0:
             copy_gbs = 2 * n_cut * per_member / (pr["copy"]["ms"] * 1e-3) / 1e9
 
+    # ---- the other two phases of a ready point on their own (CUDA events on the library's stream, median of 5) ----
+    def phase_ms(fn):
+        ts = []
+        for _ in range(5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(pop.stream)
+            fn()
+            b.record(pop.stream)
+            pop.synchronize()
+            ts.append(a.elapsed_time(b))
+        return statistics.median(ts)
+
+    def ready_point():
+        pop.set_fitness(np.arange(cfg.n_members, dtype=np.float64))   # the same n_cut copies every time
+        pop.exploit_explore()
+    phases = {"eval_ms": phase_ms(pop.eval), "exploit_explore_ms": phase_ms(ready_point),
+              "note": "one pbt_eval / one pbt_exploit_explore of the whole population; both are inside the timed region "
+                      "once per ready interval"}
+
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -442,7 +461,7 @@ def main():
                    "timing": "CUDA-graph replay; per-kernel times from a second profiled pass" if two_pass else "per-launch events inside the timed region",
                    "l2": "inputs larger than L2: population state %.1f GB" % (pop.workspace_bytes / 1e9)},
         "e2e": e2e, "gpu_launches": int(launches[0]), "clocks": clocks, "roofline": roofline,
-        "kernels": kern, "class_ms": shares,
+        "kernels": kern, "class_ms": shares, "phases": phases,
         "exploit_copy": {"achieved": copy_gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"],
                          "frac": (copy_gbs / peaks["hbm_gbs"]) if copy_gbs else None},
     }
