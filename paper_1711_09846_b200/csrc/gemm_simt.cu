@@ -162,6 +162,70 @@ __global__ void __launch_bounds__(256) k_gemm_rowdot(GemmArgs g) {
   }
 }
 
+__device__ __forceinline__ void unpack_bf16x8(const uint4& w, float* f) {
+  const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) { f[2 * j] = __uint_as_float(u[j] << 16); f[2 * j + 1] = __uint_as_float(u[j] & 0xFFFF0000u); }
+}
+
+// The row-dot kernel for bf16 operands that are both K-major with K a multiple of 8: a lane takes 8 consecutive k
+// per trip with one 16-byte load per operand row.  The scalar form above is bound by instruction issue (address
+// arithmetic, conversion and one multiply-add per 2-byte load); this one issues about a third as many.
+template <int NT>
+__global__ void __launch_bounds__(256) k_gemm_rowdot_bf16x8(GemmArgs g) {
+  const int member = blockIdx.y, lane = threadIdx.x & 31;
+  const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (m >= g.M) return;
+  const bf16* __restrict__ A = reinterpret_cast<const bf16*>(g.A) + member * g.strideA + (long long)m * g.lda;
+  const bf16* __restrict__ B = reinterpret_cast<const bf16*>(g.B) + member * g.strideB;
+  float acc[NT];
+#pragma unroll
+  for (int n = 0; n < NT; ++n) acc[n] = 0.f;
+#pragma unroll 2
+  for (int k = lane * 8; k < g.K; k += 256) {
+    float a[8];
+    unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(A + k)), a);
+    const bf16* bk = B + k;
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      float b[8];
+      unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(bk + (long long)n * g.ldb)), b);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[n] = fmaf(a[j], b[j], acc[n]);
+    }
+  }
+#pragma unroll
+  for (int n = 0; n < NT; ++n) {
+    float v = acc[n];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (lane == n) store_one(g, member, m, n, epilogue_one(g, member, m, n, v, 1));
+  }
+}
+
+static bool rowdot_vec_ok(const GemmArgs& g) {
+  return g.in_dtype == kBF16 && !g.a_mn && !g.b_mn && g.N <= kSkinny && g.K % 8 == 0 && g.K >= 64 && g.lda % 8 == 0 &&
+         g.ldb % 8 == 0 && g.strideA % 8 == 0 && g.strideB % 8 == 0 && (((uintptr_t)g.A | (uintptr_t)g.B) & 15) == 0 &&
+         g.batch <= 65535;
+}
+// one instantiation per width: no predicated-off columns in the inner loop
+template <int NT>
+static void launch_rowdot_vec_n(const GemmArgs& g, cudaStream_t s) {
+  k_gemm_rowdot_bf16x8<NT><<<dim3((g.M + 7) / 8, g.batch), 256, 0, s>>>(g);
+}
+static void launch_rowdot_vec(const GemmArgs& g, cudaStream_t s) {
+  switch (g.N) {
+    case 1: launch_rowdot_vec_n<1>(g, s); break;   case 2: launch_rowdot_vec_n<2>(g, s); break;
+    case 3: launch_rowdot_vec_n<3>(g, s); break;   case 4: launch_rowdot_vec_n<4>(g, s); break;
+    case 5: launch_rowdot_vec_n<5>(g, s); break;   case 6: launch_rowdot_vec_n<6>(g, s); break;
+    case 7: launch_rowdot_vec_n<7>(g, s); break;   case 8: launch_rowdot_vec_n<8>(g, s); break;
+    case 9: launch_rowdot_vec_n<9>(g, s); break;   case 10: launch_rowdot_vec_n<10>(g, s); break;
+    case 11: launch_rowdot_vec_n<11>(g, s); break; case 12: launch_rowdot_vec_n<12>(g, s); break;
+    case 13: launch_rowdot_vec_n<13>(g, s); break; case 14: launch_rowdot_vec_n<14>(g, s); break;
+    case 15: launch_rowdot_vec_n<15>(g, s); break; default: launch_rowdot_vec_n<16>(g, s); break;
+  }
+}
+
 // Both operands MN-major (weight gradients), the short one of M, N at most ST <= 16: thread per index of the
 // long dimension, 16 slices of K per block combined in a fixed order.  LONG_A: M is the long dimension, else N.
 template <typename T, bool LONG_A, int ST>
@@ -202,6 +266,79 @@ __global__ void __launch_bounds__(512) k_gemm_colacc(GemmArgs g) {
   }
 }
 
+// The column-accumulate kernel for bf16 operands with the long dimension a multiple of 8: a thread owns 8
+// consecutive indices of the long dimension (one 16-byte load per batch row), 16 threads cover 128 of them, and the
+// block's 16 slices of K are combined in a fixed order, one short index at a time through 8 KB of shared memory.
+template <bool LONG_A, int ST>
+__global__ void __launch_bounds__(256) k_gemm_colacc_bf16x8(GemmArgs g) {
+  __shared__ float red[16][128 + 4];
+  const int member = blockIdx.y, lg = threadIdx.x & 15, ks = threadIdx.x >> 4;
+  const int L = LONG_A ? g.M : g.N;
+  const long long ldx = LONG_A ? g.lda : g.ldb, ldy = LONG_A ? g.ldb : g.lda;
+  const bf16* __restrict__ X = reinterpret_cast<const bf16*>(LONG_A ? g.A : g.B) + member * (LONG_A ? g.strideA : g.strideB);
+  const bf16* __restrict__ Y = reinterpret_cast<const bf16*>(LONG_A ? g.B : g.A) + member * (LONG_A ? g.strideB : g.strideA);
+  const int l0 = blockIdx.x * 128 + lg * 8;
+  float acc[8][ST];
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+#pragma unroll
+    for (int t = 0; t < ST; ++t) acc[j][t] = 0.f;
+  if (l0 < L) {
+#pragma unroll 2
+    for (int k = ks; k < g.K; k += 16) {
+      float x[8];
+      unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(X + (long long)k * ldx + l0)), x);
+      const bf16* yk = Y + (long long)k * ldy;
+#pragma unroll
+      for (int t = 0; t < ST; ++t) {
+        const float y = __bfloat162float(yk[t]);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j][t] = fmaf(x[j], y, acc[j][t]);
+      }
+    }
+  }
+  const int l = blockIdx.x * 128 + threadIdx.x;
+#pragma unroll
+  for (int t = 0; t < ST; ++t) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) red[ks][lg * 8 + j] = acc[j][t];
+    __syncthreads();
+    if (threadIdx.x < 128 && l < L) {
+      float v = 0.f;
+#pragma unroll
+      for (int q = 0; q < 16; ++q) v += red[q][threadIdx.x];
+      const int m = LONG_A ? l : t, n = LONG_A ? t : l;
+      store_one(g, member, m, n, epilogue_one(g, member, m, n, v, 1));
+    }
+    __syncthreads();
+  }
+}
+
+template <bool LONG_A, int ST>
+static void launch_colacc_vec_n(const GemmArgs& g, int L, cudaStream_t s) {
+  k_gemm_colacc_bf16x8<LONG_A, ST><<<dim3((L + 127) / 128, g.batch), 256, 0, s>>>(g);
+}
+template <bool LONG_A>
+static bool launch_colacc_vec(const GemmArgs& g, cudaStream_t s) {
+  const int L = LONG_A ? g.M : g.N, S = LONG_A ? g.N : g.M;
+  const long long ldx = LONG_A ? g.lda : g.ldb, sx = LONG_A ? g.strideA : g.strideB;
+  const void* X = LONG_A ? g.A : g.B;
+  if (g.in_dtype != kBF16 || L % 8 != 0 || L < 128 || ldx % 8 != 0 || sx % 8 != 0 || ((uintptr_t)X & 15) || g.batch > 65535)
+    return false;
+  switch (S) {   // one instantiation per width: no predicated-off columns in the inner loop
+    case 1: launch_colacc_vec_n<LONG_A, 1>(g, L, s); break;   case 2: launch_colacc_vec_n<LONG_A, 2>(g, L, s); break;
+    case 3: launch_colacc_vec_n<LONG_A, 3>(g, L, s); break;   case 4: launch_colacc_vec_n<LONG_A, 4>(g, L, s); break;
+    case 5: launch_colacc_vec_n<LONG_A, 5>(g, L, s); break;   case 6: launch_colacc_vec_n<LONG_A, 6>(g, L, s); break;
+    case 7: launch_colacc_vec_n<LONG_A, 7>(g, L, s); break;   case 8: launch_colacc_vec_n<LONG_A, 8>(g, L, s); break;
+    case 9: launch_colacc_vec_n<LONG_A, 9>(g, L, s); break;   case 10: launch_colacc_vec_n<LONG_A, 10>(g, L, s); break;
+    case 11: launch_colacc_vec_n<LONG_A, 11>(g, L, s); break; case 12: launch_colacc_vec_n<LONG_A, 12>(g, L, s); break;
+    case 13: launch_colacc_vec_n<LONG_A, 13>(g, L, s); break; case 14: launch_colacc_vec_n<LONG_A, 14>(g, L, s); break;
+    case 15: launch_colacc_vec_n<LONG_A, 15>(g, L, s); break; case 16: launch_colacc_vec_n<LONG_A, 16>(g, L, s); break;
+    default: return false;
+  }
+  return true;
+}
+
 // K <= 16: every output element is a short dot product.  A thread owns one column n: it keeps B(n, 0..K-1) in
 // registers and walks kSmallKRows rows of A, whose values every thread of the block reads alike (broadcast).
 constexpr int kSmallKRows = 32;
@@ -232,12 +369,12 @@ __global__ void __launch_bounds__(256) k_gemm_smallk(GemmArgs g) {
   }
 }
 
-// The same for bf16 operands and output with K <= 4 and N a multiple of 8: a thread produces 8 consecutive columns
+// The same for bf16 operands and output with N a multiple of 8: a thread produces 8 consecutive columns
 // of a row (16-byte loads of the weights and of the ReLU mask, one 16-byte store), the block's threads are spread
 // over the 32 rows x N / 8 column groups of its slab.  Same multiply-add order per element as the kernel above.
 template <bool B_MN>
 __global__ void __launch_bounds__(256) k_gemm_smallk_bf16x8(GemmArgs g) {
-  constexpr int KV = 4;
+  constexpr int KV = kSkinny;
   const int member = blockIdx.z, m0 = blockIdx.y * kSmallKRows;
   __shared__ float As[kSmallKRows][KV];
   const bf16* __restrict__ A = reinterpret_cast<const bf16*>(g.A) + member * g.strideA;
@@ -301,7 +438,7 @@ __global__ void __launch_bounds__(256) k_gemm_smallk_bf16x8(GemmArgs g) {
 }
 
 static bool smallk_vec_ok(const GemmArgs& g) {
-  if (g.in_dtype != kBF16 || g.out_dtype != kBF16 || g.K < 1 || g.K > 4 || g.N % 8 != 0) return false;
+  if (g.in_dtype != kBF16 || g.out_dtype != kBF16 || g.K < 1 || g.K > kSkinny || g.N % 8 != 0) return false;
   if (g.ldc % 8 || g.strideC % 8 || ((uintptr_t)g.C & 15)) return false;
   if (g.b_mn && (g.ldb % 8 || g.strideB % 8 || ((uintptr_t)g.B & 15))) return false;
   if (g.mask && (g.ldmask % 8 || g.strideMask % 8 || ((uintptr_t)g.mask & 15))) return false;
@@ -342,17 +479,21 @@ static bool launch_skinny(const GemmArgs& g, cudaStream_t s) {
     k_gemm_smallk<T><<<dim3((g.N + 255) / 256, (g.M + kSmallKRows - 1) / kSmallKRows, g.batch), 256, 0, s>>>(g);
     return true;
   }
+  if (rowdot_vec_ok(g)) {
+    launch_rowdot_vec(g, s);
+    return true;
+  }
   if (g.N <= kSkinny && !g.a_mn) {
     if (g.b_mn) launch_rowdot<T, true>(g, s);
     else launch_rowdot<T, false>(g, s);
     return true;
   }
   if (g.a_mn && g.b_mn && g.N <= kSkinny) {
-    launch_colacc<T, true>(g, s);
+    if (!launch_colacc_vec<true>(g, s)) launch_colacc<T, true>(g, s);
     return true;
   }
   if (g.a_mn && g.b_mn && g.M <= kSkinny) {
-    launch_colacc<T, false>(g, s);
+    if (!launch_colacc_vec<false>(g, s)) launch_colacc<T, false>(g, s);
     return true;
   }
   return false;
