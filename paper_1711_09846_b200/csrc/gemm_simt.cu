@@ -325,6 +325,8 @@ static bool launch_colacc_vec(const GemmArgs& g, cudaStream_t s) {
   const void* X = LONG_A ? g.A : g.B;
   if (g.in_dtype != kBF16 || L % 8 != 0 || L < 128 || ldx % 8 != 0 || sx % 8 != 0 || ((uintptr_t)X & 15) || g.batch > 65535)
     return false;
+  // one block per 128 indices and problem: worth it only when that fills the GPU (the scalar kernel has 4x the blocks)
+  if ((long long)((L + 127) / 128) * g.batch < 200) return false;
   switch (S) {   // one instantiation per width: no predicated-off columns in the inner loop
     case 1: launch_colacc_vec_n<LONG_A, 1>(g, L, s); break;   case 2: launch_colacc_vec_n<LONG_A, 2>(g, L, s); break;
     case 3: launch_colacc_vec_n<LONG_A, 3>(g, L, s); break;   case 4: launch_colacc_vec_n<LONG_A, 4>(g, L, s); break;
