@@ -44,6 +44,9 @@ case; hand-computed optimiser trajectories; energy-distance special cases;
 Philox known-answer vectors; Welch's test against printed critical values, the
 closed-form t distributions with 1 and 2 degrees of freedom and an independent
 library routine; resampling against the prior's range, rate and quantiles.
+Members at their own pace (`run_schedule`): every
+schedule over small populations against each member run alone, the lockstep
+schedule against `run`, own-clock `ready` against its definition.
 `Population.run` over a whole neural-network
 config has no external truth to compare with: parity unpinned beyond the pins
 of its parts.
@@ -116,6 +119,16 @@ def ready_members(step: int, interval: int, offsets=None, n: int = 0) -> np.ndar
     if offsets is None or len(offsets) == 0:
         return np.full(n, step > 0 and step % interval == 0, dtype=bool)
     return np.array([(step - int(o)) > 0 and (step - int(o)) % interval == 0 for o in offsets], dtype=bool)
+
+
+def ready_members_own(t, interval: int, offsets=None) -> np.ndarray:
+    """`ready(p, t, P)` of Algorithm 1 with every member on its own clock (Section 3: workers run asynchronously, each
+    counting its own steps): member m is ready when its OWN step count t[m], minus its offset, is a positive
+    multiple of `interval`.  With equal counts this is ready_members."""
+    t = np.asarray(t, dtype=np.int64)
+    o = np.zeros_like(t) if offsets is None or len(offsets) == 0 else np.asarray(offsets, dtype=np.int64)
+    d = t - o
+    return (d > 0) & (d % interval == 0)
 
 
 def _is_ready(ready, i) -> bool:
@@ -403,7 +416,7 @@ class Population:
         self.bf16 = cfg.dtype == "bf16_fp32master"
         self.master = np.float64 if self.toy else np.float32
         self.q = round_bf16 if self.bf16 else (lambda a: np.asarray(a, dtype=np.float64))
-        self.step_count = 0
+        self.t = np.zeros(self.N, dtype=np.int64)    # every member's own step count (Algorithm 1's t)
         self.round = 0
         self.H = np.array(inputs.init_hparams, dtype=np.float64).astype(self.master)
         self.fitness = np.zeros(self.N, dtype=self.master)
@@ -433,6 +446,15 @@ class Population:
             self.o2W, self.o2b = z(), zb()      # Adam v
             self.gW, self.gb = z(), zb()        # last gradient (for inspection)
 
+    @property
+    def step_count(self) -> int:
+        """Steps taken by the members this population holds; in lockstep they all agree."""
+        return int(self.t[self.members].max()) if len(self.members) else 0
+
+    @step_count.setter
+    def step_count(self, value: int):
+        self.t[:] = int(value)
+
     # ----- initial weights: U(-a, a), a = sqrt(6 / fan_in), biases zero ------
     def _init_weight(self, m, s, l, fo, fi):
         n = fo * fi
@@ -456,7 +478,7 @@ class Population:
         """Start row of this (member, step) window: a multiple of 128 drawn from
         the batch stream, so both sides read identical rows of the pool."""
         n_win = (pool_rows - batch) // WINDOW_ALIGN + 1
-        w = px.draw(self.seed, m, self.step_count, px.STREAM_BATCH, block)[word_index]
+        w = px.draw(self.seed, m, int(self.t[m]), px.STREAM_BATCH, block)[word_index]
         return WINDOW_ALIGN * ((int(w) * n_win) >> 32)
 
     # ----- network forward / backward for one member -------------------------
@@ -572,7 +594,7 @@ class Population:
         holds exactly."""
         eps = np.empty(B, dtype=np.float64)
         for b in range(B):
-            w = px.draw(self.seed, m, self.step_count, px.STREAM_INTERP, j * 65536 + (b >> 2))[b & 3]
+            w = px.draw(self.seed, m, int(self.t[m]), px.STREAM_INTERP, j * 65536 + (b >> 2))[b & 3]
             eps[b] = ((int(w) >> 9) + 0.5) / 8388608.0
         return eps
 
@@ -672,8 +694,10 @@ class Population:
         self._apply(m, 0, gW, gb, self._hp(m, "lr", 0.0))
 
     def step(self, k: int = 1, members=None, batch=None):
-        """k lockstep steps for all (or the given) members (Algorithm 1, line `step`)."""
-        members = self.members if members is None else members
+        """k steps for all (or the given) members (Algorithm 1, line `step`).  Each member counts its own steps:
+        what a member does at a step (which rows it trains on, its interpolation draws) is keyed by its own count
+        t[m], so a member that is held back and resumed later continues exactly where it stopped."""
+        members = self.members if members is None else [int(m) for m in members]
         for _ in range(k):
             for m in members:
                 if self.toy:
@@ -684,7 +708,7 @@ class Population:
                     self._step_gan(m)
                 else:
                     self._step_mlp(m, batch)
-            self.step_count += 1
+                self.t[m] += 1
 
     # ----- `eval` (Eq. 1): a function of the weights only ---------------------
     def eval_member(self, m) -> float:
@@ -786,6 +810,31 @@ class Population:
         for _ in range(total):
             self.step(1)
             ready = ready_members(self.step_count, cfg.ready_interval, offsets, self.N)
+            if ready.any():
+                self.eval()
+                if on_ready is not None:
+                    on_ready(self, "pre")
+                self.exploit_explore(None if ready.all() else ready)
+                if on_ready is not None:
+                    on_ready(self, "post")
+        return self.best()
+
+    # ----- members at their own pace (Section 3: asynchronous workers) ----------
+    def run_schedule(self, schedule, on_ready=None):
+        """Algorithm 1 with members advancing at different rates.  `schedule` is a sequence of boolean masks, one per
+        tick: the members that take one step in that tick (a worker that is pre-empted or slow simply sits out).
+        After a tick, a member that stepped and whose OWN count satisfies `ready` exploits and explores; the others
+        keep their record but are ranked and can be copied from.  Evaluating everybody at such a point equals
+        Algorithm 1's per-step eval, because a member that did not step has not changed."""
+        cfg = self.cfg
+        offsets = getattr(cfg, "ready_offsets", ())
+        for mask in schedule:
+            mask = np.asarray(mask, dtype=bool)
+            active = [m for m in self.members if mask[m]]
+            if not active:
+                continue
+            self.step(1, members=active)
+            ready = ready_members_own(self.t, cfg.ready_interval, offsets) & mask
             if ready.any():
                 self.eval()
                 if on_ready is not None:
