@@ -2,8 +2,12 @@
 """Throughput of the PBT hot path on synthetic data: population member-samples per second.
 
 One "step" = one lockstep pass of the whole hot path over one batch per member: batch
-window, forward, loss, backward, fused optimiser; at every ready point (the workload's
-ready interval) also evaluation and exploit/explore.  Prints ONE JSON line.
+window, forward, loss, backward, fused optimiser.  The timed region is K such steps plus
+exactly ONE ready point (evaluation, exploit / explore) whatever K is; it is repeated R
+times and the headline is the median repeat.  `ms_per_step` and `value` come from that
+whole region; `train_ms_per_step` is the K steps alone and `amortised_ms_per_step` adds
+the ready point at the workload's own ready interval.  After the headline the other
+benchmark populations are timed in compact form (`workloads`).  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--impl ours|reference]
 
@@ -107,8 +111,8 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-# DRAM bytes per parameter of the fused weight-gradient + Adam kernel, from one `ncu --set full` capture of a
-# small case (profiles/k_wgrad_adam_c5_8members.md), valid for the source file with this sha1 only.
+# DRAM bytes per parameter of the fused weight-gradient + Adam kernel, from one `ncu --set full` capture of an
+# 8-member case (the traffic is proportional to the members), valid for the source file with this sha1 only.
 _NCU_TRAFFIC = {"wgrad_adam": {"bytes_per_param": 25.41, "source": "paper_1711_09846_b200/csrc/wgrad_adam_tcgen05.cu",
                                "sha1": "361db330e5ece7f9d58438bc88611d1a377a3299"}}
 
@@ -243,20 +247,136 @@ def run_reference(args, cfg, inp):
     }))
 
 
+def _time_population(pop, cfg, steps, repeats, torch, barrier, two_pass):
+    """R timed repeats of [K training steps + ONE ready point (eval, exploit/explore)], CUDA events on the
+    library's stream.  Returns per-repeat totals, the split into training and ready-point time, launches of one
+    repeat and (from the last repeat when profiled in place, else from an extra profiled pass) per-class times."""
+    totals, trains, readys = [], [], []
+    launches = 0
+    prof = None
+    for r in range(repeats):
+        profiled = (not two_pass) and r == repeats - 1
+        barrier()
+        if profiled:
+            pop.profile_begin()
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        n = 0
+        e0.record(pop.stream)
+        pop.step(steps)
+        n += pop.launch_count()
+        e1.record(pop.stream)
+        pop.eval()
+        n += pop.launch_count()
+        pop.exploit_explore()
+        n += pop.launch_count()
+        e2.record(pop.stream)
+        if profiled:
+            prof = pop.profile_end()
+        barrier()
+        totals.append(e0.elapsed_time(e2))
+        trains.append(e0.elapsed_time(e1))
+        readys.append(e1.elapsed_time(e2))
+        launches = n
+    if prof is None:
+        pop.profile_begin()
+        pop.step(steps)
+        pop.eval()
+        pop.exploit_explore()
+        prof = pop.profile_end()
+    return {"total_ms": totals, "train_ms": trains, "ready_ms": readys, "launches": launches, "prof": prof}
+
+
+def _class_rooflines(cfg, prof, steps, peaks):
+    """Achieved rate of every kernel class against its roofline: algorithmic work of `steps` steps / summed event
+    time of the class (the ready point's few launches are in the class times too; its GEMM and loss work is not in
+    the numerator, which makes the fractions slightly conservative)."""
+    work = _algorithmic_work(cfg)
+    kern = {}
+
+    def add(name, bound, amount, unit, peak, src):
+        if prof[name]["launches"] and amount > 0 and prof[name]["ms"] > 0:
+            ach = amount * steps / (prof[name]["ms"] * 1e-3) / (1e12 if unit == "TFLOP/s" else 1e9)
+            nominal = {"TFLOP/s": 2250.0 if bound == "tensor" else None, "GB/s": 8000.0}[unit]
+            kern[name] = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                          "frac_of_nominal": (ach / nominal) if nominal else None, "nominal_peak": nominal, "traffic": None,
+                          "ms_per_step": prof[name]["ms"] / steps,
+                          "launches_per_step": prof[name]["launches"] / steps, "peak_source": src}
+
+    fused = prof["wgrad_adam"]["launches"] > 0
+    tensor = cfg.dtype == "bf16_fp32master"
+    gemm_flops = work["flops"] - (work["fused_flops"] if fused else 0.0)
+    add("gemm", "tensor" if tensor else "alu", gemm_flops, "TFLOP/s",
+        peaks["bf16_tflops_sustained"] if tensor else 2 * 148 * 128 * 1.965e9 / 1e12,
+        peaks["source"] + (" sustained bf16" if tensor else ": n/a, 148 SM x 128 FMA x 2 x 1.965 GHz fp32"))
+    if fused:
+        # HBM-bound: 12 B read + 14 B written per weight (master, two moments, bf16 shadow); the gradient stays on chip
+        add("wgrad_adam", "hbm", work["fused_params"] * 26.0, "GB/s", peaks["hbm_gbs"], peaks["source"])
+        if "wgrad_adam" in kern:
+            k = kern["wgrad_adam"]
+            per_step = prof["wgrad_adam"]["launches"] / steps
+            k["tflops"] = work["fused_flops"] * steps / (prof["wgrad_adam"]["ms"] * 1e-3) / 1e12
+            k["algorithmic_bytes_per_launch"] = work["fused_params"] * 26.0 / per_step
+            k["traffic"] = _ncu_traffic("wgrad_adam", work["fused_params"] / per_step)
+    opt_params = work["opt_params"] - (work["fused_params"] if fused else 0)
+    add("optimizer", "hbm", opt_params * work["opt_bytes_per_param"], "GB/s", peaks["hbm_gbs"], peaks["source"])
+    return kern
+
+
+def _median_spread(xs):
+    return statistics.median(xs), [min(xs), max(xs)]
+
+
+def _side_workload(pkg, torch, name, steps, repeats, peaks, device):
+    """One of the other benchmark populations: K graph-replayed steps + one ready point, R repeats; compact record."""
+    from workloads import get_config, make_inputs
+    cfg = get_config(name)
+    pop = pkg.Population(cfg, make_inputs(cfg), device=device)
+
+    def barrier():
+        torch.cuda.synchronize()
+    for _ in range(3):
+        pop.step(5)
+    pop.eval()
+    pop.exploit_explore()
+    t = _time_population(pop, cfg, steps, repeats, torch, barrier, two_pass=True)
+    train, spread = _median_spread([x / steps for x in t["train_ms"]])
+    ready = statistics.median(t["ready_ms"])
+    amort = train + ready / cfg.ready_interval
+    kern = _class_rooflines(cfg, t["prof"], steps, peaks)
+    cls_ms = {k: v["ms"] for k, v in t["prof"].items() if v["ms"] > 0}
+    tot = sum(cls_ms.values()) or 1.0
+    dom = max(cls_ms, key=cls_ms.get) if cls_ms else None
+    out = {"workload": cfg.name, "members": cfg.n_members, "batch": cfg.batch, "steps": steps, "repeats": repeats,
+           "train_ms_per_step": train, "train_ms_per_step_spread": spread, "ready_point_ms": ready,
+           "amortised_ms_per_step": amort, "ready_interval": cfg.ready_interval,
+           "member_samples_per_s": cfg.n_members * max(cfg.batch, 1) / (amort * 1e-3),
+           "launches_per_step": sum(v["launches"] for v in t["prof"].values()) / steps,
+           "dominant_class": dom, "dominant_share_of_kernel_time": (cls_ms[dom] / tot) if dom else None,
+           "dominant_frac_of_roofline": kern.get(dom, {}).get("frac") if dom else None,
+           "dominant_bound": kern.get(dom, {}).get("bound") if dom else None}
+    pop.close()
+    del pop
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--repeats", type=int, default=5, help="the timed region (K steps + one ready point) is run this often; the headline is the median")
     ap.add_argument("--workload", default="c5")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the compact figures of the other benchmark populations")
     ap.add_argument("--fuse-adam", type=int, default=-1, help="1/0: apply Adam inside the weight-gradient GEMM (default: the library's choice)")
     ap.add_argument("--graph", type=int, default=-1, help="1: time CUDA-graph replays and profile in a second pass; 0: profile the timed region; -1: by step length")
     ap.add_argument("--members", type=int, default=0, help="override the population size (profiling a small case)")
     ap.add_argument("--pool-rows", type=int, default=0, help="override the training-pool size (default: the workload's)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    args.repeats = max(args.repeats, 1)
 
     from workloads import get_config, make_inputs
     cfg = get_config(args.workload)
@@ -289,60 +409,38 @@ def main():
     pop = pkg.Population(cfg, inp, device=f"cuda:{local}", **kw)
     interval = cfg.ready_interval
 
-    def hot_path_step(i, launches):
-        pop.step(1)
-        launches[0] += pop.launch_count()
-        if (i + 1) % interval == 0:
-            pop.eval()
-            launches[0] += pop.launch_count()
-            pop.exploit_explore()
-            launches[0] += pop.launch_count()
-
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    scratch = [0]
     for i in range(args.warmup):
-        hot_path_step(i, scratch)
+        pop.step(1)
     # one ready point in the warm-up regardless of its length
     pop.eval()
     pop.exploit_explore()
 
     # Launch-bound workloads (a step of a few hundred microseconds) replay the step as a CUDA graph, which the
     # per-launch event records of the profiler would prevent: for those the timed region runs unprofiled and the
-    # per-kernel times come from a second, profiled pass of the same K steps.  Long steps are profiled in place.
+    # per-kernel times come from an extra, profiled pass of the same K steps.  Long steps are profiled in place
+    # (in the last repeat only, so the other repeats show what the event records cost).
     t_probe0 = time.perf_counter()
     pop.step(3)
     pop.synchronize()
     probe_ms = (time.perf_counter() - t_probe0) / 3 * 1e3
     two_pass = args.graph == 1 or (args.graph < 0 and probe_ms < 6.0)
 
-    # ---- timed region: device-resident inputs, CUDA events on the library's stream ----
+    # ---- timed region: device-resident inputs; K steps and exactly one ready point, R times ----
     sampler = ClockSampler(local)
     sampler.start()
-    barrier()
-    launches = [0]
-    if not two_pass:
-        pop.profile_begin()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(pop.stream)
-    for i in range(args.steps):
-        hot_path_step(i, launches)
-    e1.record(pop.stream)
-    if not two_pass:
-        prof = pop.profile_end()
-    barrier()
+    t = _time_population(pop, cfg, args.steps, args.repeats, torch, barrier, two_pass)
     clocks = sampler.stop()
-    ms = e0.elapsed_time(e1)
-    if two_pass:
-        pop.profile_begin()
-        for i in range(args.steps):
-            hot_path_step(i, [0])
-        prof = pop.profile_end()
-    ms = max_over_ranks(ms, f"cuda:{local}")
-    value = job_value(cfg, world, args.steps, ms)
+    prof = t["prof"]
+    total_ms, total_spread = _median_spread(t["total_ms"])
+    total_ms = max_over_ranks(total_ms, f"cuda:{local}")
+    train_ms, train_spread = _median_spread([x / args.steps for x in t["train_ms"]])
+    ready_ms = statistics.median(t["ready_ms"])
+    value = job_value(cfg, world, args.steps, total_ms)
 
     # ---- end to end: host buffers in, loss out, through the C ABI (MLP populations) ----
     e2e = None
@@ -363,7 +461,7 @@ def main():
             pop.step_host(xs[j % n_host], ys[j % n_host], loss_out)
         barrier()
         # every step: upload of that step's rows from pinned host memory (on the library's copy stream, overlapping
-        # the previous step), the step, and the read-back of the losses
+        # the previous step), the step, and the read-back of the losses; one ready point at the end
         t0 = time.perf_counter()
         pop.prefetch_host_batch(xs[0], ys[0])
         for j in range(e2e_steps):
@@ -371,50 +469,22 @@ def main():
             if j + 1 < e2e_steps:
                 pop.prefetch_host_batch(xs[(j + 1) % n_host], ys[(j + 1) % n_host])
             loss_out = pop.last_loss()
-            if (j + 1) % interval == 0:
-                pop.eval()
-                pop.exploit_explore()
+        pop.eval()
+        pop.exploit_explore()
         pop.synchronize()
         dt = time.perf_counter() - t0
         dt = max_over_ranks(dt, f"cuda:{local}")
         e2e = {"value": world * cfg.n_members * cfg.batch * e2e_steps / dt, "unit": UNIT,
                "h2d_bytes_per_step": int(xs[0].numel() * xs[0].element_size() + ys[0].numel() * ys[0].element_size()),
                "d2h_bytes_per_step": int(cfg.n_members * 2 * 4), "steps": e2e_steps,
-               "timing": "host wall clock; per step: H2D of the batch (pbt_prefetch_host_batch, overlapping the previous step), pbt_step_prefetched, D2H of the losses"}
+               "timing": "host wall clock; per step: H2D of the batch (pbt_prefetch_host_batch, overlapping the previous step), pbt_step_prefetched, D2H of the losses; one ready point (pbt_eval + pbt_exploit_explore) after the last step"}
     else:
         e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                "note": "host-fed steps exist for MLP populations only"}
 
-    # ---- roofline per kernel class, from the CUDA events recorded inside the timed region ----
+    # ---- roofline per kernel class, from CUDA events recorded around every launch ----
     peaks = _peaks()
-    work = _algorithmic_work(cfg)
-    kern = {}
-
-    def add(name, bound, amount, unit, peak, src):
-        if prof[name]["launches"] and amount > 0:
-            ach = amount * args.steps / (prof[name]["ms"] * 1e-3) / (1e12 if unit == "TFLOP/s" else 1e9)
-            nominal = {"TFLOP/s": 2250.0 if bound == "tensor" else None, "GB/s": 8000.0}[unit]
-            kern[name] = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
-                          "frac_of_nominal": (ach / nominal) if nominal else None, "nominal_peak": nominal, "traffic": None,
-                          "ms_per_step": prof[name]["ms"] / args.steps,
-                          "launches_per_step": prof[name]["launches"] / args.steps, "peak_source": src}
-
-    fused = prof["wgrad_adam"]["launches"] > 0
-    tensor = cfg.dtype == "bf16_fp32master"
-    gemm_flops = work["flops"] - (work["fused_flops"] if fused else 0.0)
-    add("gemm", "tensor" if tensor else "alu", gemm_flops, "TFLOP/s",
-        peaks["bf16_tflops_sustained"] if tensor else 2 * 148 * 128 * 1.965e9 / 1e12,
-        peaks["source"] + (" sustained bf16" if tensor else ": n/a, 148 SM x 128 FMA x 2 x 1.965 GHz fp32"))
-    if fused:
-        # HBM-bound: 12 B read + 14 B written per weight (master, two moments, bf16 shadow); the gradient stays on chip
-        add("wgrad_adam", "hbm", work["fused_params"] * 26.0, "GB/s", peaks["hbm_gbs"], peaks["source"])
-        if "wgrad_adam" in kern:
-            k = kern["wgrad_adam"]
-            k["tflops"] = work["fused_flops"] * args.steps / (prof["wgrad_adam"]["ms"] * 1e-3) / 1e12
-            k["algorithmic_bytes_per_launch"] = work["fused_params"] * 26.0 / k["launches_per_step"]
-            k["traffic"] = _ncu_traffic("wgrad_adam", work["fused_params"] / k["launches_per_step"])
-    opt_params = work["opt_params"] - (work["fused_params"] if fused else 0)
-    add("optimizer", "hbm", opt_params * work["opt_bytes_per_param"], "GB/s", peaks["hbm_gbs"], peaks["source"])
+    kern = _class_rooflines(cfg, prof, args.steps, peaks)
     shares = {k: v["ms"] for k, v in prof.items()}
     dominant = max(kern, key=lambda k: kern[k]["ms_per_step"]) if kern else None
     roofline = dict(kern[dominant], kernel=dominant) if dominant else None
@@ -433,7 +503,7 @@ def main():
         if pr["copy"]["ms"] > 0:
             copy_gbs = 2 * n_cut * per_member / (pr["copy"]["ms"] * 1e-3) / 1e9
 
-    # ---- the other two phases of a ready point on their own (CUDA events on the library's stream, median of 5) ----
+    # ---- the two phases of a ready point on their own (CUDA events on the library's stream, median of 5) ----
     def phase_ms(fn):
         ts = []
         for _ in range(5):
@@ -449,31 +519,60 @@ def main():
         pop.set_fitness(np.arange(cfg.n_members, dtype=np.float64))   # the same n_cut copies every time
         pop.exploit_explore()
     phases = {"eval_ms": phase_ms(pop.eval), "exploit_explore_ms": phase_ms(ready_point),
-              "note": "one pbt_eval / one pbt_exploit_explore of the whole population; both are inside the timed region "
-                      "once per ready interval"}
+              "note": "one pbt_eval / one pbt_exploit_explore of the whole population, timed on their own after the "
+                      "timed region; the timed region itself contains exactly one ready point (ready_point_ms)"}
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": {"bf16_fp32master": "bf16", "fp32": "f32", "fp64_toy": "f64"}[cfg.dtype], "data": "synthetic",
         "config": {"workload": cfg.name, "members": cfg.n_members, "batch": cfg.batch, "widths": [list(w) for w in cfg.widths],
                    "optimizer": cfg.optimizer, "ready_interval": interval, "parallelism": "replicas only" if world > 1 else "1 gpu",
-                   "timing": "CUDA-graph replay; per-kernel times from a second profiled pass" if two_pass else "per-launch events inside the timed region",
+                   "timed_region": f"{args.steps} lockstep steps + 1 ready point (pbt_eval, pbt_exploit_explore); "
+                                   f"median of {args.repeats} repeats",
+                   "timing": "CUDA-graph replay; per-kernel times from an extra profiled pass" if two_pass else "per-launch events in the last repeat",
                    "l2": "inputs larger than L2: population state %.1f GB" % (pop.workspace_bytes / 1e9)},
-        "e2e": e2e, "gpu_launches": int(launches[0]), "clocks": clocks, "roofline": roofline,
+        "repeats": args.repeats, "ms_per_step_spread": [x / args.steps for x in total_spread],
+        "train_ms_per_step": train_ms, "train_ms_per_step_spread": train_spread, "ready_point_ms": ready_ms,
+        "amortised_ms_per_step": train_ms + ready_ms / interval,
+        "amortised_value": world * cfg.n_members * max(cfg.batch, 1) / ((train_ms + ready_ms / interval) * 1e-3),
+        "e2e": e2e, "gpu_launches": int(t["launches"]), "clocks": clocks, "roofline": roofline,
         "kernels": kern, "class_ms": shares, "phases": phases,
         "exploit_copy": {"achieved": copy_gbs, "unit": "GB/s", "peak": peaks["hbm_gbs"],
                          "frac": (copy_gbs / peaks["hbm_gbs"]) if copy_gbs else None},
     }
+    pop.close()
+    del pop
+    torch.cuda.empty_cache()
+
+    if rank == 0 and world == 1 and not args.no_workloads:
+        side = {}
+        for name in ("c1", "c2", "c3", "c4", "c4_wgan", "c5"):
+            if get_config(name).name == cfg.name:
+                continue
+            try:
+                side[name] = _side_workload(pkg, torch, name, 200 if name != "c5" else 25, 3, peaks, f"cuda:{local}")
+            except Exception as ex:      # a side figure must not take the headline down with it
+                side[name] = {"error": repr(ex)}
+        result["workloads"] = side
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         members, steps = _oracle_budget(cfg)
         small = cfg.replace(pool_rows=min(cfg.pool_rows, 4096), eval_batch=min(cfg.eval_batch, 512))
-        v, dt = _oracle_sample(small, make_inputs(small), members, steps)
+        small_inp = make_inputs(small)
+        v, dt = _oracle_sample(small, small_inp, members, steps)
         result["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": _cpu_count_used(), "kind": "oracle",
                                   "sample": f"{members} of {cfg.n_members} members x {steps} step(s), {dt:.1f} s, "
                                             f"float64 NumPy oracle, training step only"}
-    pop.close()
+        try:
+            from threadpoolctl import threadpool_limits
+            with threadpool_limits(limits=1):
+                m1 = max(1, members // 8)
+                v1, dt1 = _oracle_sample(small, small_inp, m1, 1)
+            result["cpu_baseline"]["single_thread"] = {"value": v1, "unit": UNIT, "cores": 1,
+                                                       "sample": f"{m1} member(s) x 1 step, {dt1:.1f} s"}
+        except Exception as ex:
+            result["cpu_baseline"]["single_thread"] = {"error": repr(ex)}
     if rank == 0:
         print(json.dumps(result))
     if world > 1:

@@ -9,7 +9,7 @@ from oracle import pbt_oracle as O
 from workloads import configs as C
 from workloads import get_config, make_inputs
 
-from util import TOL, assert_state_close, critic_offset, rel_err, tensor_slices
+from util import TOL, assert_kept_fractions, assert_state_close, critic_offset, rel_err, tensor_slices
 
 pytestmark = pytest.mark.gpu
 
@@ -52,6 +52,7 @@ def test_full_size_step_eval_and_exploit(pkg, name, sample, pool, eval_rows):
         got[0] += critic_offset(cfg, g)
         want[0] += critic_offset(cfg, c)
         np.testing.assert_allclose(got, want, rtol=ftol, atol=1e-5)
+    assert_kept_fractions(name, 0.98, cfg)
 
     gpu.eval()
     cpu.eval(sample)

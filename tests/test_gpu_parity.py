@@ -10,7 +10,7 @@ from oracle import pbt_oracle as O
 from workloads import configs as C
 from workloads import get_config, make_inputs
 
-from util import TOL, assert_state_close, critic_offset, oracle_history_arrays, push_oracle_state, rel_err
+from util import TOL, assert_kept_fractions, assert_state_close, critic_offset, oracle_history_arrays, push_oracle_state, rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -161,6 +161,32 @@ def test_toy_with_tournament_matches_oracle(pkg):
     gpu.close()
 
 
+def test_toy_select_explore_bit_exact_at_the_largest_population(pkg):
+    """The fp64 instantiation of the select / explore kernel with one member per thread at the largest population
+    the library takes (1024), against the oracle, bit for bit."""
+    n = 1024
+    cfg = get_config("c1").replace(n_members=n, flags=C.COPY_WEIGHTS | C.COPY_HPARAMS | C.EXPLORE, name="toy1024")
+    inp = make_inputs(cfg)
+    h0 = np.random.default_rng(3).random((n, cfg.nh)) + 0.5
+    inp = type(inp)(**{**inp.__dict__, "init_hparams": h0})
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    rng = np.random.default_rng(4)
+    for rnd in range(3):
+        gpu.step(2)
+        cpu.step(2)
+        f = np.round(rng.standard_normal(n), 2)          # ties included
+        cpu.fitness[:] = f
+        gpu.set_fitness(f)
+        gpu.exploit_explore()
+        src = cpu.exploit_explore()
+        assert np.array_equal(gpu.copy_map(), src)
+        assert np.array_equal(gpu.hparams(), cpu.H)
+        assert np.array_equal(gpu.fitness(), cpu.fitness)
+        for m in range(0, n, 37):
+            assert np.array_equal(gpu.get_state(m)["w"], cpu.theta[m])
+    gpu.close()
+
+
 @pytest.mark.parametrize("flags", [0, C.COPY_WEIGHTS, C.COPY_HPARAMS | C.EXPLORE, C.COPY_WEIGHTS | C.EXPLORE])
 def test_flag_variants_bit_exact(pkg, flags):
     cfg = _tiny_cfg(10, C.FP32, flags=flags, num=2, den=5)
@@ -255,24 +281,26 @@ def test_checkpoint_resume_is_bit_exact(pkg, name, tmp_path):
     the decisions of the following ready points, bit for bit."""
     cfg = get_config(name)
     inp = make_inputs(cfg)
+    iv = cfg.ready_interval
     a = pkg.Population(cfg, inp)
-    a.run(2 * cfg.ready_interval)
+    a.run(2 * iv + 1)                       # stops in the middle of an interval
     path = str(tmp_path / "pop.npz")
     a.save(path)
     b = pkg.Population(cfg, inp)
     b.load(path)
-    for pop in (a, b):
-        for _ in range(2):
-            pop.step(cfg.ready_interval)
-            pop.eval()
-            pop.exploit_explore()
-    sa, sb = a.state_dict(), b.state_dict()
-    assert set(sa) == set(sb)
-    for key in sa:
-        assert np.array_equal(sa[key], sb[key], equal_nan=True), (name, key)
-    assert np.array_equal(a.copy_map(), b.copy_map())
-    a.close()
-    b.close()
+    c = pkg.Population(cfg, inp)            # never interrupted
+    for pop in (a, b, c):
+        pop.run(4 * iv + 1)                 # absolute target: the ready points fall on the same steps for all three
+    sa = a.state_dict()
+    for other in (b, c):
+        so = other.state_dict()
+        assert set(sa) == set(so)
+        for key in sa:
+            assert np.array_equal(sa[key], so[key], equal_nan=True), (name, key)
+        assert np.array_equal(a.copy_map(), other.copy_map())
+    assert int(sa["step"]) == 4 * iv + 1
+    for pop in (a, b, c):
+        pop.close()
 
 
 @pytest.mark.parametrize("name", ["c2_mini", "c3_mini", "c4_mini", "c4_mini_wgan", "c5_mini", "c3_mid", "c5_mid", "c4_mid_wgan",
@@ -413,6 +441,7 @@ def test_step_eval_exploit_parity(pkg, name):
                 assert np.array_equal(gc, cc) and np.array_equal(gh, ch)
         # every step starts from identical state: training is chaotic, parity is per step
         push_oracle_state(gpu, cpu)
+    assert_kept_fractions(name, 0.98, cfg)
     gpu.close()
 
 
@@ -554,6 +583,72 @@ def test_host_fed_steps_plain_and_prefetched_agree(pkg):
             assert np.array_equal(sa[key], sb[key])
     a.close()
     b.close()
+
+
+def test_ready_point_is_enqueue_only_under_the_tournament_rule(pkg):
+    """step -> eval -> ready point (binary tournament, whose copies may need several passes) -> step, enqueued
+    behind a busy stream: none of the calls waits for the device (the number of copy passes stays on the device),
+    and the result is the oracle's."""
+    import torch
+    cfg = _tiny_cfg(24, C.FP32).replace(exploit="tournament")
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    gpu.step(1)
+    cpu.step(1)
+    push_oracle_state(gpu, cpu)
+    gpu.synchronize()
+    done = torch.cuda.Event()
+    with torch.cuda.stream(gpu.stream):
+        torch.cuda._sleep(int(1.5e9))            # keeps the stream busy for most of a second
+    gpu.step(2)
+    gpu.eval()
+    gpu.exploit_explore()
+    gpu.step(1)
+    done.record(gpu.stream)
+    assert not done.query(), "a call of the training loop waited for the device"
+    gpu.synchronize()
+    cpu.step(2)
+    cpu.eval()
+    src = cpu.exploit_explore()
+    cpu.step(1)
+    assert np.array_equal(gpu.copy_map(), src)
+    assert (src != np.arange(cfg.n_members)).sum() > 0
+    assert np.array_equal(gpu.hparams(), cpu.H.astype(np.float64))
+    for m in range(cfg.n_members):
+        g = gpu.get_state(m)
+        assert g["step"] == 4 and g["round"] == 1
+        assert_state_close(cfg, g, cpu.get_flat(m), ("w", "opt1"), {"w": 1e-5, "opt1": 1e-4}, what="enqueue_only")
+    gpu.close()
+
+
+def test_prefetched_steps_after_pool_steps_match_the_oracle(pkg):
+    """pbt_step(k) followed at once by two prefetched host-fed steps without waiting: the uploads must not land in
+    row buffers that the still-running pool steps read (the spare buffer pair of the second upload is the pair the
+    pool steps used)."""
+    import torch
+    cfg = get_config("c2_mini")
+    inp = make_inputs(cfg)
+    gpu, cpu = pkg.Population(cfg, inp), O.Population(cfg, inp)
+    rng = np.random.default_rng(11)
+    xs = [rng.standard_normal((cfg.batch, cfg.widths[0][0])).astype(np.float32) for _ in range(2)]
+    ys = [rng.standard_normal((cfg.batch, 1)).astype(np.float32) for _ in range(2)]
+    hx = [torch.from_numpy(np.tile(x, (cfg.n_members, 1, 1))).contiguous().pin_memory() for x in xs]
+    hy = [torch.from_numpy(np.tile(y, (cfg.n_members, 1, 1))).contiguous().pin_memory() for y in ys]
+    k = 40
+    gpu.step(k)
+    gpu.prefetch_host_batch(hx[0], hy[0])
+    gpu.step_prefetched(wait=False)
+    gpu.prefetch_host_batch(hx[1], hy[1])
+    gpu.step_prefetched(wait=False)
+    gpu.synchronize()
+    cpu.step(k)
+    cpu.step(1, batch=(xs[0], ys[0]))
+    cpu.step(1, batch=(xs[1], ys[1]))
+    for m in range(cfg.n_members):
+        g = gpu.get_state(m)
+        assert g["step"] == k + 2
+        assert_state_close(cfg, g, cpu.get_flat(m), ("w",), {"w": 1e-5}, what="prefetch_after_pool_steps")
+    gpu.close()
 
 
 def test_invalid_arguments_are_reported_not_fatal(pkg):

@@ -4,8 +4,9 @@ Some hosts may not allocate device memory at all (the application owns the devic
 its own arena and hands plug-ins only the buffers it chooses).  For them the library has
 pbt_energy_fitness_static, whose reduction scratch is a fixed array inside the library.
 This file checks, through the C ABI, that it gives the same fitness as pbt_eval does for a
-GAN population, on two calls in a row (the second call reuses the scratch the first one
-left dirty), and that it refuses problems larger than its built-in scratch.
+GAN population and as the CPU oracle's energy distance gives for the same points, on two
+calls in a row (the second call reuses the scratch the first one left dirty), and that it
+refuses problems larger than its built-in scratch.
 
 Named so that pytest collects it last.
 """
@@ -14,6 +15,7 @@ import ctypes as C
 import numpy as np
 import pytest
 
+from oracle import pbt_oracle as O
 from workloads import get_config, make_inputs
 
 pytestmark = pytest.mark.gpu
@@ -56,6 +58,7 @@ def test_static_scratch_scorer_matches_eval_twice():
 
     z = inp.x_eval[:, :2].astype(np.float32)                   # bf16-representable, so G(z) is exact
     x = np.stack([s * z for s in scales]).astype(np.float32)   # [members, n, 2]
+    oracle = np.array([-O.energy_distance_to_ring(xm.astype(np.float64)) for xm in x])   # fitness = -energy distance
     x_dev = torch.from_numpy(x).cuda().contiguous()
     out = torch.full((cfg.n_members,), float("nan"), device="cuda", dtype=torch.float32)
     stream = torch.cuda.Stream()
@@ -64,6 +67,7 @@ def test_static_scratch_scorer_matches_eval_twice():
     pkg.energy_fitness_static(x_dev, out, stream)
     stream.synchronize()
     np.testing.assert_allclose(out.cpu().numpy(), expect, rtol=1e-6, atol=1e-7)
+    np.testing.assert_allclose(out.cpu().numpy(), oracle, rtol=1e-5, atol=1e-6)
 
     # second call straight after, other data, same shared scratch
     x_rev = torch.from_numpy(x[::-1].copy()).cuda().contiguous()
@@ -72,6 +76,7 @@ def test_static_scratch_scorer_matches_eval_twice():
     pkg.energy_fitness_static(x_rev, out2, stream)
     stream.synchronize()
     np.testing.assert_allclose(out2.cpu().numpy(), expect[::-1], rtol=1e-6, atol=1e-7)
+    np.testing.assert_allclose(out2.cpu().numpy(), oracle[::-1], rtol=1e-5, atol=1e-6)
     pop.close()
 
 
@@ -87,4 +92,9 @@ def test_static_scratch_scorer_rejects_oversize_and_bad_arguments():
     assert b"scratch" in lib.pbt_last_error(None)
     assert lib.pbt_energy_fitness_static(None, 16, 1, p, None) == 1
     assert lib.pbt_energy_fitness_static(p, 0, 1, p, None) == 1
+    # sizes that would overflow 32-bit arithmetic, more members than a grid dimension holds, host memory
+    assert lib.pbt_energy_fitness_static(p, 2**31 - 1, 1, p, None) == 3
+    assert lib.pbt_energy_fitness_static(p, 16, 65536, p, None) == 3
+    host = np.zeros(64, dtype=np.float32)
+    assert lib.pbt_energy_fitness_static(C.c_void_p(host.ctypes.data), 16, 1, p, None) == 1
     torch.cuda.synchronize()
