@@ -15,9 +15,18 @@
  *     "host" pointers are ordinary host memory.  The library allocates no device
  *     memory: the caller passes one workspace (size from pbt_query_workspace)
  *     and the data pools, and keeps both alive until pbt_destroy.
- *   - All work is enqueued on the stream given to pbt_create.  Calls that
- *     return data to the host (pbt_get_*) synchronise that stream; the others
- *     return as soon as the work is enqueued.
+ *   - All work is enqueued on the stream given to pbt_create.  The calls of
+ *     the training loop only enqueue and return: pbt_step, pbt_eval,
+ *     pbt_step_subset, pbt_exploit_explore(_ready) under every exploit rule, pbt_set_batch,
+ *     pbt_prefetch_host_batch, pbt_step_prefetched / pbt_step_host without a
+ *     loss buffer, pbt_grouped_gemm.  Calls that move data between ordinary
+ *     host memory and the device synchronise that stream before they return:
+ *     pbt_create, every pbt_get_*, and pbt_set_state / pbt_set_fitness /
+ *     pbt_set_hparams / pbt_set_history (their host arguments may be reused
+ *     at once).
+ *   - A handle belongs to the device that was current in pbt_create; make
+ *     that device current for every later call on it.  Several handles on
+ *     several devices may live in one process.
  *   - There is no CPU fallback: without a CUDA device every call that would
  *     launch work fails with PBT_ERR_CUDA.
  *
@@ -124,6 +133,10 @@ typedef struct pbt_spec {
   int32_t fuse_adam; /* 1: apply Adam inside the epilogue of tensor-core weight-gradient GEMMs (the gradient of those
                         layers never goes to HBM); 0: weight gradients are written once and one streaming pass over
                         the slabs applies the update.  Results are bit-identical; only the traffic pattern differs. */
+  int32_t serial_launches; /* 0 (default): kernels are launched with programmatic stream serialization: a kernel may be
+                        scheduled while its predecessor drains and waits on the device until the predecessor's results
+                        are visible (same dependences as stream order, less launch latency); 1: plain stream order.
+                        Results are bit-identical.  The setting of the handle used last applies to the process. */
   int32_t exploit_rule; /* 0: truncation selection (Section 4.1.1 (b)); 1: binary tournament (Section 4.3.1 (b)): every
                            member draws one other member uniformly and copies it if its fitness is strictly higher;
                            2: t-test selection (Section 4.1.1, exploit (a)): one other member drawn uniformly is
@@ -170,8 +183,9 @@ typedef struct pbt_data {
  * Every pointer is caller-owned host memory and may be NULL to skip that part.
  * w/opt1/opt2/grad hold P elements in flat order: float (double for the toy).
  * `grad` (last gradient applied) is filled by pbt_get_state, ignored by set.
- * step and round are population-wide (lockstep); setting them through any
- * member sets them for the population.
+ * step is the member's own step count t (equal for all members as long as only
+ * pbt_step is used); round, the number of ready points passed, is population-wide:
+ * setting it through any member sets it for the population.
  */
 typedef struct pbt_state_view {
   void* w;
@@ -218,6 +232,19 @@ int pbt_destroy(pbt_t* p);
  * Toy: one gradient-ascent step on the surrogate objective.
  */
 int pbt_step(pbt_t* p, int k);
+
+/*
+ * Members at their own pace (Algorithm 1 is a loop per member; Section 3 lets the workers run asynchronously,
+ * and Appendix A.1's partial synchrony exists to tolerate workers that are pre-empted): k steps for the members
+ * whose byte in active_host (n_members bytes of host memory) is non-zero, none for the others, whose records
+ * stay untouched.  Every member counts its own steps t (pbt_state_view.step): the rows it trains on and its
+ * interpolation draws are keyed by (member, its own t), so a member that sat out some calls continues exactly
+ * where it stopped, and a call with every byte set equals pbt_step(k).  `ready(p, t, P)` for such a population
+ * is a matter of the member's own t; give the ready members to pbt_exploit_explore_ready.  Consecutive active
+ * members share their launches (one pass of the step's kernels per run of consecutive active members).
+ * PBT_ERR_STATE if a batch set by pbt_set_batch is pending.  Only enqueues.
+ */
+int pbt_step_subset(pbt_t* p, const uint8_t* active_host, int k);
 
 /*
  * p <- eval(theta) for every member (Eq. 1): minus the held-out loss, the toy's
@@ -378,8 +405,10 @@ int pbt_selftest_bounded_wait(void* status_device, int polls, void* stream);
  * The partial sums of the reduction live in a fixed 1 MiB array inside the library image
  * (held by every GPU that loads the library until the process exits), so the call performs
  * no cudaMalloc / cudaFree.  Limits and rules:
- *   - n_members * 2 * ceil(n / 256) must not exceed 131072, else PBT_ERR_WORKSPACE with a
- *     message naming the size; NULL pointers or non-positive sizes give PBT_ERR_INVALID_ARG;
+ *   - n_members * 2 * ceil(n / 256) must not exceed 131072 and n_members must not exceed 65535,
+ *     else PBT_ERR_WORKSPACE with a message naming the size; NULL pointers, non-positive sizes,
+ *     or buffers that are not device memory of the CURRENT device give PBT_ERR_INVALID_ARG
+ *     (the scratch that is used, and the GPU the kernels run on, are the current device's);
  *   - the array is shared by all calls and keeps the previous call's contents; nothing in it
  *     needs clearing, every slot read is first rewritten by the same call;
  *   - calls that overlap on the GPU (other streams or threads) race on that array: serialise them;

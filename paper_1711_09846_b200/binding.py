@@ -38,7 +38,7 @@ class PbtSpec(C.Structure):
         ("slot_lr", C.c_int32), ("slot_lr_d", C.c_int32), ("slot_momentum", C.c_int32),
         ("slot_beta1", C.c_int32), ("slot_wd", C.c_int32),
         ("perturb_mask", C.c_uint32), ("flags", C.c_uint32),
-        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("exploit_rule", C.c_int32),
+        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("serial_launches", C.c_int32), ("exploit_rule", C.c_int32),
         ("explore_rule", C.c_int32), ("prior_kind", C.c_int32 * PBT_MAX_NH),
         ("const_lr", C.c_double), ("const_momentum", C.c_double), ("const_beta1", C.c_double),
         ("const_beta2", C.c_double), ("const_eps", C.c_double), ("const_wd", C.c_double),
@@ -76,7 +76,7 @@ class PbtGemmDesc(C.Structure):
 
 
 EXPORTS = [
-    "pbt_query_workspace", "pbt_param_count", "pbt_create", "pbt_destroy", "pbt_step", "pbt_eval",
+    "pbt_query_workspace", "pbt_param_count", "pbt_create", "pbt_destroy", "pbt_step", "pbt_step_subset", "pbt_eval",
     "pbt_exploit_explore", "pbt_exploit_explore_ready", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
     "pbt_get_history", "pbt_set_history",
     "pbt_get_hparams", "pbt_set_hparams", "pbt_get_copy_map", "pbt_get_best", "pbt_get_last_loss",
@@ -108,6 +108,7 @@ def load_library() -> C.CDLL:
                                C.POINTER(PbtData), vp, C.c_size_t, vp]
     lib.pbt_destroy.argtypes = [vp]
     lib.pbt_step.argtypes = [vp, C.c_int]
+    lib.pbt_step_subset.argtypes = [vp, C.POINTER(C.c_uint8), C.c_int]
     lib.pbt_eval.argtypes = [vp]
     lib.pbt_exploit_explore.argtypes = [vp]
     lib.pbt_exploit_explore_ready.argtypes = [vp, C.POINTER(C.c_uint8)]
@@ -146,7 +147,7 @@ class PbtError(RuntimeError):
         self.code = code
 
 
-def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True) -> PbtSpec:
+def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True, serial_launches: bool = False) -> PbtSpec:
     """Translate a declarative population description (see workloads.configs.PBTConfig) into pbt_spec."""
     s = PbtSpec()
     s.n_members = cfg.n_members
@@ -174,6 +175,7 @@ def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True) -> Pb
     s.flags = cfg.flags
     s.trunc_num, s.trunc_den = cfg.trunc_num, cfg.trunc_den
     s.keep_grad = 1 if keep_grad else 0
+    s.serial_launches = 1 if serial_launches else 0
     s.exploit_rule = {"truncation": 0, "tournament": 1, "ttest": 2}[getattr(cfg, "exploit", "truncation")]
     s.explore_rule = {"perturb": 0, "resample": 1}[getattr(cfg, "explore", "perturb")]
     s.ttest_alpha = getattr(cfg, "ttest_alpha", 0.05)
@@ -266,7 +268,7 @@ class Population:
     """One population living on one GPU.  Thin wrapper over the pbt_* calls."""
 
     def __init__(self, cfg, inputs, seed: Optional[int] = None, device: str = "cuda:0", keep_grad: bool = False,
-                 fuse_adam: bool = True, guard_bytes: int = 0):
+                 fuse_adam: bool = True, guard_bytes: int = 0, serial_launches: bool = False):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -275,7 +277,7 @@ class Population:
         self.cfg = cfg
         self.device = torch.device(device)
         self.seed = int(cfg.seed if seed is None else seed)
-        self.spec = spec_from_config(cfg, keep_grad, fuse_adam)
+        self.spec = spec_from_config(cfg, keep_grad, fuse_adam, serial_launches or bool(os.environ.get("PBT_SERIAL_LAUNCHES")))
         self.N, self.nh = cfg.n_members, cfg.nh
         self.toy = cfg.model == "toy_quadratic"
         torch.cuda.set_device(self.device)
@@ -358,6 +360,12 @@ class Population:
     # ----- the hot path ---------------------------------------------------
     def step(self, k: int = 1):
         self._check(self.lib.pbt_step(self.handle, int(k)))
+
+    def step_subset(self, active, k: int = 1):
+        """k steps for the members whose entry of `active` (bools, one per member) is set; the others sit out."""
+        mask = np.ascontiguousarray(np.asarray(active, dtype=bool).astype(np.uint8))
+        assert mask.shape == (self.cfg.n_members,)
+        self._check(self.lib.pbt_step_subset(self.handle, mask.ctypes.data_as(C.POINTER(C.c_uint8)), int(k)))
 
     def eval(self):
         self._check(self.lib.pbt_eval(self.handle))
@@ -519,7 +527,6 @@ class Population:
             out[cls] = {"ms": ms.value, "launches": n.value}
         return out
 
-    # ----- Algorithm 1 in partial synchrony ---------------------------------
     # ----- checkpoint / resume (Appendix A.1: members checkpoint themselves; here the whole population record) -----
     def state_dict(self) -> Dict[str, np.ndarray]:
         """The population record (theta, h, p, t) of every member plus optimiser state, score histories and the
@@ -554,6 +561,7 @@ class Population:
         with np.load(path) as z:
             self.load_state_dict({k: z[k] for k in z.files})
 
+    # ----- Algorithm 1 in partial synchrony ---------------------------------
     def _ready_point(self, step, ready, log):
         """eval, exploit / explore and, if asked, one record of the ready point (Section 4.4's analyses are made
         from such records: score and hyperparameter traces, who copied whom)."""
@@ -577,30 +585,25 @@ class Population:
         return anc
 
     def run(self, total_steps: Optional[int] = None, log=None) -> int:
-        """Algorithm 1 in partial synchrony: steps, and a ready point whenever `ready` holds.  `log`: a list (or a
-        bounded collections.deque) that receives one record per ready point; each record costs four small
-        device-to-host reads."""
+        """Algorithm 1 in partial synchrony: steps, and a ready point whenever `ready` holds.  `total_steps` is the
+        ABSOLUTE step count to reach (default: the configuration's): the schedule is taken from the population's own
+        step counter, so a population restored from a checkpoint (Appendix A.1) in the middle of an interval has its
+        ready points at the same steps as the run that was never interrupted.  `log`: a list (or a bounded
+        collections.deque) that receives one record per ready point; each record costs four small device-to-host
+        reads."""
         cfg = self.cfg
         total = cfg.total_steps if total_steps is None else total_steps
-        done = 0
-        offsets = tuple(getattr(cfg, "ready_offsets", ()))
-        if offsets:
-            # staggered ready points (Algorithm 1's `ready`, member by member): member m is ready when
-            # step - offsets[m] is a positive multiple of the interval; run to the next step at which anybody is
-            iv = cfg.ready_interval
-            while done < total:
-                nxt = min(o + iv * ((done - o) // iv + 1) if done >= o else o + iv for o in offsets)
-                k = min(nxt, total) - done
-                self.step(k)
-                done += k
-                ready = [(done - o) > 0 and (done - o) % iv == 0 for o in offsets]
-                if any(ready):
-                    self._ready_point(done, None if all(ready) else ready, log)
-            return self.best()
+        done = int(self.get_state(0)["step"])
+        offsets = tuple(getattr(cfg, "ready_offsets", ())) or (0,) * cfg.n_members
+        iv = cfg.ready_interval
         while done < total:
-            k = min(cfg.ready_interval, total - done)
+            # member m is ready when step - offsets[m] is a positive multiple of the interval (Algorithm 1's `ready`,
+            # member by member; all offsets zero = everybody together): run to the next step at which anybody is
+            nxt = min(o + iv * ((done - o) // iv + 1) if done >= o else o + iv for o in offsets)
+            k = min(nxt, total) - done
             self.step(k)
             done += k
-            if done % cfg.ready_interval == 0:
-                self._ready_point(done, None, log)
+            ready = [(done - o) > 0 and (done - o) % iv == 0 for o in offsets]
+            if any(ready):
+                self._ready_point(done, None if all(ready) else ready, log)
         return self.best()

@@ -76,14 +76,34 @@ extern "C" int pbt_energy_fitness_static(const float* x_device, int n, int n_mem
     pbt::set_last_error("n and n_members must be positive");
     return PBT_ERR_INVALID_ARG;
   }
-  const long long need = (long long)n_members * pbt::energy_partial_count(n);
-  if (need > kScratchDoubles) {
+  // sizes are checked in 64-bit arithmetic before anything derived from them is used: 2 * ceil(n / 256) partial sums
+  // per member (the layout of launch_energy_distance), at most 65535 members (the grid's second dimension)
+  const long long need = (long long)n_members * (2ll * (((long long)n + 255) / 256));
+  if (need > kScratchDoubles || n_members > 65535) {
     char msg[256];
     snprintf(msg, sizeof(msg),
              "problem too large for the built-in scratch: n_members * 2 * ceil(n / 256) = %lld doubles, limit %d "
              "(use pbt_eval with a caller-provided workspace instead)", need, kScratchDoubles);
     pbt::set_last_error(msg);
     return PBT_ERR_WORKSPACE;
+  }
+  // The scratch address that is looked up belongs to the CURRENT device, and the kernels run there: both buffers
+  // must live on it too (a buffer of another GPU would be dereferenced as peer memory).
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    pbt::set_last_error("no current CUDA device");
+    return PBT_ERR_CUDA;
+  }
+  const void* bufs[2] = {x_device, fitness_out_device};
+  for (const void* b : bufs) {
+    cudaPointerAttributes attr;
+    const cudaError_t pe = cudaPointerGetAttributes(&attr, b);
+    if (pe != cudaSuccess || (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged) ||
+        (attr.type == cudaMemoryTypeDevice && attr.device != dev)) {
+      if (pe != cudaSuccess) cudaGetLastError();
+      pbt::set_last_error("x_device and fitness_out_device must be device memory of the current device");
+      return PBT_ERR_INVALID_ARG;
+    }
   }
   double* scratch = nullptr;
   int rc = scratch_for_current_device(&scratch);

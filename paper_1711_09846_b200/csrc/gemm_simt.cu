@@ -20,6 +20,7 @@ __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloat162float(v)
 
 template <typename T, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(256) k_gemm_simt(GemmArgs g) {
+  pdl_prologue();
   // double-buffered k-slabs: the global loads of slab k+1 are in flight (in registers) while slab k is multiplied
   __shared__ float As[2][BK][BM + 4];
   __shared__ float Bs[2][BK][BN + 4];
@@ -138,6 +139,7 @@ __device__ __forceinline__ void store_one(const GemmArgs& g, int member, int m, 
 // N <= NT <= 16, A K-major: one warp per output row, lanes stride over K, shuffle reduction.
 template <typename T, bool B_MN, int NT>
 __global__ void __launch_bounds__(256) k_gemm_rowdot(GemmArgs g) {
+  pdl_prologue();
   const int member = blockIdx.y, lane = threadIdx.x & 31;
   const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
   if (m >= g.M) return;
@@ -173,6 +175,7 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& w, float* f) {
 // arithmetic, conversion and one multiply-add per 2-byte load); this one issues about a third as many.
 template <int NT>
 __global__ void __launch_bounds__(256) k_gemm_rowdot_bf16x8(GemmArgs g) {
+  pdl_prologue();
   const int member = blockIdx.y, lane = threadIdx.x & 31;
   const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
   if (m >= g.M) return;
@@ -211,7 +214,7 @@ static bool rowdot_vec_ok(const GemmArgs& g) {
 // one instantiation per width: no predicated-off columns in the inner loop
 template <int NT>
 static void launch_rowdot_vec_n(const GemmArgs& g, cudaStream_t s) {
-  k_gemm_rowdot_bf16x8<NT><<<dim3((g.M + 7) / 8, g.batch), 256, 0, s>>>(g);
+  launch_with(dim3((g.M + 7) / 8, g.batch), 256, 0, s)(k_gemm_rowdot_bf16x8<NT>, g);
 }
 static void launch_rowdot_vec(const GemmArgs& g, cudaStream_t s) {
   switch (g.N) {
@@ -230,6 +233,7 @@ static void launch_rowdot_vec(const GemmArgs& g, cudaStream_t s) {
 // long dimension, 16 slices of K per block combined in a fixed order.  LONG_A: M is the long dimension, else N.
 template <typename T, bool LONG_A, int ST>
 __global__ void __launch_bounds__(512) k_gemm_colacc(GemmArgs g) {
+  pdl_prologue();
   __shared__ float red[16][32][ST + 1];
   const int member = blockIdx.y, tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int L = LONG_A ? g.M : g.N, S = LONG_A ? g.N : g.M;
@@ -271,6 +275,7 @@ __global__ void __launch_bounds__(512) k_gemm_colacc(GemmArgs g) {
 // block's 16 slices of K are combined in a fixed order, one short index at a time through 8 KB of shared memory.
 template <bool LONG_A, int ST>
 __global__ void __launch_bounds__(256) k_gemm_colacc_bf16x8(GemmArgs g) {
+  pdl_prologue();
   __shared__ float red[16][128 + 4];
   const int member = blockIdx.y, lg = threadIdx.x & 15, ks = threadIdx.x >> 4;
   const int L = LONG_A ? g.M : g.N;
@@ -316,7 +321,7 @@ __global__ void __launch_bounds__(256) k_gemm_colacc_bf16x8(GemmArgs g) {
 
 template <bool LONG_A, int ST>
 static void launch_colacc_vec_n(const GemmArgs& g, int L, cudaStream_t s) {
-  k_gemm_colacc_bf16x8<LONG_A, ST><<<dim3((L + 127) / 128, g.batch), 256, 0, s>>>(g);
+  launch_with(dim3((L + 127) / 128, g.batch), 256, 0, s)(k_gemm_colacc_bf16x8<LONG_A, ST>, g);
 }
 template <bool LONG_A>
 static bool launch_colacc_vec(const GemmArgs& g, cudaStream_t s) {
@@ -346,6 +351,7 @@ static bool launch_colacc_vec(const GemmArgs& g, cudaStream_t s) {
 constexpr int kSmallKRows = 32;
 template <typename T>
 __global__ void __launch_bounds__(256) k_gemm_smallk(GemmArgs g) {
+  pdl_prologue();
   const int member = blockIdx.z, m0 = blockIdx.y * kSmallKRows;
   const int n = blockIdx.x * 256 + threadIdx.x;
   __shared__ float As[kSmallKRows][kSkinny];
@@ -376,6 +382,7 @@ __global__ void __launch_bounds__(256) k_gemm_smallk(GemmArgs g) {
 // over the 32 rows x N / 8 column groups of its slab.  Same multiply-add order per element as the kernel above.
 template <bool B_MN>
 __global__ void __launch_bounds__(256) k_gemm_smallk_bf16x8(GemmArgs g) {
+  pdl_prologue();
   constexpr int KV = kSkinny;
   const int member = blockIdx.z, m0 = blockIdx.y * kSmallKRows;
   __shared__ float As[kSmallKRows][KV];
@@ -451,21 +458,21 @@ static bool smallk_vec_ok(const GemmArgs& g) {
 template <typename T, bool B_MN>
 static void launch_rowdot(const GemmArgs& g, cudaStream_t s) {
   dim3 grid((g.M + 7) / 8, g.batch);
-  if (g.N == 1) k_gemm_rowdot<T, B_MN, 1><<<grid, 256, 0, s>>>(g);
-  else if (g.N == 2) k_gemm_rowdot<T, B_MN, 2><<<grid, 256, 0, s>>>(g);
-  else if (g.N <= 4) k_gemm_rowdot<T, B_MN, 4><<<grid, 256, 0, s>>>(g);
-  else if (g.N <= 8) k_gemm_rowdot<T, B_MN, 8><<<grid, 256, 0, s>>>(g);
-  else k_gemm_rowdot<T, B_MN, 16><<<grid, 256, 0, s>>>(g);
+  if (g.N == 1) launch_with(grid, 256, 0, s)(k_gemm_rowdot<T, B_MN, 1>, g);
+  else if (g.N == 2) launch_with(grid, 256, 0, s)(k_gemm_rowdot<T, B_MN, 2>, g);
+  else if (g.N <= 4) launch_with(grid, 256, 0, s)(k_gemm_rowdot<T, B_MN, 4>, g);
+  else if (g.N <= 8) launch_with(grid, 256, 0, s)(k_gemm_rowdot<T, B_MN, 8>, g);
+  else launch_with(grid, 256, 0, s)(k_gemm_rowdot<T, B_MN, 16>, g);
 }
 template <typename T, bool LONG_A>
 static void launch_colacc(const GemmArgs& g, cudaStream_t s) {
   const int L = LONG_A ? g.M : g.N, S = LONG_A ? g.N : g.M;
   dim3 grid((L + 31) / 32, g.batch);
-  if (S == 1) k_gemm_colacc<T, LONG_A, 1><<<grid, 512, 0, s>>>(g);
-  else if (S == 2) k_gemm_colacc<T, LONG_A, 2><<<grid, 512, 0, s>>>(g);
-  else if (S <= 4) k_gemm_colacc<T, LONG_A, 4><<<grid, 512, 0, s>>>(g);
-  else if (S <= 8) k_gemm_colacc<T, LONG_A, 8><<<grid, 512, 0, s>>>(g);
-  else k_gemm_colacc<T, LONG_A, 16><<<grid, 512, 0, s>>>(g);
+  if (S == 1) launch_with(grid, 512, 0, s)(k_gemm_colacc<T, LONG_A, 1>, g);
+  else if (S == 2) launch_with(grid, 512, 0, s)(k_gemm_colacc<T, LONG_A, 2>, g);
+  else if (S <= 4) launch_with(grid, 512, 0, s)(k_gemm_colacc<T, LONG_A, 4>, g);
+  else if (S <= 8) launch_with(grid, 512, 0, s)(k_gemm_colacc<T, LONG_A, 8>, g);
+  else launch_with(grid, 512, 0, s)(k_gemm_colacc<T, LONG_A, 16>, g);
 }
 
 template <typename T>
@@ -473,12 +480,12 @@ static bool launch_skinny(const GemmArgs& g, cudaStream_t s) {
   if (smallk_vec_ok(g)) {
     const int per_slab = kSmallKRows * (g.N / 8);
     const dim3 grid((per_slab + 255) / 256 > 8 ? 8 : (per_slab + 255) / 256, (g.M + kSmallKRows - 1) / kSmallKRows, g.batch);
-    if (g.b_mn) k_gemm_smallk_bf16x8<true><<<grid, 256, 0, s>>>(g);
-    else k_gemm_smallk_bf16x8<false><<<grid, 256, 0, s>>>(g);
+    if (g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_smallk_bf16x8<true>, g);
+    else launch_with(grid, 256, 0, s)(k_gemm_smallk_bf16x8<false>, g);
     return true;
   }
   if (g.K <= kSkinny && g.K > 0 && (g.M + kSmallKRows - 1) / kSmallKRows <= 65535 && g.batch <= 65535) {
-    k_gemm_smallk<T><<<dim3((g.N + 255) / 256, (g.M + kSmallKRows - 1) / kSmallKRows, g.batch), 256, 0, s>>>(g);
+    launch_with(dim3((g.N + 255) / 256, (g.M + kSmallKRows - 1) / kSmallKRows, g.batch), 256, 0, s)(k_gemm_smallk<T>, g);
     return true;
   }
   if (rowdot_vec_ok(g)) {
@@ -504,10 +511,10 @@ static bool launch_skinny(const GemmArgs& g, cudaStream_t s) {
 template <typename T>
 static cudaError_t launch_t(const GemmArgs& g, cudaStream_t s) {
   dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.batch);
-  if (!g.a_mn && !g.b_mn) k_gemm_simt<T, false, false><<<grid, 256, 0, s>>>(g);
-  else if (!g.a_mn && g.b_mn) k_gemm_simt<T, false, true><<<grid, 256, 0, s>>>(g);
-  else if (g.a_mn && g.b_mn) k_gemm_simt<T, true, true><<<grid, 256, 0, s>>>(g);
-  else k_gemm_simt<T, true, false><<<grid, 256, 0, s>>>(g);
+  if (!g.a_mn && !g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt<T, false, false>, g);
+  else if (!g.a_mn && g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt<T, false, true>, g);
+  else if (g.a_mn && g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt<T, true, true>, g);
+  else launch_with(grid, 256, 0, s)(k_gemm_simt<T, true, false>, g);
   return cudaGetLastError();
 }
 

@@ -38,6 +38,7 @@ struct Smem {
 template <int BN, int STAGES, int EPI, int NEPIW>
 __global__ void __launch_bounds__(64 + 32 * NEPIW, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+  pdl_prologue();
   using L = Smem<BN, STAGES, NEPIW>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -186,23 +187,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 template <int BN, int STAGES, int EPI, int NEPIW>
 cudaError_t launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, TcParams& p, cudaStream_t s) {
   using L = Smem<BN, STAGES, NEPIW>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_gemm_tc<BN, STAGES, EPI, NEPIW>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static DeviceSetup setup;   // one per kernel instantiation
+  int sms = 0;
+  cudaError_t e = device_setup(&setup, k_gemm_tc<BN, STAGES, EPI, NEPIW>, L::kTotal, &sms);
+  if (e != cudaSuccess) return e;
   p.tiles_n = (p.N + BN - 1) / BN;
   p.num_tiles = p.tiles_m * p.tiles_n * p.batch;
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (sms <= 0) sms = 148;
-  }
   const int grid = p.num_tiles < sms ? p.num_tiles : sms;
-  k_gemm_tc<BN, STAGES, EPI, NEPIW><<<grid, 64 + 32 * NEPIW, L::kTotal, s>>>(tmA, tmB, p);
+  launch_with(grid, 64 + 32 * NEPIW, L::kTotal, s)(k_gemm_tc<BN, STAGES, EPI, NEPIW>, tmA, tmB, p);
   return cudaGetLastError();
 }
 
@@ -211,6 +203,7 @@ cudaError_t launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, TcParams&
 // Self-test of the bounded wait every tensor-core kernel relies on: one CTA waits on a barrier that nothing ever
 // signals; when the limit runs out it records PBT_ERR_TIMEOUT like the real kernels do and returns normally.
 __global__ void k_selftest_bounded_wait(Counters* counters, uint32_t limit) {
+  pdl_prologue();
   __shared__ uint64_t bar;
   __shared__ int abort_flag;
   if (threadIdx.x == 0) {
@@ -228,7 +221,7 @@ __global__ void k_selftest_bounded_wait(Counters* counters, uint32_t limit) {
 }
 
 cudaError_t launch_selftest_bounded_wait(Counters* counters, uint32_t limit, cudaStream_t s) {
-  k_selftest_bounded_wait<<<1, 32, 0, s>>>(counters, limit);
+  launch_with(1, 32, 0, s)(k_selftest_bounded_wait, counters, limit);
   return cudaGetLastError();
 }
 

@@ -85,6 +85,7 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t cluster_addr) {
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
 k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+  pdl_prologue();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kPBarOffset);   // used in the leader only
@@ -267,22 +268,13 @@ cudaError_t launch_gemm_tc_pair(const GemmArgs& g, Counters* counters, cudaStrea
   if (!g.b_mn) ok = make_map(&tmB, g.B, g.K, b_rows, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kPN / 2);
   else ok = make_map(&tmB, g.B, g.N, b_rows, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kBK);
   if (!ok) return cudaErrorInvalidValue;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_gemm_tc_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmemTotal);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (sms <= 0) sms = 148;
-  }
+  static DeviceSetup setup;
+  int sms = 0;
+  cudaError_t e = device_setup(&setup, k_gemm_tc_pair, kPSmemTotal, &sms);
+  if (e != cudaSuccess) return e;
   int pairs = sms / 2;
   if (pairs > p.num_tiles) pairs = p.num_tiles;
-  k_gemm_tc_pair<<<2 * pairs, kPThreads, kPSmemTotal, s>>>(tmA, tmB, p);
+  launch_with(2 * pairs, kPThreads, kPSmemTotal, s)(k_gemm_tc_pair, tmA, tmB, p);
   return cudaGetLastError();
 }
 

@@ -13,6 +13,7 @@ namespace pbt {
 // ---------------------------------------------------------------------------
 __global__ void k_init_weights(float* __restrict__ w32, long long p_pad, long long w_off, long long count,
                                int tensor_id, float bound, uint64_t seed) {
+  pdl_prologue();
   const int m = blockIdx.y;
   const long long blk = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (blk * 4 >= count) return;
@@ -33,11 +34,12 @@ cudaError_t launch_init_weights(float* w32, long long p_pad, int n_members, long
   const long long count = (long long)fan_out * fan_in;
   const long long blocks4 = (count + 3) / 4;
   dim3 grid((unsigned)((blocks4 + 255) / 256), n_members);
-  k_init_weights<<<grid, 256, 0, s>>>(w32, p_pad, w_off, count, tensor_id, bound, seed);
+  launch_with(grid, 256, 0, s)(k_init_weights, w32, p_pad, w_off, count, tensor_id, bound, seed);
   return cudaGetLastError();
 }
 
 __global__ void k_f32_to_bf16(const float* __restrict__ in, bf16* __restrict__ out, long long n) {
+  pdl_prologue();
   long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (; i < n; i += stride) out[i] = __float2bfloat16_rn(in[i]);
@@ -47,7 +49,7 @@ cudaError_t launch_f32_to_bf16(const float* in, bf16* out, long long n, cudaStre
   if (n <= 0) return cudaSuccess;
   long long blocks = (n + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
-  k_f32_to_bf16<<<(unsigned)blocks, 256, 0, s>>>(in, out, n);
+  launch_with((unsigned)blocks, 256, 0, s)(k_f32_to_bf16, in, out, n);
   return cudaGetLastError();
 }
 
@@ -57,10 +59,11 @@ cudaError_t launch_f32_to_bf16(const float* in, bf16* out, long long n, cudaStre
 // ---------------------------------------------------------------------------
 __global__ void k_gather_window(char* __restrict__ dst, long long dst_stride_bytes, long long dst_offset_bytes,
                                 const char* __restrict__ pool, int row_bytes, int rows, int pool_rows, int block,
-                                int word_index, uint64_t seed, const Counters* __restrict__ counters) {
+                                int word_index, uint64_t seed, const Counters* __restrict__ counters, StepClock clk) {
+  pdl_prologue();
   if (counters->use_supplied_batch) return;
   const int m = blockIdx.y;
-  const U4 r = philox4x32_10((uint32_t)m, (uint32_t)counters->step, kStreamBatch, (uint32_t)block, seed);
+  const U4 r = philox4x32_10((uint32_t)(clk.member_base + m), (uint32_t)clk.t[m], kStreamBatch, (uint32_t)block, seed);
   const uint32_t n_win = (uint32_t)((pool_rows - rows) / 128 + 1);
   const long long off = 128ll * (long long)(((uint64_t)r.x[word_index] * n_win) >> 32);
   const long long bytes = (long long)rows * row_bytes;
@@ -80,31 +83,32 @@ __global__ void k_gather_window(char* __restrict__ dst, long long dst_stride_byt
 }
 
 __global__ void k_window_offsets(int* __restrict__ off, int rows, int pool_rows, int n_members, int block, int word_index,
-                                 uint64_t seed, const Counters* __restrict__ counters) {
+                                 uint64_t seed, StepClock clk) {
+  pdl_prologue();
   const int m = blockIdx.x * blockDim.x + threadIdx.x;
   if (m >= n_members) return;
-  const U4 r = philox4x32_10((uint32_t)m, (uint32_t)counters->step, kStreamBatch, (uint32_t)block, seed);
+  const U4 r = philox4x32_10((uint32_t)(clk.member_base + m), (uint32_t)clk.t[m], kStreamBatch, (uint32_t)block, seed);
   const uint32_t n_win = (uint32_t)((pool_rows - rows) / 128 + 1);
   off[m] = (int)(128ll * (long long)(((uint64_t)r.x[word_index] * n_win) >> 32));
 }
 
 cudaError_t launch_window_offsets(int* off, int rows, int pool_rows, int n_members, int block, int word_index,
-                                  uint64_t seed, const Counters* counters, cudaStream_t s) {
-  k_window_offsets<<<(n_members + 127) / 128, 128, 0, s>>>(off, rows, pool_rows, n_members, block, word_index, seed, counters);
+                                  uint64_t seed, StepClock clk, cudaStream_t s) {
+  launch_with((n_members + 127) / 128, 128, 0, s)(k_window_offsets, off, rows, pool_rows, n_members, block, word_index, seed, clk);
   return cudaGetLastError();
 }
 
 cudaError_t launch_gather_window(char* dst, long long dst_stride_bytes, long long dst_offset_bytes,
                                  const char* pool, int row_bytes, int rows, int pool_rows, int n_members,
                                  int block, int word_index, uint64_t seed, const Counters* counters,
-                                 cudaStream_t s) {
+                                 StepClock clk, cudaStream_t s) {
   const long long bytes = (long long)rows * row_bytes;
   long long blocks = (bytes / 16 + 255) / 256;
   if (blocks < 1) blocks = 1;
   if (blocks > 64) blocks = 64;
   dim3 grid((unsigned)blocks, n_members);
-  k_gather_window<<<grid, 256, 0, s>>>(dst, dst_stride_bytes, dst_offset_bytes, pool, row_bytes, rows, pool_rows,
-                                       block, word_index, seed, counters);
+  launch_with(grid, 256, 0, s)(k_gather_window, dst, dst_stride_bytes, dst_offset_bytes, pool, row_bytes, rows, pool_rows,
+                                       block, word_index, seed, counters, clk);
   return cudaGetLastError();
 }
 
@@ -112,6 +116,7 @@ template <typename TD>
 __global__ void k_copy_rows(TD* __restrict__ dst, long long dst_ld, long long dst_stride,
                             const float* __restrict__ src, long long src_ld, long long src_stride, int rows,
                             int cols) {
+  pdl_prologue();
   const int m = blockIdx.y;
   const long long total = (long long)rows * cols;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
@@ -131,9 +136,9 @@ cudaError_t launch_copy_rows(void* dst, int dst_dtype, long long dst_ld, long lo
   if (blocks > 32) blocks = 32;
   dim3 grid((unsigned)blocks, n_members);
   if (dst_dtype == kBF16)
-    k_copy_rows<bf16><<<grid, 256, 0, s>>>((bf16*)dst, dst_ld, dst_stride, src, src_ld, src_stride, rows, cols);
+    launch_with(grid, 256, 0, s)(k_copy_rows<bf16>, (bf16*)dst, dst_ld, dst_stride, src, src_ld, src_stride, rows, cols);
   else
-    k_copy_rows<float><<<grid, 256, 0, s>>>((float*)dst, dst_ld, dst_stride, src, src_ld, src_stride, rows, cols);
+    launch_with(grid, 256, 0, s)(k_copy_rows<float>, (float*)dst, dst_ld, dst_stride, src, src_ld, src_stride, rows, cols);
   return cudaGetLastError();
 }
 
@@ -166,6 +171,7 @@ __device__ __forceinline__ float sigmoid_f(float x) {
 }
 
 __global__ void k_loss_rows(LossArgs a) {
+  pdl_prologue();
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   const int m = blockIdx.y;
@@ -241,6 +247,7 @@ __global__ void k_loss_rows(LossArgs a) {
 // 29 us per row and warp on the 1024-wide output layer).  Same formulas, different summation order.
 template <int ITERS>
 __global__ void __launch_bounds__(256) k_loss_ce_soft_vec(LossArgs a) {
+  pdl_prologue();
   const int lane = threadIdx.x & 31;
   const int m = blockIdx.y;
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -301,14 +308,14 @@ static bool launch_ce_soft_vec(const LossArgs& a, cudaStream_t s) {
   if (a.stride_target % 4 != 0 || ((uintptr_t)a.target & 7)) return false;
   dim3 grid((a.rows + 7) / 8, a.n_members);
   switch (a.cols / 128) {
-    case 1: k_loss_ce_soft_vec<1><<<grid, 256, 0, s>>>(a); break;
-    case 2: k_loss_ce_soft_vec<2><<<grid, 256, 0, s>>>(a); break;
-    case 3: k_loss_ce_soft_vec<3><<<grid, 256, 0, s>>>(a); break;
-    case 4: k_loss_ce_soft_vec<4><<<grid, 256, 0, s>>>(a); break;
-    case 5: k_loss_ce_soft_vec<5><<<grid, 256, 0, s>>>(a); break;
-    case 6: k_loss_ce_soft_vec<6><<<grid, 256, 0, s>>>(a); break;
-    case 7: k_loss_ce_soft_vec<7><<<grid, 256, 0, s>>>(a); break;
-    default: k_loss_ce_soft_vec<8><<<grid, 256, 0, s>>>(a); break;
+    case 1: launch_with(grid, 256, 0, s)(k_loss_ce_soft_vec<1>, a); break;
+    case 2: launch_with(grid, 256, 0, s)(k_loss_ce_soft_vec<2>, a); break;
+    case 3: launch_with(grid, 256, 0, s)(k_loss_ce_soft_vec<3>, a); break;
+    case 4: launch_with(grid, 256, 0, s)(k_loss_ce_soft_vec<4>, a); break;
+    case 5: launch_with(grid, 256, 0, s)(k_loss_ce_soft_vec<5>, a); break;
+    case 6: launch_with(grid, 256, 0, s)(k_loss_ce_soft_vec<6>, a); break;
+    case 7: launch_with(grid, 256, 0, s)(k_loss_ce_soft_vec<7>, a); break;
+    default: launch_with(grid, 256, 0, s)(k_loss_ce_soft_vec<8>, a); break;
   }
   return true;
 }
@@ -317,7 +324,7 @@ cudaError_t launch_loss_rows(const LossArgs& a, cudaStream_t s) {
   if (launch_ce_soft_vec(a, s)) return cudaGetLastError();
   const int warps = 8;
   dim3 grid((a.rows + warps - 1) / warps, a.n_members);
-  k_loss_rows<<<grid, warps * 32, 0, s>>>(a);
+  launch_with(grid, warps * 32, 0, s)(k_loss_rows, a);
   return cudaGetLastError();
 }
 
@@ -338,6 +345,7 @@ __device__ __forceinline__ T block_sum_256(T v, T* sh) {
 
 __global__ void k_reduce_rows(const float* __restrict__ row_loss, int rows, float scale, void* out,
                               int out_is_double, int out_stride) {
+  pdl_prologue();
   __shared__ double sh[256];
   const int m = blockIdx.x;
   double acc = 0.0;
@@ -352,7 +360,7 @@ __global__ void k_reduce_rows(const float* __restrict__ row_loss, int rows, floa
 
 cudaError_t launch_reduce_rows(const float* row_loss, int rows, int n_members, float scale, void* out,
                                int out_is_double, int out_stride, cudaStream_t s) {
-  k_reduce_rows<<<n_members, 256, 0, s>>>(row_loss, rows, scale, out, out_is_double, out_stride);
+  launch_with(n_members, 256, 0, s)(k_reduce_rows, row_loss, rows, scale, out, out_is_double, out_stride);
   return cudaGetLastError();
 }
 
@@ -362,6 +370,7 @@ cudaError_t launch_reduce_rows(const float* row_loss, int rows, int n_members, f
 template <typename T>
 __global__ void k_bias_grad(const T* __restrict__ dz, long long ld, long long stride, int rows, int cols,
                             float* __restrict__ out, long long out_stride) {
+  pdl_prologue();
   __shared__ float sh[8][33];
   const int m = blockIdx.y;
   const int c = blockIdx.x * 32 + threadIdx.x;
@@ -387,6 +396,7 @@ __global__ void k_bias_grad(const T* __restrict__ dz, long long ld, long long st
 // w, w + 8, ... and the eight partial sums are combined in order, exactly like the scalar kernel above (same bits).
 __global__ void __launch_bounds__(256) k_bias_grad_bf16x8(const bf16* __restrict__ dz, long long ld, long long stride, int rows,
                                                           int cols, float* __restrict__ out, long long out_stride) {
+  pdl_prologue();
   __shared__ float sh[8][256 + 8];
   const int m = blockIdx.y, lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int c0 = blockIdx.x * 256 + lane * 8;
@@ -422,14 +432,14 @@ cudaError_t launch_bias_grad(const void* dz, int dz_dtype, long long ld, long lo
   if (dz_dtype == kBF16 && cols % 8 == 0 && (long long)((cols + 255) / 256) * n_members >= 296 && ld % 8 == 0 &&
       stride % 8 == 0 && ((uintptr_t)dz & 15) == 0) {
     dim3 grid((cols + 255) / 256, n_members);
-    k_bias_grad_bf16x8<<<grid, 256, 0, s>>>((const bf16*)dz, ld, stride, rows, cols, out, out_stride);
+    launch_with(grid, 256, 0, s)(k_bias_grad_bf16x8, (const bf16*)dz, ld, stride, rows, cols, out, out_stride);
     return cudaGetLastError();
   }
   dim3 grid((cols + 31) / 32, n_members), block(32, 8);
   if (dz_dtype == kBF16)
-    k_bias_grad<bf16><<<grid, block, 0, s>>>((const bf16*)dz, ld, stride, rows, cols, out, out_stride);
+    launch_with(grid, block, 0, s)(k_bias_grad<bf16>, (const bf16*)dz, ld, stride, rows, cols, out, out_stride);
   else
-    k_bias_grad<float><<<grid, block, 0, s>>>((const float*)dz, ld, stride, rows, cols, out, out_stride);
+    launch_with(grid, block, 0, s)(k_bias_grad<float>, (const float*)dz, ld, stride, rows, cols, out, out_stride);
   return cudaGetLastError();
 }
 
@@ -438,6 +448,7 @@ cudaError_t launch_bias_grad(const void* dz, int dz_dtype, long long ld, long lo
 // Explicitly rounded operations (no fused multiply-add) so the CPU reproduces every bit.
 // ---------------------------------------------------------------------------
 __global__ void k_toy_step(double* theta, const double* __restrict__ H, int n_members, int dim, double eta) {
+  pdl_prologue();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_members * dim) return;
   const int m = i / dim, k = i % dim;
@@ -447,6 +458,7 @@ __global__ void k_toy_step(double* theta, const double* __restrict__ H, int n_me
 }
 
 __global__ void k_toy_eval(const double* __restrict__ theta, double* fitness, int n_members, int dim) {
+  pdl_prologue();
   const int m = blockIdx.x * blockDim.x + threadIdx.x;
   if (m >= n_members) return;
   double s = 0.0;
@@ -456,11 +468,11 @@ __global__ void k_toy_eval(const double* __restrict__ theta, double* fitness, in
 
 cudaError_t launch_toy_step(double* theta, const double* H, int n_members, int dim, double eta, cudaStream_t s) {
   const int n = n_members * dim;
-  k_toy_step<<<(n + 127) / 128, 128, 0, s>>>(theta, H, n_members, dim, eta);
+  launch_with((n + 127) / 128, 128, 0, s)(k_toy_step, theta, H, n_members, dim, eta);
   return cudaGetLastError();
 }
 cudaError_t launch_toy_eval(const double* theta, double* fitness, int n_members, int dim, cudaStream_t s) {
-  k_toy_eval<<<(n_members + 127) / 128, 128, 0, s>>>(theta, fitness, n_members, dim);
+  launch_with((n_members + 127) / 128, 128, 0, s)(k_toy_eval, theta, fitness, n_members, dim);
   return cudaGetLastError();
 }
 
@@ -472,6 +484,7 @@ constexpr int kEdBlock = 256;
 int energy_partial_count(int n) { return 2 * ((n + kEdBlock - 1) / kEdBlock); }
 
 __global__ void k_energy_partial(const float* __restrict__ x, long long stride, int n, double* __restrict__ partial) {
+  pdl_prologue();
   __shared__ float2 tile[kEdBlock];
   __shared__ double sh[256];
   const int m = blockIdx.y;
@@ -511,6 +524,7 @@ __global__ void k_energy_partial(const float* __restrict__ x, long long stride, 
 }
 
 __global__ void k_energy_final(const double* __restrict__ partial, int nblocks, int n, float* fitness) {
+  pdl_prologue();
   const int m = blockIdx.x * blockDim.x + threadIdx.x;
   if (m >= (int)gridDim.x * (int)blockDim.x) return;
   double within = 0.0, cross = 0.0;
@@ -534,10 +548,10 @@ cudaError_t launch_energy_distance(const float* x, long long stride, int n, int 
                                    float* fitness, cudaStream_t s) {
   const int nblocks = (n + kEdBlock - 1) / kEdBlock;
   dim3 grid(nblocks, n_members);
-  k_energy_partial<<<grid, kEdBlock, 0, s>>>(x, stride, n, partial);
+  launch_with(grid, kEdBlock, 0, s)(k_energy_partial, x, stride, n, partial);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  k_energy_final<<<n_members, 1, 0, s>>>(partial, nblocks, n, fitness);
+  launch_with(n_members, 1, 0, s)(k_energy_final, partial, nblocks, n, fitness);
   return cudaGetLastError();
 }
 
@@ -546,12 +560,13 @@ cudaError_t launch_energy_distance(const float* x, long long stride, int n, int 
 // penalty on the norm of the critic's input gradient with its derivative.
 // ---------------------------------------------------------------------------
 template <typename T>
-__global__ void k_gp_interp(T* __restrict__ x, long long stride, int B, int dim, int j, uint64_t seed,
-                            const Counters* __restrict__ counters) {
+__global__ void k_gp_interp(T* __restrict__ x, long long stride, int B, int dim, int j, uint64_t seed, StepClock clk) {
+  pdl_prologue();
   const int m = blockIdx.y;
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
-  const U4 r = philox4x32_10((uint32_t)m, (uint32_t)counters->step, kStreamInterp, (uint32_t)(j * 65536 + (b >> 2)), seed);
+  const U4 r = philox4x32_10((uint32_t)(clk.member_base + m), (uint32_t)clk.t[m], kStreamInterp,
+                             (uint32_t)(j * 65536 + (b >> 2)), seed);
   // (w >> 9) + 1/2 has 24 significant bits, and so has its complement: both are exact in float
   const float e = ((float)(r.x[b & 3] >> 9) + 0.5f) * 1.1920928955078125e-07f;
   const float ome = 1.0f - e;
@@ -571,10 +586,10 @@ __global__ void k_gp_interp(T* __restrict__ x, long long stride, int B, int dim,
 }
 
 cudaError_t launch_gp_interp(void* x, int dtype, long long stride, int B, int dim, int j, int n_members, uint64_t seed,
-                             const Counters* counters, cudaStream_t s) {
+                             StepClock clk, cudaStream_t s) {
   dim3 grid((B + 127) / 128, n_members);
-  if (dtype == kBF16) k_gp_interp<bf16><<<grid, 128, 0, s>>>((bf16*)x, stride, B, dim, j, seed, counters);
-  else k_gp_interp<float><<<grid, 128, 0, s>>>((float*)x, stride, B, dim, j, seed, counters);
+  if (dtype == kBF16) launch_with(grid, 128, 0, s)(k_gp_interp<bf16>, (bf16*)x, stride, B, dim, j, seed, clk);
+  else launch_with(grid, 128, 0, s)(k_gp_interp<float>, (float*)x, stride, B, dim, j, seed, clk);
   return cudaGetLastError();
 }
 
@@ -582,6 +597,7 @@ cudaError_t launch_gp_interp(void* x, int dtype, long long stride, int B, int di
 __global__ void k_gp_penalty(const float* __restrict__ gx, long long gx_stride, int B, int dim, float lam,
                              float inv_batch, float* __restrict__ row_loss, int rows_total, int row_off, void* dv,
                              int dv_dtype, long long dv_stride) {
+  pdl_prologue();
   const int lane = threadIdx.x & 31;
   const int m = blockIdx.y;
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -602,17 +618,20 @@ cudaError_t launch_gp_penalty(const float* gx, long long gx_stride, int B, int d
                               long long dv_stride, int n_members, cudaStream_t s) {
   const int warps = 8;
   dim3 grid((B + warps - 1) / warps, n_members);
-  k_gp_penalty<<<grid, warps * 32, 0, s>>>(gx, gx_stride, B, dim, lam, inv_batch, row_loss, rows_total, row_off, dv,
+  launch_with(grid, warps * 32, 0, s)(k_gp_penalty, gx, gx_stride, B, dim, lam, inv_batch, row_loss, rows_total, row_off, dv,
                                            dv_dtype, dv_stride);
   return cudaGetLastError();
 }
 
-__global__ void k_advance_step(Counters* c) {
-  c->step += 1;
-  c->use_supplied_batch = 0;
+// every member of the window has taken one more step (Algorithm 1's t, counted per member)
+__global__ void k_advance_step(Counters* c, long long* __restrict__ t, int n_members) {
+  pdl_prologue();
+  const int m = blockIdx.x * blockDim.x + threadIdx.x;
+  if (m < n_members) t[m] += 1;
+  if (m == 0) c->use_supplied_batch = 0;
 }
-cudaError_t launch_advance_step(Counters* c, cudaStream_t s) {
-  k_advance_step<<<1, 1, 0, s>>>(c);
+cudaError_t launch_advance_step(Counters* c, long long* t, int n_members, cudaStream_t s) {
+  launch_with((n_members + 127) / 128, 128, 0, s)(k_advance_step, c, t, n_members);
   return cudaGetLastError();
 }
 

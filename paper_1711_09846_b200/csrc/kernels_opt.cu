@@ -16,6 +16,7 @@ constexpr int kOptTile = kOptThreads * kOptVecPerThread * 4;     // elements per
 
 // v <- mu v + g ; theta <- theta - lr v
 __global__ void __launch_bounds__(kOptThreads) k_sgdm(OptArgs a) {
+  pdl_prologue();
   const int m = blockIdx.y;
   const float* Hrow = a.H + (long long)m * a.nh_stride;
   const float lr = hp(Hrow, a.slot_lr, a.const_lr);
@@ -48,6 +49,7 @@ __global__ void __launch_bounds__(kOptThreads) k_sgdm(OptArgs a) {
 // theta <- theta - lr (m / (1-c1)) / (sqrt(v / (1-c2)) + eps) - lr wd theta,
 // c1, c2 = running products of the betas including this step.
 __global__ void __launch_bounds__(kOptThreads) k_adam(OptArgs a) {
+  pdl_prologue();
   const int m = blockIdx.y;
   const float* Hrow = a.H + (long long)m * a.nh_stride;
   const float lr = hp(Hrow, a.slot_lr, a.const_lr);
@@ -94,6 +96,7 @@ __global__ void __launch_bounds__(kOptThreads) k_adam(OptArgs a) {
 
 // ms <- rho ms + (1-rho) g^2 ; theta <- theta - lr g / (sqrt(ms) + eps)
 __global__ void __launch_bounds__(kOptThreads) k_rmsprop(OptArgs a) {
+  pdl_prologue();
   const int m = blockIdx.y;
   const float* Hrow = a.H + (long long)m * a.nh_stride;
   const float lr = hp(Hrow, a.slot_lr, a.const_lr);
@@ -124,6 +127,7 @@ __global__ void __launch_bounds__(kOptThreads) k_rmsprop(OptArgs a) {
 
 // after the Adam pass of a stack: store the advanced beta products
 __global__ void k_adam_advance(OptArgs a) {
+  pdl_prologue();
   const int m = blockIdx.x * blockDim.x + threadIdx.x;
   if (m >= a.n_members) return;
   const float* Hrow = a.H + (long long)m * a.nh_stride;
@@ -145,21 +149,21 @@ static unsigned opt_grid_x(const OptArgs& a) {
 
 cudaError_t launch_sgdm(const OptArgs& a, cudaStream_t s) {
   dim3 grid(opt_grid_x(a), a.n_members);
-  k_sgdm<<<grid, kOptThreads, 0, s>>>(a);
+  launch_with(grid, kOptThreads, 0, s)(k_sgdm, a);
   return cudaGetLastError();
 }
 cudaError_t launch_rmsprop(const OptArgs& a, cudaStream_t s) {
   dim3 grid(opt_grid_x(a), a.n_members);
-  k_rmsprop<<<grid, kOptThreads, 0, s>>>(a);
+  launch_with(grid, kOptThreads, 0, s)(k_rmsprop, a);
   return cudaGetLastError();
 }
 cudaError_t launch_adam(const OptArgs& a, cudaStream_t s) {
   dim3 grid(opt_grid_x(a), a.n_members);
-  k_adam<<<grid, kOptThreads, 0, s>>>(a);
+  launch_with(grid, kOptThreads, 0, s)(k_adam, a);
   return cudaGetLastError();
 }
 cudaError_t launch_adam_advance(const OptArgs& a, cudaStream_t s) {
-  k_adam_advance<<<(a.n_members + 127) / 128, 128, 0, s>>>(a);
+  launch_with((a.n_members + 127) / 128, 128, 0, s)(k_adam_advance, a);
   return cudaGetLastError();
 }
 

@@ -62,6 +62,8 @@ struct pbt_handle {
   void* hist;        // [N][PBT_HISTORY] scores for t-test selection, same type as fitness
   int* hist_n;       // [N]
   Counters* counters;
+  long long* tm;     // [N] every member's own step count (Algorithm 1's t)
+  int member_base;   // population index of the first member the pointers below refer to (0 unless a window is open)
   float* last_loss;  // [N][2]
   double* theta;     // toy: [N][nh]
   void* act[2][PBT_MAX_LAYERS];  // input of layer l of stack s: [N][rows_cap][in_l]
@@ -84,7 +86,7 @@ struct pbt_handle {
   void* act0_alt;
   void* ybatch_alt;
   cudaStream_t copy_stream;
-  cudaEvent_t ev_copied, ev_stepdone[2];
+  cudaEvent_t ev_copied, ev_release;   // ev_release: see pbt_step_prefetched
   bool prefetched;
   long long pf_steps;  // prefetched steps taken so far
   float* row_loss;
@@ -120,6 +122,11 @@ int fail(pbt_t* p, int code, const char* fmt, ...) {
 }  // namespace
 namespace pbt {
 void set_last_error(const char* msg) { snprintf(g_err, sizeof(g_err), "%s", msg); }
+namespace {
+bool g_serial_launches = false;
+}
+void set_serial_launches(bool serial) { g_serial_launches = serial; }
+bool serial_launches() { return g_serial_launches; }
 }  // namespace pbt
 namespace {
 
@@ -128,6 +135,8 @@ namespace {
     cudaError_t e_ = (expr);                                                                          \
     if (e_ != cudaSuccess) return fail(p, PBT_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_));     \
   } while (0)
+
+const int kOne = 1;   // source of small asynchronous host-to-device copies: must outlive the call
 
 long long pad32(long long n) { return (n + 31) / 32 * 32; }
 size_t align256(size_t n) { return (n + 255) / 256 * 256; }
@@ -208,6 +217,8 @@ size_t plan(pbt_handle* h, char* base) {
   };
   const size_t N = h->N;
   h->counters = (Counters*)take(sizeof(Counters));
+  h->tm = (long long*)take(N * sizeof(long long));
+  h->member_base = 0;
   h->src = (int*)take(N * sizeof(int));
   h->level = (int*)take(N * sizeof(int));
   h->H = take(N * PBT_MAX_NH * sizeof(double));
@@ -316,6 +327,45 @@ long long logits_stride(const pbt_handle* h, int k) {
   return (long long)st.rows_cap * st.L[st.nl - 1].out;
 }
 long long dz_stride(const pbt_handle* h) { return (long long)h->dz_rows_cap * h->max_width; }
+
+StepClock clock(const pbt_handle* h) { return StepClock{h->tm, h->member_base}; }
+
+// A member window: for the duration of a subset step the handle's per-member STATE pointers refer to members
+// [first, first + count) only, so that every launch of the step machinery covers just those members.  The scratch
+// buffers (activations, deltas, row losses, window offsets) are not shifted: the window uses their first `count`
+// member slots.  Kernels that need a member's population index (counter-based draws) add member_base.
+struct MemberWindow {
+  int N, member_base;
+  float *W32, *O1, *O2, *G, *scalars, *last_loss;
+  bf16* W16;
+  void* H;
+  double* theta;
+  long long* tm;
+};
+
+MemberWindow open_window(pbt_handle* h, int first, int count) {
+  MemberWindow w{h->N, h->member_base, h->W32, h->O1, h->O2, h->G, h->scalars, h->last_loss, h->W16, h->H, h->theta, h->tm};
+  const size_t f = (size_t)first;
+  if (h->W32) h->W32 += f * h->P_pad;
+  if (h->O1) h->O1 += f * h->P_pad;
+  if (h->O2) h->O2 += f * h->P_pad;
+  if (h->G) h->G += f * h->P_pad;
+  if (h->W16) h->W16 += f * h->P_pad;
+  h->scalars += f * PBT_N_SCALARS;
+  h->last_loss += f * 2;
+  h->H = (char*)h->H + f * PBT_MAX_NH * (h->toy ? 8 : 4);
+  if (h->theta) h->theta += f * h->nh;
+  h->tm += f;
+  h->N = count;
+  h->member_base += first;
+  return w;
+}
+
+void close_window(pbt_handle* h, const MemberWindow& w) {
+  h->N = w.N; h->member_base = w.member_base;
+  h->W32 = w.W32; h->O1 = w.O1; h->O2 = w.O2; h->G = w.G; h->scalars = w.scalars; h->last_loss = w.last_loss;
+  h->W16 = w.W16; h->H = w.H; h->theta = w.theta; h->tm = w.tm;
+}
 
 // ----- launch bookkeeping -----------------------------------------------------
 cudaEvent_t get_event(pbt_handle* h) {
@@ -563,7 +613,7 @@ int step_mlp(pbt_handle* h) {
   const int in = st.L[0].in;
   if (h->direct_pool && !h->supplied_next) {
     // the first layer's forward and weight-gradient GEMMs and the loss read the window of each member in place
-    LAUNCH(h, kCopy, launch_window_offsets(h->win_off, s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, h->stream));
+    LAUNCH(h, kCopy, launch_window_offsets(h->win_off, s.batch, s.pool_rows, h->N, 0, 0, h->seed, clock(h), h->stream));
     int rc = forward(h, 0, s.batch, h->data.x_pool, 0, h->win_off, s.pool_rows);
     if (rc) return rc;
     rc = loss_and_dz(h, 0, s.batch, s.batch, h->data.y_pool, 0, true, 0, 1.0f / s.batch, h->last_loss, 2, h->win_off);
@@ -572,11 +622,11 @@ int step_mlp(pbt_handle* h) {
     return backward(h, 0, s.batch, h->data.x_pool, 0, true, false, &cur, s.slot_lr, 0, h->win_off, s.pool_rows);
   }
   LAUNCH(h, kCopy, launch_gather_window((char*)h->act[0][0], act_stride(h, 0, 0) * h->esz, 0, (const char*)h->data.x_pool,
-                                        in * h->esz, s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, h->stream));
+                                        in * h->esz, s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, clock(h), h->stream));
   const size_t trb = target_row_bytes(h);
   const size_t tsz = s.loss == PBT_LOSS_CE_SOFT ? h->esz : 4;
   LAUNCH(h, kCopy, launch_gather_window((char*)h->ybatch, h->ybatch_stride * tsz, 0, (const char*)h->data.y_pool, (int)trb,
-                                        s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, h->stream));
+                                        s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, clock(h), h->stream));
   int rc = forward(h, 0, s.batch, h->act[0][0], act_stride(h, 0, 0));
   if (rc) return rc;
   rc = loss_and_dz(h, 0, s.batch, s.batch, h->ybatch, h->ybatch_stride, true, 0, 1.0f / s.batch, h->last_loss, 2);
@@ -596,9 +646,9 @@ int step_gan(pbt_handle* h) {
     const bool d_phase = j < s.gan_d_steps;
     if (d_phase)
       LAUNCH(h, kCopy, launch_gather_window((char*)h->act[1][0], d_in_stride * h->esz, 0, (const char*)h->data.x_pool,
-                                            xdim * h->esz, B, s.pool_rows, h->N, j, 0, h->seed, h->counters, h->stream));
+                                            xdim * h->esz, B, s.pool_rows, h->N, j, 0, h->seed, h->counters, clock(h), h->stream));
     LAUNCH(h, kCopy, launch_gather_window((char*)h->act[0][0], act_stride(h, 0, 0) * h->esz, 0, (const char*)h->data.z_pool,
-                                          zdim * h->esz, B, s.pool_rows, h->N, j, 1, h->seed, h->counters, h->stream));
+                                          zdim * h->esz, B, s.pool_rows, h->N, j, 1, h->seed, h->counters, clock(h), h->stream));
     rc = forward(h, 0, B, h->act[0][0], act_stride(h, 0, 0));
     if (rc) return rc;
     // generated samples become discriminator input rows (after the real rows in a discriminator update)
@@ -644,14 +694,14 @@ int step_wgan(pbt_handle* h) {
   int rc;
   for (int j = 0; j < s.gan_d_steps; ++j) {
     LAUNCH(h, kCopy, launch_gather_window((char*)h->act[1][0], d_in_stride * h->esz, 0, (const char*)h->data.x_pool,
-                                          xdim * h->esz, B, s.pool_rows, h->N, j, 0, h->seed, h->counters, h->stream));
+                                          xdim * h->esz, B, s.pool_rows, h->N, j, 0, h->seed, h->counters, clock(h), h->stream));
     LAUNCH(h, kCopy, launch_gather_window((char*)h->act[0][0], act_stride(h, 0, 0) * h->esz, 0, (const char*)h->data.z_pool,
-                                          zdim * h->esz, B, s.pool_rows, h->N, j, 1, h->seed, h->counters, h->stream));
+                                          zdim * h->esz, B, s.pool_rows, h->N, j, 1, h->seed, h->counters, clock(h), h->stream));
     rc = forward(h, 0, B, h->act[0][0], act_stride(h, 0, 0));
     if (rc) return rc;
     LAUNCH(h, kCopy, launch_copy_rows((char*)h->act[1][0] + (size_t)B * xdim * h->esz, h->cdt, xdim, d_in_stride, h->logits[0],
                                       xdim, logits_stride(h, 0), B, xdim, h->N, h->stream));
-    LAUNCH(h, kOther, launch_gp_interp(h->act[1][0], h->cdt, d_in_stride, B, xdim, j, h->N, h->seed, h->counters, h->stream));
+    LAUNCH(h, kOther, launch_gp_interp(h->act[1][0], h->cdt, d_in_stride, B, xdim, j, h->N, h->seed, clock(h), h->stream));
     rc = forward(h, 1, 3 * B, h->act[1][0], d_in_stride);
     if (rc) return rc;
     // deltas of the last layer for all 3B rows; losses of the real and generated rows
@@ -703,7 +753,7 @@ int step_wgan(pbt_handle* h) {
   }
   // generator update
   LAUNCH(h, kCopy, launch_gather_window((char*)h->act[0][0], act_stride(h, 0, 0) * h->esz, 0, (const char*)h->data.z_pool,
-                                        zdim * h->esz, B, s.pool_rows, h->N, s.gan_d_steps, 1, h->seed, h->counters, h->stream));
+                                        zdim * h->esz, B, s.pool_rows, h->N, s.gan_d_steps, 1, h->seed, h->counters, clock(h), h->stream));
   rc = forward(h, 0, B, h->act[0][0], act_stride(h, 0, 0));
   if (rc) return rc;
   LAUNCH(h, kCopy, launch_copy_rows(h->act[1][0], h->cdt, xdim, d_in_stride, h->logits[0], xdim, logits_stride(h, 0), B, xdim,
@@ -732,7 +782,7 @@ int one_step(pbt_handle* h) {
     rc = step_mlp(h);
     if (rc) return rc;
   }
-  LAUNCH(h, kOther, launch_advance_step(h->counters, h->stream));
+  LAUNCH(h, kOther, launch_advance_step(h->counters, h->tm, h->N, h->stream));
   h->supplied_next = false;
   return PBT_OK;
 }
@@ -873,8 +923,7 @@ int pbt_destroy(pbt_t* p) {
   if (p->copy_stream) {
     cudaStreamSynchronize(p->copy_stream);
     cudaEventDestroy(p->ev_copied);
-    cudaEventDestroy(p->ev_stepdone[0]);
-    cudaEventDestroy(p->ev_stepdone[1]);
+    cudaEventDestroy(p->ev_release);
     cudaStreamDestroy(p->copy_stream);
   }
   for (auto& r : p->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -885,6 +934,7 @@ int pbt_destroy(pbt_t* p) {
 
 int pbt_step(pbt_t* p, int k) {
   if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  set_serial_launches(p->spec.serial_launches != 0);
   if (k < 0) return fail(p, PBT_ERR_INVALID_ARG, "k must be >= 0");
   p->launches = 0;
   // Small populations are launch-bound: replay one captured step as a CUDA graph.  Capture needs a
@@ -930,6 +980,28 @@ int pbt_step(pbt_t* p, int k) {
   return PBT_OK;
 }
 
+int pbt_step_subset(pbt_t* p, const uint8_t* active_host, int k) {
+  if (!p || !active_host) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  set_serial_launches(p->spec.serial_launches != 0);
+  if (k < 0) return fail(p, PBT_ERR_INVALID_ARG, "k must be >= 0");
+  if (p->supplied_next) return fail(p, PBT_ERR_STATE, "a caller-supplied batch is pending: it belongs to a step of the whole population");
+  p->launches = 0;
+  // one pass of the step machinery per maximal run of consecutive active members
+  int m = 0;
+  while (m < p->N) {
+    if (!active_host[m]) { ++m; continue; }
+    int e = m;
+    while (e < p->N && active_host[e]) ++e;
+    const MemberWindow w = open_window(p, m, e - m);
+    int rc = PBT_OK;
+    for (int i = 0; i < k && rc == PBT_OK; ++i) rc = one_step(p);
+    close_window(p, w);
+    if (rc) return rc;
+    m = e;
+  }
+  return PBT_OK;
+}
+
 // t-test selection compares the last PBT_HISTORY scores of two members: every evaluation is appended
 static int record_scores(pbt_t* p) {
   if (p->spec.exploit_rule != 2) return PBT_OK;
@@ -939,6 +1011,7 @@ static int record_scores(pbt_t* p) {
 
 int pbt_eval(pbt_t* p) {
   if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  set_serial_launches(p->spec.serial_launches != 0);
   p->launches = 0;
   const pbt_spec& s = p->spec;
   if (p->toy) {
@@ -971,6 +1044,7 @@ int pbt_exploit_explore(pbt_t* p) { return pbt_exploit_explore_ready(p, nullptr)
 
 int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host) {
   if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  set_serial_launches(p->spec.serial_launches != 0);
   p->launches = 0;
   const pbt_spec& s = p->spec;
   SelectArgs a;
@@ -1008,14 +1082,7 @@ int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host) {
   if (!(s.flags & PBT_COPY_WEIGHTS) || p->N < 2 || (s.exploit_rule == 0 && n_cut == 0)) return PBT_OK;
   // Truncation: donors are never recipients, one parallel copy pass.  Tournament, t-test: a donor may be a recipient
   // too; recipients are copied in passes (deepest readers first) so that every copy reads the donor's record
-  // as it was before this ready point.  The number of passes is read back from the device.
-  int passes = 1;
-  if (s.exploit_rule != 0) {
-    Counters cnt;
-    CU(p, cudaMemcpyAsync(&cnt, p->counters, sizeof(cnt), cudaMemcpyDeviceToHost, p->stream));
-    CU(p, cudaStreamSynchronize(p->stream));
-    passes = cnt.max_level + 1;
-  }
+  // as it was before this ready point.  The number of passes stays on the device: one launch walks them all.
   CopyArgs c;
   memset(&c, 0, sizeof(c));
   c.n = p->N; c.src = p->src;
@@ -1033,14 +1100,16 @@ int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host) {
     add(p->W16, p->P_pad * 2, p->P_pad * 2);
     add(p->scalars, PBT_N_SCALARS * 4, PBT_N_SCALARS * 4);
   }
-  for (int pass = 0; pass < passes; ++pass) {
-    c.want_level = pass;
-    if (p->toy) {
-      // nh doubles per member: tiny, and not a multiple of 16 bytes in general
-      LAUNCH(p, kCopy, launch_copy_small((char*)p->theta, (long long)p->nh * 8, p->src, p->N, c.level, pass, p->stream));
-    } else {
-      LAUNCH(p, kCopy, launch_slab_copy(c, p->stream));
-    }
+  if (p->toy) {
+    // nh doubles per member: tiny, and not a multiple of 16 bytes in general
+    if (s.exploit_rule != 0)
+      LAUNCH(p, kCopy, launch_copy_small_levels((char*)p->theta, (long long)p->nh * 8, p->src, p->N, p->level, p->counters, p->stream));
+    else
+      LAUNCH(p, kCopy, launch_copy_small((char*)p->theta, (long long)p->nh * 8, p->src, p->N, nullptr, 0, p->stream));
+  } else if (s.exploit_rule != 0) {
+    LAUNCH(p, kCopy, launch_slab_copy_levels(c, p->counters, p->stream));
+  } else {
+    LAUNCH(p, kCopy, launch_slab_copy(c, p->stream));
   }
   return PBT_OK;
 }
@@ -1075,6 +1144,8 @@ int pbt_get_state(pbt_t* p, int member, pbt_state_view* v) {
   }
   CU(p, cudaMemcpyAsync(sc.data(), p->scalars + (size_t)member * PBT_N_SCALARS, PBT_N_SCALARS * 4, cudaMemcpyDeviceToHost, p->stream));
   CU(p, cudaMemcpyAsync(&c, p->counters, sizeof(c), cudaMemcpyDeviceToHost, p->stream));
+  long long tstep = 0;
+  CU(p, cudaMemcpyAsync(&tstep, p->tm + member, 8, cudaMemcpyDeviceToHost, p->stream));
   double hd[PBT_MAX_NH];
   float hf[PBT_MAX_NH];
   double fd = 0;
@@ -1091,7 +1162,7 @@ int pbt_get_state(pbt_t* p, int member, pbt_state_view* v) {
   if (v->scalars) for (int i = 0; i < PBT_N_SCALARS; ++i) v->scalars[i] = sc[i];
   if (v->hparams) for (int k = 0; k < p->nh; ++k) v->hparams[k] = p->toy ? hd[k] : (double)hf[k];
   if (v->fitness) *v->fitness = p->toy ? fd : (double)ff;
-  if (v->step) *v->step = c.step;
+  if (v->step) *v->step = tstep;
   if (v->round) *v->round = c.round;
   return PBT_OK;
 }
@@ -1142,7 +1213,7 @@ int pbt_set_state(pbt_t* p, int member, const pbt_state_view* v) {
     else CU(p, cudaMemcpyAsync((float*)p->fitness + member, &ff, 4, cudaMemcpyHostToDevice, p->stream));
   }
   long long st = 0, rd = 0;
-  if (v->step) { st = *v->step; CU(p, cudaMemcpyAsync(&p->counters->step, &st, 8, cudaMemcpyHostToDevice, p->stream)); }
+  if (v->step) { st = *v->step; CU(p, cudaMemcpyAsync(p->tm + member, &st, 8, cudaMemcpyHostToDevice, p->stream)); }
   if (v->round) { rd = *v->round; CU(p, cudaMemcpyAsync(&p->counters->round, &rd, 8, cudaMemcpyHostToDevice, p->stream)); }
   CU(p, cudaStreamSynchronize(p->stream));  // host staging above lives on this frame
   return PBT_OK;
@@ -1284,9 +1355,7 @@ int pbt_set_batch(pbt_t* p, const void* x, const void* y) {
   const size_t trb = target_row_bytes(p) * s.batch;
   const size_t tsz = s.loss == PBT_LOSS_CE_SOFT ? p->esz : 4;
   CU(p, cudaMemcpy2DAsync(p->ybatch, p->ybatch_stride * tsz, y, trb, trb, p->N, cudaMemcpyDeviceToDevice, p->stream));
-  const int one = 1;
-  CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &one, 4, cudaMemcpyHostToDevice, p->stream));
-  CU(p, cudaStreamSynchronize(p->stream));
+  CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &kOne, 4, cudaMemcpyHostToDevice, p->stream));
   p->supplied_next = true;
   return PBT_OK;
 }
@@ -1295,14 +1364,14 @@ int pbt_step_host(pbt_t* p, const void* x_host, const void* y_host, double* loss
   if (!p || !x_host || !y_host) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
   if (p->toy || p->gan) return fail(p, PBT_ERR_UNSUPPORTED, "host-fed steps are for MLP populations");
   p->launches = 0;
+  set_serial_launches(p->spec.serial_launches != 0);
   const pbt_spec& s = p->spec;
   const size_t xb = (size_t)p->N * s.batch * p->st[0].L[0].in * p->esz;
   CU(p, cudaMemcpyAsync(p->act[0][0], x_host, xb, cudaMemcpyHostToDevice, p->stream));
   const size_t trb = target_row_bytes(p) * s.batch;
   const size_t tsz = s.loss == PBT_LOSS_CE_SOFT ? p->esz : 4;
   CU(p, cudaMemcpy2DAsync(p->ybatch, p->ybatch_stride * tsz, y_host, trb, trb, p->N, cudaMemcpyHostToDevice, p->stream));
-  const int one = 1;
-  CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &one, 4, cudaMemcpyHostToDevice, p->stream));
+  CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &kOne, 4, cudaMemcpyHostToDevice, p->stream));
   p->supplied_next = true;
   int rc = one_step(p);
   if (rc) return rc;
@@ -1321,12 +1390,13 @@ int pbt_prefetch_host_batch(pbt_t* p, const void* x_host, const void* y_host) {
   if (!p->copy_stream) {
     CU(p, cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking));
     CU(p, cudaEventCreateWithFlags(&p->ev_copied, cudaEventDisableTiming));
-    CU(p, cudaEventCreateWithFlags(&p->ev_stepdone[0], cudaEventDisableTiming));
-    CU(p, cudaEventCreateWithFlags(&p->ev_stepdone[1], cudaEventDisableTiming));
+    CU(p, cudaEventCreateWithFlags(&p->ev_release, cudaEventDisableTiming));
   }
   if (p->prefetched) return fail(p, PBT_ERR_STATE, "the previously prefetched batch has not been consumed yet");
-  // the spare buffers were the active ones of the step BEFORE the latest one (which may still be running)
-  if (p->pf_steps >= 2) CU(p, cudaStreamWaitEvent(p->copy_stream, p->ev_stepdone[p->pf_steps & 1], 0));
+  // The spare buffers were the current ones until the latest swap; everything that used them (earlier prefetched
+  // steps, but also pbt_step / pbt_set_batch / pbt_step_host calls made in between) was enqueued before that swap,
+  // where ev_release was recorded.  The step enqueued after the swap may still be running: it uses the other pair.
+  if (p->pf_steps >= 1) CU(p, cudaStreamWaitEvent(p->copy_stream, p->ev_release, 0));
   const pbt_spec& s = p->spec;
   const size_t xb = (size_t)p->N * s.batch * p->st[0].L[0].in * p->esz;
   CU(p, cudaMemcpyAsync(p->act0_alt, x_host, xb, cudaMemcpyHostToDevice, p->copy_stream));
@@ -1340,20 +1410,22 @@ int pbt_prefetch_host_batch(pbt_t* p, const void* x_host, const void* y_host) {
 
 int pbt_step_prefetched(pbt_t* p, double* loss_out_host) {
   if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  set_serial_launches(p->spec.serial_launches != 0);
   if (!p->prefetched) return fail(p, PBT_ERR_STATE, "no batch has been prefetched");
   p->launches = 0;
   p->prefetched = false;
   CU(p, cudaStreamWaitEvent(p->stream, p->ev_copied, 0));
+  // every launch that reads or writes the buffers that become spare now is already in the stream: the next upload
+  // into them waits for this point, not for the step enqueued below
+  CU(p, cudaEventRecord(p->ev_release, p->stream));
   // the uploaded buffers become the current ones; a captured step graph holds the old addresses
   std::swap(p->act[0][0], p->act0_alt);
   std::swap(p->ybatch, p->ybatch_alt);
   if (p->step_graph) { cudaGraphExecDestroy(p->step_graph); p->step_graph = nullptr; }
-  const int one = 1;
-  CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &one, 4, cudaMemcpyHostToDevice, p->stream));
+  CU(p, cudaMemcpyAsync(&p->counters->use_supplied_batch, &kOne, 4, cudaMemcpyHostToDevice, p->stream));
   p->supplied_next = true;
   int rc = one_step(p);
   if (rc) return rc;
-  CU(p, cudaEventRecord(p->ev_stepdone[p->pf_steps & 1], p->stream));
   p->pf_steps++;
   if (loss_out_host) {
     float* tmp = p->host_loss.data();

@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include "pbt.h"
 
@@ -44,15 +45,65 @@ __host__ __device__ inline U4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c
 }
 
 // ---------------------------------------------------------------------------
+// Launching.  Every kernel of the library is launched through launch_with and begins with pdl_prologue(): the
+// launch carries the programmatic-stream-serialization attribute, so the grid may be scheduled while its
+// predecessor in the stream is still draining, and its threads wait in griddepcontrol.wait until the predecessor
+// has completed and its writes are visible; only then do they let their own successor be scheduled.  At most one
+// successor is therefore resident ahead of time, and the data dependences are exactly those of stream order.
+// What is saved is the launch latency and the tail of every kernel boundary, which is most of the time of the
+// small populations.  set_serial_launches(true) drops the attribute (plain stream order).
+// ---------------------------------------------------------------------------
+void set_serial_launches(bool serial);
+bool serial_launches();
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_prologue() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+struct LaunchCfg {
+  dim3 grid, block;
+  size_t smem;
+  cudaStream_t stream;
+  template <typename... KArgs, typename... Args>
+  cudaError_t operator()(void (*kernel)(KArgs...), Args&&... args) const {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = serial_launches() ? 0 : 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(static_cast<Args&&>(args))...);
+  }
+};
+inline LaunchCfg launch_with(dim3 grid, dim3 block, size_t smem, cudaStream_t stream) { return LaunchCfg{grid, block, smem, stream}; }
+#endif
+
+// ---------------------------------------------------------------------------
 // Device-resident counters and status
 // ---------------------------------------------------------------------------
 struct Counters {
-  long long step;    // optimisation steps taken so far (lockstep: one value for the population)
+  long long reserved;  // (the members' step counts live in their own per-member array: see StepClock)
   long long round;   // ready points passed so far
   int status;        // 0, or a pbt_status set by a kernel (bounded wait expired, ...)
   int status_info;   // where it was set
   int use_supplied_batch;  // next step trains on rows supplied by the caller
   int max_level;           // copy passes minus one needed by the last ready point (tournament chains)
+  // (the 32 bytes above are what pbt_grouped_gemm / pbt_selftest_bounded_wait callers provide; the rest exists
+  // only inside a population's workspace)
+  unsigned int bar_count;  // grid barrier of the multi-pass slab copy: arrivals of the current generation
+  unsigned int bar_gen;    // ... and the generation
+};
+
+// Algorithm 1's t, counted per member (members may advance at their own pace).  Kernels that draw from the
+// counter-based generator for "member m at its step t" get the step counts of the members they work on (t[i] belongs
+// to the i-th member of the launch) and the population index of the launch's first member.
+struct StepClock {
+  const long long* t;
+  int member_base;
 };
 
 // ---------------------------------------------------------------------------
@@ -198,6 +249,13 @@ struct CopyArgs {
 cudaError_t launch_slab_copy(const CopyArgs& a, cudaStream_t s);
 cudaError_t launch_copy_small(char* base, long long bytes, const int* src, int n, const int* level, int want_level,
                               cudaStream_t s);
+// Every copy pass 0..counters->max_level in ONE launch (a.level must be set; a.want_level is ignored): the number of
+// passes is read on the device, so the host never waits for the select kernel.  Between passes the blocks meet at a
+// grid barrier (cooperative launch: all blocks are resident), whose wait is bounded: on expiry the kernel sets
+// counters->status = PBT_ERR_TIMEOUT and returns.
+cudaError_t launch_slab_copy_levels(const CopyArgs& a, Counters* counters, cudaStream_t s);
+cudaError_t launch_copy_small_levels(char* base, long long bytes, const int* src, int n, const int* level,
+                                     const Counters* counters, cudaStream_t s);
 
 // misc kernels -------------------------------------------------------------
 cudaError_t launch_init_weights(float* w32, long long p_pad, int n_members, long long w_off, int fan_out,
@@ -207,11 +265,11 @@ cudaError_t launch_f32_to_bf16(const float* in, bf16* out, long long n, cudaStre
 // off = 128 * ((word * n_win) >> 32), word = philox(seed; m, step, batch stream, block).x[word_index]
 // off[m] = first pool row of member m's training window for the current step (the rule of launch_gather_window)
 cudaError_t launch_window_offsets(int* off, int rows, int pool_rows, int n_members, int block, int word_index,
-                                  uint64_t seed, const Counters* counters, cudaStream_t s);
+                                  uint64_t seed, StepClock clk, cudaStream_t s);
 cudaError_t launch_gather_window(char* dst, long long dst_stride_bytes, long long dst_offset_bytes,
                                  const char* pool, int row_bytes, int rows, int pool_rows, int n_members,
                                  int block, int word_index, uint64_t seed, const Counters* counters,
-                                 cudaStream_t s);
+                                 StepClock clk, cudaStream_t s);
 // strided row copy with optional conversion (float -> operand type), per member
 cudaError_t launch_copy_rows(void* dst, int dst_dtype, long long dst_ld, long long dst_stride,
                              const float* src, long long src_ld, long long src_stride, int rows, int cols,
@@ -246,12 +304,12 @@ int energy_partial_count(int n);  // doubles of scratch per member
 // WGAN-GP (Section 4.3.1).  x holds, per member, rows [0,B) real, [B,2B) generated; writes rows [2B,3B):
 // xhat_b = eps_b real_b + (1 - eps_b) fake_b, eps_b from the interpolation stream at (member, step, block j*65536 + b/4)
 cudaError_t launch_gp_interp(void* x, int dtype, long long stride, int B, int dim, int j, int n_members, uint64_t seed,
-                             const Counters* counters, cudaStream_t s);
+                             StepClock clk, cudaStream_t s);
 // gx[m][b][dim] = grad_x D(xhat_b).  row_loss[m][row_off + b] = lam (||gx_b|| - 1)^2 (row stride rows_total) and
 // dv[m][b][:] = (2 lam / B)(||gx_b|| - 1) / ||gx_b|| * gx_b (zero where the norm is zero), in the operand type
 cudaError_t launch_gp_penalty(const float* gx, long long gx_stride, int B, int dim, float lam, float inv_batch,
                               float* row_loss, int rows_total, int row_off, void* dv, int dv_dtype,
                               long long dv_stride, int n_members, cudaStream_t s);
-cudaError_t launch_advance_step(Counters* c, cudaStream_t s);
+cudaError_t launch_advance_step(Counters* c, long long* t, int n_members, cudaStream_t s);
 
 }  // namespace pbt

@@ -195,5 +195,34 @@ inline bool make_map(CUtensorMap* map, const void* base, long long cols, long lo
 }
 
 
+// Per-device launch set-up.  The opt-in shared-memory size is an attribute of the function ON ONE DEVICE, and the SM
+// count differs between devices, so both are resolved for the device that is current at the launch and remembered
+// per device ordinal (a process may drive several GPUs).  Returns the SM count through *sms.
+struct DeviceSetup {
+  static constexpr int kMaxDevices = 64;
+  bool configured[kMaxDevices];
+  int sms[kMaxDevices];
+};
+template <typename Kernel>
+inline cudaError_t device_setup(DeviceSetup* st, Kernel kernel, int smem_bytes, int* sms) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool cached = dev >= 0 && dev < DeviceSetup::kMaxDevices;
+  if (!cached || !st->configured[dev]) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+    if (e != cudaSuccess) return e;
+    int n = 0;
+    e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    if (n <= 0) n = 148;
+    if (cached) { st->sms[dev] = n; st->configured[dev] = true; }
+    *sms = n;
+    return cudaSuccess;
+  }
+  *sms = st->sms[dev];
+  return cudaSuccess;
+}
+
 }  // namespace tc
 }  // namespace pbt

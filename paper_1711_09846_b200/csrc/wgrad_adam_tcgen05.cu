@@ -65,6 +65,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 k_wgrad_adam(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
              const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmM,
              const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmW16, const FusedParams p) {
+  pdl_prologue();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kBarOffset);
@@ -307,21 +308,12 @@ cudaError_t launch_wgrad_adam(const GemmArgs& g, Counters* counters, cudaStream_
   if (!ok) return cudaErrorInvalidValue;
   if (g.a_rowoff) return cudaErrorInvalidValue;   // only the layer input can come from a pool
   if (g.batch > 1 && (g.strideA == 0 || (g.strideB == 0 && !g.b_rowoff))) return cudaErrorInvalidValue;  // operands are per member here
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_wgrad_adam, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (sms <= 0) sms = 148;
-  }
+  static DeviceSetup setup;
+  int sms = 0;
+  cudaError_t e = device_setup(&setup, k_wgrad_adam, kSmemTotal, &sms);
+  if (e != cudaSuccess) return e;
   const int grid = p.num_tiles < sms ? p.num_tiles : sms;
-  k_wgrad_adam<<<grid, kThreads, kSmemTotal, s>>>(tmA, tmB, tmW, tmM, tmV, tmW16, p);
+  launch_with(grid, kThreads, kSmemTotal, s)(k_wgrad_adam, tmA, tmB, tmW, tmM, tmV, tmW16, p);
   return cudaGetLastError();
 }
 
