@@ -371,6 +371,11 @@ def energy_distance_to_ring(x: np.ndarray, n_modes: int = 8) -> float:
 # --------------------------------------------------------------------------
 # optimiser updates on one tensor (float64 arithmetic; caller stores in master precision)
 # --------------------------------------------------------------------------
+def sgd_update(theta, g, lr):
+    """Plain stochastic gradient descent, the `step` Section 3 takes as its example: theta <- theta - lr g."""
+    return theta - lr * g
+
+
 def sgdm_update(theta, vel, g, lr, mu):
     """v <- mu v + g;  theta <- theta - lr v  (no dampening, no Nesterov)."""
     vel = mu * vel + g
@@ -521,7 +526,11 @@ class Population:
         for t in ts:
             self.gW[m][t] = _f32(gW[t])
             self.gb[m][t] = _f32(gb[t])
-        if cfg.optimizer == "sgdm":
+        if cfg.optimizer == "sgd_plain":
+            for t in ts:
+                for P, g in ((self.W, gW[t]), (self.b, gb[t])):
+                    P[m][t] = _f32(sgd_update(P[m][t].astype(np.float64), _f32(g).astype(np.float64), lr))
+        elif cfg.optimizer == "sgdm":
             mu = self._hp(m, "momentum", cfg.momentum)
             for t in ts:
                 for P, O, g in ((self.W, self.o1W, gW[t]), (self.b, self.o1b, gb[t])):

@@ -15,8 +15,9 @@ from workloads import configs as C
 from workloads.generate import Inputs
 
 
-def _mlp_cfg(loss, widths, dtype=C.FP32, opt=C.OPT_SGDM, n=2, batch=6, **kw):
-    slots = ("lr", "momentum") if opt == C.OPT_SGDM else ("lr", "beta1", "wd")
+def _mlp_cfg(loss, widths, dtype=C.FP32, opt=C.OPT_SGDM, n=2, batch=6, slots=None, **kw):
+    if slots is None:
+        slots = ("lr", "momentum") if opt == C.OPT_SGDM else ("lr", "beta1", "wd")
     nh = len(slots)
     return C.PBTConfig(name="t", n_members=n, dtype=dtype, model=C.MLP, loss=loss, optimizer=opt,
                        widths=(tuple(widths),), batch=batch, eval_batch=batch, pool_rows=batch,
@@ -348,3 +349,39 @@ def test_rmsprop_population_step_uses_the_gradient_of_the_loss():
     expect = w0 - 1e-2 * g / (np.sqrt(0.1 * g * g) + float(np.float32(1e-8)))
     np.testing.assert_allclose(pop.W[0][0], expect, rtol=2e-6, atol=1e-9)
     np.testing.assert_allclose(pop.o1W[0][0], np.float32(1.0 - np.float32(0.9)) * g * g, rtol=2e-6)
+
+
+def test_plain_sgd_is_gradient_descent_and_the_zero_momentum_limit():
+    """Section 3's example of `step`: theta <- theta - lr * gradient.  Pinned three ways: the update function on a
+    hand trajectory; one population step against torch.optim.SGD on the same network and batch; and SGD with
+    momentum 0, which takes the same steps."""
+    th = np.array([1.0, -2.0])
+    for _ in range(3):                       # gradient of (1/2)|theta|^2 is theta: theta shrinks by (1 - lr) per step
+        th = O.sgd_update(th, th, 0.25)
+    np.testing.assert_allclose(th, np.array([1.0, -2.0]) * 0.75 ** 3, rtol=1e-15)
+
+    rng = np.random.default_rng(8)
+    cfg = _mlp_cfg(C.LOSS_MSE, (5, 7, 3), batch=16, n=1, opt=C.OPT_SGD, slots=("lr",))
+    inp = _inputs(cfg, rng, [0.05])
+    pop = O.Population(cfg, inp, seed=0)
+    for b in pop.b[0]:
+        b[:] = rng.standard_normal(b.shape).astype(np.float32) * 0.1
+    Ws = [torch.tensor(w.astype(np.float64), requires_grad=True) for w in pop.W[0]]
+    bs = [torch.tensor(b.astype(np.float64), requires_grad=True) for b in pop.b[0]]
+    opt = torch.optim.SGD(Ws + bs, lr=0.05)
+    for _ in range(3):
+        opt.zero_grad()
+        _torch_loss(cfg, Ws, bs, inp.x_pool, inp.y_pool).backward()
+        opt.step()
+        pop.step(1)
+    for w, tw in zip(pop.W[0] + pop.b[0], Ws + bs):
+        np.testing.assert_allclose(w, tw.detach().numpy(), rtol=2e-6, atol=1e-7)
+    assert not any(o.any() for o in pop.o1W[0] + pop.o1b[0])          # no optimiser state is kept
+
+    mom = O.Population(_mlp_cfg(C.LOSS_MSE, (5, 7, 3), batch=16, n=1, opt=C.OPT_SGDM, slots=("lr", "momentum")),
+                       _inputs(cfg, np.random.default_rng(8), [0.05, 0.0]), seed=0)
+    ref = O.Population(cfg, _inputs(cfg, np.random.default_rng(8), [0.05]), seed=0)
+    mom.step(3)
+    ref.step(3)
+    for a, b in zip(mom.W[0] + mom.b[0], ref.W[0] + ref.b[0]):
+        np.testing.assert_array_equal(a, b)

@@ -182,6 +182,13 @@ CONFIGS: Dict[str, PBTConfig] = {
                    pool=512, interval=2, steps=6, name="c4_mini"),
     "c5_mini": _c5(n=10, widths=(128, 192, 256, 136, 72), batch=136, eval_batch=200,
                    pool=768, interval=2, steps=6, name="c5_mini"),
+    # plain SGD (Section 3's example of `step`): learning rate is the only slot
+    "c2_mini_sgd": _c2(n=5, widths=(40, 72, 56, 1), batch=24, eval_batch=40, pool=512, interval=3, steps=6,
+                       name="c2_mini_sgd").replace(optimizer=OPT_SGD, slots=("lr",), priors=(("logu", 1e-4, 1e-1),),
+                                                   perturb=(True,), clamp_lo=(-INF,), clamp_hi=(INF,)),
+    "c3_mini_sgd": _c3(n=6, widths=(72, 136, 200, 10), batch=40, eval_batch=96, pool=640, interval=3, steps=6,
+                       name="c3_mini_sgd").replace(optimizer=OPT_SGD, slots=("lr",), priors=(("logu", 1e-4, 1e-1),),
+                                                   perturb=(True,), clamp_lo=(-INF,), clamp_hi=(INF,)),
     # RMSProp (the optimiser of the paper's RL experiments) on the same small shapes; learning rate is the only slot
     "c2_mini_rms": _c2(n=5, widths=(40, 72, 56, 1), batch=24, eval_batch=40, pool=512, interval=3, steps=6,
                        name="c2_mini_rms").replace(optimizer=OPT_RMSPROP, slots=("lr",), priors=(("logu", 1e-4, 1e-2),),
