@@ -113,8 +113,8 @@ class ClockSampler:
 
 # DRAM bytes per parameter of the fused weight-gradient + Adam kernel, from one `ncu --set full` capture of an
 # 8-member case (the traffic is proportional to the members), valid for the source file with this sha1 only.
-_NCU_TRAFFIC = {"wgrad_adam": {"bytes_per_param": 25.41, "source": "paper_1711_09846_b200/csrc/wgrad_adam_tcgen05.cu",
-                               "sha1": "361db330e5ece7f9d58438bc88611d1a377a3299"}}
+_NCU_TRAFFIC = {"wgrad_adam": {"bytes_per_param": 25.37, "source": "paper_1711_09846_b200/csrc/wgrad_adam_tcgen05.cu",
+                               "sha1": "4f3a44b941b70cfe935a561e5010283c3990f8bd"}}
 
 
 def _ncu_traffic(name, params_per_launch):
@@ -178,7 +178,8 @@ def _algorithmic_work(cfg):
                 if _tc_layer(w[i], w[i + 1], B):
                     fused_params += w[i] * w[i + 1]
                     fused_flops += 2 * B * w[i] * w[i + 1]
-    bpp = {"adam": 16 + 12, "sgdm": 12 + 8, "sgd_plain": 0}[cfg.optimizer] + (2 if cfg.dtype == "bf16_fp32master" else 0)
+    bpp = {"adam": 16 + 12, "sgdm": 12 + 8, "rmsprop": 12 + 8, "sgd_plain": 8 + 4}[cfg.optimizer] + \
+        (2 if cfg.dtype == "bf16_fp32master" else 0)
     n = cfg.n_members
     return {"flops": n * flops, "fused_flops": n * fused_flops, "fused_params": n * fused_params,
             "opt_params": n * opt_params, "opt_bytes_per_param": bpp}

@@ -79,8 +79,8 @@ typedef enum pbt_loss {
 } pbt_loss;
 
 typedef enum pbt_optimizer {
-  PBT_OPT_SGD_PLAIN = 0,
-  PBT_OPT_SGDM = 1,
+  PBT_OPT_SGD_PLAIN = 0, /* theta <- theta - lr g (Section 3's example of step); no optimiser state */
+  PBT_OPT_SGDM = 1,      /* v <- mu v + g, theta <- theta - lr v */
   PBT_OPT_ADAM = 2,
   PBT_OPT_RMSPROP = 3 /* ms <- rho ms + (1-rho) g^2, theta <- theta - lr g / (sqrt(ms) + eps); rho = const_beta2; ms in opt1 */
 } pbt_optimizer;
@@ -133,10 +133,11 @@ typedef struct pbt_spec {
   int32_t fuse_adam; /* 1: apply Adam inside the epilogue of tensor-core weight-gradient GEMMs (the gradient of those
                         layers never goes to HBM); 0: weight gradients are written once and one streaming pass over
                         the slabs applies the update.  Results are bit-identical; only the traffic pattern differs. */
-  int32_t serial_launches; /* 0 (default): kernels are launched with programmatic stream serialization: a kernel may be
-                        scheduled while its predecessor drains and waits on the device until the predecessor's results
-                        are visible (same dependences as stream order, less launch latency); 1: plain stream order.
-                        Results are bit-identical.  The setting of the handle used last applies to the process. */
+  int32_t programmatic_launches; /* 0 (default): plain stream order.  1: kernels are launched with programmatic stream
+                        serialization: a kernel may be scheduled while its predecessor drains and waits on the device
+                        until the predecessor's results are visible (same dependences, bit-identical results).  On a
+                        B200 this was not faster than replaying the captured step in stream order.  The setting of
+                        the handle used last applies to the process. */
   int32_t exploit_rule; /* 0: truncation selection (Section 4.1.1 (b)); 1: binary tournament (Section 4.3.1 (b)): every
                            member draws one other member uniformly and copies it if its fitness is strictly higher;
                            2: t-test selection (Section 4.1.1, exploit (a)): one other member drawn uniformly is

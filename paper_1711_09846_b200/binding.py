@@ -38,7 +38,7 @@ class PbtSpec(C.Structure):
         ("slot_lr", C.c_int32), ("slot_lr_d", C.c_int32), ("slot_momentum", C.c_int32),
         ("slot_beta1", C.c_int32), ("slot_wd", C.c_int32),
         ("perturb_mask", C.c_uint32), ("flags", C.c_uint32),
-        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("serial_launches", C.c_int32), ("exploit_rule", C.c_int32),
+        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("programmatic_launches", C.c_int32), ("exploit_rule", C.c_int32),
         ("explore_rule", C.c_int32), ("prior_kind", C.c_int32 * PBT_MAX_NH),
         ("const_lr", C.c_double), ("const_momentum", C.c_double), ("const_beta1", C.c_double),
         ("const_beta2", C.c_double), ("const_eps", C.c_double), ("const_wd", C.c_double),
@@ -147,7 +147,7 @@ class PbtError(RuntimeError):
         self.code = code
 
 
-def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True, serial_launches: bool = False) -> PbtSpec:
+def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True, programmatic_launches: bool = False) -> PbtSpec:
     """Translate a declarative population description (see workloads.configs.PBTConfig) into pbt_spec."""
     s = PbtSpec()
     s.n_members = cfg.n_members
@@ -175,7 +175,7 @@ def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True, seria
     s.flags = cfg.flags
     s.trunc_num, s.trunc_den = cfg.trunc_num, cfg.trunc_den
     s.keep_grad = 1 if keep_grad else 0
-    s.serial_launches = 1 if serial_launches else 0
+    s.programmatic_launches = 1 if programmatic_launches else 0
     s.exploit_rule = {"truncation": 0, "tournament": 1, "ttest": 2}[getattr(cfg, "exploit", "truncation")]
     s.explore_rule = {"perturb": 0, "resample": 1}[getattr(cfg, "explore", "perturb")]
     s.ttest_alpha = getattr(cfg, "ttest_alpha", 0.05)
@@ -268,7 +268,7 @@ class Population:
     """One population living on one GPU.  Thin wrapper over the pbt_* calls."""
 
     def __init__(self, cfg, inputs, seed: Optional[int] = None, device: str = "cuda:0", keep_grad: bool = False,
-                 fuse_adam: bool = True, guard_bytes: int = 0, serial_launches: bool = False):
+                 fuse_adam: bool = True, guard_bytes: int = 0, programmatic_launches: bool = False):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -277,7 +277,7 @@ class Population:
         self.cfg = cfg
         self.device = torch.device(device)
         self.seed = int(cfg.seed if seed is None else seed)
-        self.spec = spec_from_config(cfg, keep_grad, fuse_adam, serial_launches or bool(os.environ.get("PBT_SERIAL_LAUNCHES")))
+        self.spec = spec_from_config(cfg, keep_grad, fuse_adam, programmatic_launches)
         self.N, self.nh = cfg.n_members, cfg.nh
         self.toy = cfg.model == "toy_quadratic"
         torch.cuda.set_device(self.device)

@@ -147,6 +147,36 @@ static unsigned opt_grid_x(const OptArgs& a) {
   return (unsigned)tiles;
 }
 
+// theta <- theta - lr g (plain gradient descent: no optimiser state is read or written)
+__global__ void __launch_bounds__(kOptThreads) k_sgd(OptArgs a) {
+  pdl_prologue();
+  const int m = blockIdx.y;
+  const float lr = hp(a.H + (long long)m * a.nh_stride, a.slot_lr, a.const_lr);
+  const long long base = (long long)m * a.p_pad + a.begin;
+  float* w = a.w32 + base;
+  const float* g = a.grad + base;
+  bf16* w16 = a.w16 ? a.w16 + base : nullptr;
+  for (long long t0 = (long long)blockIdx.x * kOptTile; t0 < a.count; t0 += (long long)gridDim.x * kOptTile) {
+#pragma unroll
+    for (int j = 0; j < kOptVecPerThread; ++j) {
+      const long long i = t0 + ((long long)j * kOptThreads + threadIdx.x) * 4;
+      if (i < a.count) {
+        const float4 gw = ld_stream(g + i), ww = ld_stream(w + i);
+        float4 nw;
+        nw.x = __fmaf_rn(-lr, gw.x, ww.x); nw.y = __fmaf_rn(-lr, gw.y, ww.y);
+        nw.z = __fmaf_rn(-lr, gw.z, ww.z); nw.w = __fmaf_rn(-lr, gw.w, ww.w);
+        st_stream(w + i, nw);
+        if (w16) st_bf16x4(w16 + i, nw);
+      }
+    }
+  }
+}
+
+cudaError_t launch_sgd(const OptArgs& a, cudaStream_t s) {
+  dim3 grid(opt_grid_x(a), a.n_members);
+  launch_with(grid, kOptThreads, 0, s)(k_sgd, a);
+  return cudaGetLastError();
+}
 cudaError_t launch_sgdm(const OptArgs& a, cudaStream_t s) {
   dim3 grid(opt_grid_x(a), a.n_members);
   launch_with(grid, kOptThreads, 0, s)(k_sgdm, a);

@@ -123,7 +123,7 @@ int fail(pbt_t* p, int code, const char* fmt, ...) {
 namespace pbt {
 void set_last_error(const char* msg) { snprintf(g_err, sizeof(g_err), "%s", msg); }
 namespace {
-bool g_serial_launches = false;
+bool g_serial_launches = true;
 }
 void set_serial_launches(bool serial) { g_serial_launches = serial; }
 bool serial_launches() { return g_serial_launches; }
@@ -170,8 +170,9 @@ int validate(const pbt_spec* s) {
   if (s->model != PBT_MLP && s->model != PBT_GAN_PAIR) return fail(nullptr, PBT_ERR_INVALID_ARG, "unknown model");
   if (s->dtype != PBT_FP32 && s->dtype != PBT_BF16_FP32MASTER)
     return fail(nullptr, PBT_ERR_UNSUPPORTED, "networks run in fp32 or bf16 with fp32 masters");
-  if (s->optimizer != PBT_OPT_SGDM && s->optimizer != PBT_OPT_ADAM && s->optimizer != PBT_OPT_RMSPROP)
-    return fail(nullptr, PBT_ERR_UNSUPPORTED, "network optimiser must be SGD-momentum, RMSProp or Adam");
+  if (s->optimizer != PBT_OPT_SGD_PLAIN && s->optimizer != PBT_OPT_SGDM && s->optimizer != PBT_OPT_ADAM &&
+      s->optimizer != PBT_OPT_RMSPROP)
+    return fail(nullptr, PBT_ERR_UNSUPPORTED, "network optimiser must be plain SGD, SGD-momentum, RMSProp or Adam");
   const int ns = s->model == PBT_GAN_PAIR ? 2 : 1;
   for (int k = 0; k < ns; ++k) {
     if (s->n_layers[k] < 1 || s->n_layers[k] > PBT_MAX_LAYERS) return fail(nullptr, PBT_ERR_INVALID_ARG, "n_layers out of range");
@@ -524,7 +525,8 @@ int finish_optimizer(pbt_handle* h, int k, const bool* fused, const OptArgs& opt
     OptArgs a = opt;
     a.begin = rb; a.count = re - rb;
     rb = re = -1;
-    if (s.optimizer == PBT_OPT_SGDM) { LAUNCH(h, kOpt, launch_sgdm(a, h->stream)); }
+    if (s.optimizer == PBT_OPT_SGD_PLAIN) { LAUNCH(h, kOpt, launch_sgd(a, h->stream)); }
+    else if (s.optimizer == PBT_OPT_SGDM) { LAUNCH(h, kOpt, launch_sgdm(a, h->stream)); }
     else if (s.optimizer == PBT_OPT_RMSPROP) { LAUNCH(h, kOpt, launch_rmsprop(a, h->stream)); }
     else { LAUNCH(h, kOpt, launch_adam(a, h->stream)); }
     return PBT_OK;
@@ -934,7 +936,7 @@ int pbt_destroy(pbt_t* p) {
 
 int pbt_step(pbt_t* p, int k) {
   if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
-  set_serial_launches(p->spec.serial_launches != 0);
+  set_serial_launches(p->spec.programmatic_launches == 0);
   if (k < 0) return fail(p, PBT_ERR_INVALID_ARG, "k must be >= 0");
   p->launches = 0;
   // Small populations are launch-bound: replay one captured step as a CUDA graph.  Capture needs a
@@ -982,7 +984,7 @@ int pbt_step(pbt_t* p, int k) {
 
 int pbt_step_subset(pbt_t* p, const uint8_t* active_host, int k) {
   if (!p || !active_host) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
-  set_serial_launches(p->spec.serial_launches != 0);
+  set_serial_launches(p->spec.programmatic_launches == 0);
   if (k < 0) return fail(p, PBT_ERR_INVALID_ARG, "k must be >= 0");
   if (p->supplied_next) return fail(p, PBT_ERR_STATE, "a caller-supplied batch is pending: it belongs to a step of the whole population");
   p->launches = 0;
@@ -1011,7 +1013,7 @@ static int record_scores(pbt_t* p) {
 
 int pbt_eval(pbt_t* p) {
   if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
-  set_serial_launches(p->spec.serial_launches != 0);
+  set_serial_launches(p->spec.programmatic_launches == 0);
   p->launches = 0;
   const pbt_spec& s = p->spec;
   if (p->toy) {
@@ -1044,7 +1046,7 @@ int pbt_exploit_explore(pbt_t* p) { return pbt_exploit_explore_ready(p, nullptr)
 
 int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host) {
   if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
-  set_serial_launches(p->spec.serial_launches != 0);
+  set_serial_launches(p->spec.programmatic_launches == 0);
   p->launches = 0;
   const pbt_spec& s = p->spec;
   SelectArgs a;
@@ -1364,7 +1366,7 @@ int pbt_step_host(pbt_t* p, const void* x_host, const void* y_host, double* loss
   if (!p || !x_host || !y_host) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
   if (p->toy || p->gan) return fail(p, PBT_ERR_UNSUPPORTED, "host-fed steps are for MLP populations");
   p->launches = 0;
-  set_serial_launches(p->spec.serial_launches != 0);
+  set_serial_launches(p->spec.programmatic_launches == 0);
   const pbt_spec& s = p->spec;
   const size_t xb = (size_t)p->N * s.batch * p->st[0].L[0].in * p->esz;
   CU(p, cudaMemcpyAsync(p->act[0][0], x_host, xb, cudaMemcpyHostToDevice, p->stream));
@@ -1410,7 +1412,7 @@ int pbt_prefetch_host_batch(pbt_t* p, const void* x_host, const void* y_host) {
 
 int pbt_step_prefetched(pbt_t* p, double* loss_out_host) {
   if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
-  set_serial_launches(p->spec.serial_launches != 0);
+  set_serial_launches(p->spec.programmatic_launches == 0);
   if (!p->prefetched) return fail(p, PBT_ERR_STATE, "no batch has been prefetched");
   p->launches = 0;
   p->prefetched = false;

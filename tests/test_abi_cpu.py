@@ -87,7 +87,7 @@ def test_invalid_specs_are_rejected_with_a_message(pkg):
                          (lambda s: setattr(s, "nh", 99), 1),
                          (lambda s: setattr(s, "slot_lr", 7), 1),
                          (lambda s: setattr(s, "dtype", 0), 2),
-                         (lambda s: setattr(s, "optimizer", 0), 2),
+                         (lambda s: setattr(s, "optimizer", 9), 2),
                          (lambda s: setattr(s, "pool_rows", 1), 1),
                          (lambda s: setattr(s, "trunc_den", 0), 1)):
         spec = pkg.spec_from_config(get_config("c2_mini"))

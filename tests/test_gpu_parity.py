@@ -367,6 +367,10 @@ def _check_optimizer_arithmetic(cfg, s0, s1, h):
     g = s1["grad"].astype(np.float64)
     w0, m0, v0 = (s0[k].astype(np.float64) for k in ("w", "opt1", "opt2"))
     lr = h[cfg.slot("lr")]
+    if cfg.optimizer == C.OPT_SGD:
+        np.testing.assert_allclose(s1["w"], O.sgd_update(w0, g, lr), rtol=2e-6, atol=1e-5 * lr)
+        assert not s1["opt1"].any() and not s1["opt2"].any()
+        return
     if cfg.optimizer == C.OPT_SGDM:
         w, m = O.sgdm_update(w0, m0, g, lr, h[cfg.slot("momentum")])
         v = v0
@@ -391,6 +395,7 @@ def _check_optimizer_arithmetic(cfg, s0, s1, h):
 # step / eval parity, step by step, re-seeding the GPU from the oracle at ready points
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("name", ["c2_mini", "c3_mini", "c4_mini", "c5_mini", "c3_mid", "c5_mid", "c4_mid", "c2_mini_rms",
+                                  "c2_mini_sgd", "c3_mini_sgd",
                                   "c3_mini_rms", "c2_mini_ttest", "c3_mini_resample", "c4_mini_wgan", "c4_mini_wgan_fp32",
                                   "c4_mid_wgan", "c2_mini_stagger", "c3_mini_stagger_tournament"])
 def test_step_eval_exploit_parity(pkg, name):
