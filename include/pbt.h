@@ -138,6 +138,12 @@ typedef struct pbt_spec {
                         until the predecessor's results are visible (same dependences, bit-identical results).  On a
                         B200 this was not faster than replaying the captured step in stream order.  The setting of
                         the handle used last applies to the process. */
+  int32_t member_base;  /* this handle holds members [member_base, member_base + n_members) of a larger population that
+                           is sharded over several handles (one per GPU).  Everything that is drawn per member (initial
+                           weights, training rows, interpolation coefficients, donors, explore draws) is keyed by the
+                           member's index in the WHOLE population, so a sharded run takes exactly the steps of the
+                           unsharded one.  0 for an ordinary population. */
+  int32_t n_global;     /* members of the whole population (0: n_members, i.e. not sharded; at most 1024) */
   int32_t exploit_rule; /* 0: truncation selection (Section 4.1.1 (b)); 1: binary tournament (Section 4.3.1 (b)): every
                            member draws one other member uniformly and copies it if its fitness is strictly higher;
                            2: t-test selection (Section 4.1.1, exploit (a)): one other member drawn uniformly is
@@ -275,6 +281,44 @@ int pbt_exploit_explore(pbt_t* p);
  * one per call whatever the mask, so the random draws of successive calls differ.
  */
 int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host);
+
+/*
+ * Ready point of a population that is sharded over several handles (Algorithm 1's exploit / explore; the exchange
+ * takes the place of the shared store of Appendix A.1).  The per-member records that selection looks at are small,
+ * so every shard decides for the WHOLE population and all shards reach the same decisions:
+ *   fitness_global_host  [n_global] doubles, in: p of every member (each shard's pbt_get_fitness, all-gathered);
+ *                        out: after p[b] <- p[src[b]]
+ *   hparams_global_host  [n_global][nh] doubles, in: h of every member; out: after copy and explore
+ *   ready_global_host    n_global bytes or NULL (everybody), as for pbt_exploit_explore_ready
+ *   src_global_out_host  [n_global] int32: the copy map, in indices of the whole population
+ *   level_global_out_host [n_global] int32: copy pass of each recipient (0 under truncation selection; under the
+ *                        tournament rule a donor that is itself a recipient has a higher pass than its readers)
+ *   n_levels_out_host    number of passes
+ * The call runs the same selection / explore kernel as pbt_exploit_explore on these vectors (same draws, keyed by
+ * the ready-point counter, which advances by one), writes the rows of this shard's members back into its own h and
+ * p, and translates the copy map for the shard (pbt_get_copy_map then gives, per local member, its donor's LOCAL
+ * index, or the member itself if it keeps its record or its donor lives on another shard).  It moves no weights.
+ * The caller then goes through the passes in order: for pass L, every slab copy whose recipient has level L is
+ * carried out, the local ones by pbt_copy_members_level(p, L), the ones that cross shards by sending the donor's
+ * slabs (pbt_member_slabs) into the recipient's slabs on the other device (peer copy or send / receive; the data
+ * lands in the recipient's own memory before any kernel reads it).  Within a pass no recipient is anybody's donor.
+ * Truncation selection and the binary tournament; PBT_ERR_UNSUPPORTED for t-test selection (the score histories are
+ * not exchanged).  Synchronises the stream (it returns data to the host).
+ */
+int pbt_exploit_explore_global(pbt_t* p, double* fitness_global_host, double* hparams_global_host,
+                               const uint8_t* ready_global_host, int32_t* src_global_out_host,
+                               int32_t* level_global_out_host, int32_t* n_levels_out_host);
+
+/* The local slab copies of one pass of the copy map left by pbt_exploit_explore_global.  Only enqueues. */
+int pbt_copy_members_level(pbt_t* p, int level);
+
+/*
+ * Device addresses of the arrays that make up one local member's copied record, in a fixed order: fp32 master
+ * weights, first optimiser state, second optimiser state (Adam), bf16 shadow (bf16 populations), Adam's running
+ * beta products; the toy: theta.  ptrs_out_host and bytes_out_host hold up to 5 entries, *count_out_host says how
+ * many are used.  The memory belongs to the caller's workspace; the addresses stay valid until pbt_destroy.
+ */
+int pbt_member_slabs(pbt_t* p, int member, void** ptrs_out_host, size_t* bytes_out_host, int32_t* count_out_host);
 
 /* Read / overwrite one member's record.  get synchronises the stream. */
 int pbt_get_state(pbt_t* p, int member, pbt_state_view* out_host);

@@ -38,7 +38,7 @@ class PbtSpec(C.Structure):
         ("slot_lr", C.c_int32), ("slot_lr_d", C.c_int32), ("slot_momentum", C.c_int32),
         ("slot_beta1", C.c_int32), ("slot_wd", C.c_int32),
         ("perturb_mask", C.c_uint32), ("flags", C.c_uint32),
-        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("programmatic_launches", C.c_int32), ("exploit_rule", C.c_int32),
+        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("programmatic_launches", C.c_int32), ("member_base", C.c_int32), ("n_global", C.c_int32), ("exploit_rule", C.c_int32),
         ("explore_rule", C.c_int32), ("prior_kind", C.c_int32 * PBT_MAX_NH),
         ("const_lr", C.c_double), ("const_momentum", C.c_double), ("const_beta1", C.c_double),
         ("const_beta2", C.c_double), ("const_eps", C.c_double), ("const_wd", C.c_double),
@@ -77,7 +77,8 @@ class PbtGemmDesc(C.Structure):
 
 EXPORTS = [
     "pbt_query_workspace", "pbt_param_count", "pbt_create", "pbt_destroy", "pbt_step", "pbt_step_subset", "pbt_eval",
-    "pbt_exploit_explore", "pbt_exploit_explore_ready", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
+    "pbt_exploit_explore", "pbt_exploit_explore_ready", "pbt_exploit_explore_global", "pbt_copy_members_level",
+    "pbt_member_slabs", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
     "pbt_get_history", "pbt_set_history",
     "pbt_get_hparams", "pbt_set_hparams", "pbt_get_copy_map", "pbt_get_best", "pbt_get_last_loss",
     "pbt_set_batch", "pbt_step_host", "pbt_prefetch_host_batch", "pbt_step_prefetched", "pbt_get_launch_count", "pbt_profile_begin", "pbt_profile_end", "pbt_profile_get",
@@ -112,6 +113,10 @@ def load_library() -> C.CDLL:
     lib.pbt_eval.argtypes = [vp]
     lib.pbt_exploit_explore.argtypes = [vp]
     lib.pbt_exploit_explore_ready.argtypes = [vp, C.POINTER(C.c_uint8)]
+    lib.pbt_exploit_explore_global.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_uint8),
+                                               C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.pbt_copy_members_level.argtypes = [vp, C.c_int]
+    lib.pbt_member_slabs.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(C.c_size_t), C.POINTER(C.c_int32)]
     lib.pbt_get_state.argtypes = [vp, C.c_int, C.POINTER(PbtStateView)]
     lib.pbt_set_state.argtypes = [vp, C.c_int, C.POINTER(PbtStateView)]
     lib.pbt_get_fitness.argtypes = [vp, C.POINTER(C.c_double)]
@@ -268,7 +273,11 @@ class Population:
     """One population living on one GPU.  Thin wrapper over the pbt_* calls."""
 
     def __init__(self, cfg, inputs, seed: Optional[int] = None, device: str = "cuda:0", keep_grad: bool = False,
-                 fuse_adam: bool = True, guard_bytes: int = 0, programmatic_launches: bool = False):
+                 fuse_adam: bool = True, guard_bytes: int = 0, programmatic_launches: bool = False,
+                 member_base: int = 0, n_global: int = 0):
+        """cfg.n_members members on `device`.  member_base / n_global: this population is the shard
+        [member_base, member_base + cfg.n_members) of a population of n_global members (see sharding.py);
+        inputs.init_hparams then holds the rows of the whole population."""
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -278,6 +287,8 @@ class Population:
         self.device = torch.device(device)
         self.seed = int(cfg.seed if seed is None else seed)
         self.spec = spec_from_config(cfg, keep_grad, fuse_adam, programmatic_launches)
+        self.member_base, self.n_global = int(member_base), int(n_global)
+        self.spec.member_base, self.spec.n_global = self.member_base, self.n_global
         self.N, self.nh = cfg.n_members, cfg.nh
         self.toy = cfg.model == "toy_quadratic"
         torch.cuda.set_device(self.device)
@@ -316,6 +327,9 @@ class Population:
             self.workspace[:self._ws_off].fill_(0xA5)
             self.workspace[self._ws_off + nbytes.value:].fill_(0xA5)
         h0 = np.ascontiguousarray(inputs.init_hparams, dtype=np.float64)
+        if self.n_global:
+            assert h0.shape == (self.n_global, self.nh)
+            h0 = np.ascontiguousarray(h0[self.member_base:self.member_base + self.N])
         assert h0.shape == (self.N, self.nh)
         self.handle = C.c_void_p(None)
         torch.cuda.synchronize(self.device)
@@ -378,6 +392,37 @@ class Population:
         mask = np.ascontiguousarray(np.asarray(ready, dtype=bool).astype(np.uint8))
         assert mask.shape == (self.cfg.n_members,)
         self._check(self.lib.pbt_exploit_explore_ready(self.handle, mask.ctypes.data_as(C.POINTER(C.c_uint8))))
+
+    # ----- sharded populations (see sharding.py) ---------------------------
+    def exploit_explore_global(self, fitness_global, hparams_global, ready=None):
+        """Selection and explore for the WHOLE population on this shard's device (every shard gets the same answer);
+        returns (src, level, n_levels, fitness_after, hparams_after) in indices of the whole population and
+        applies the rows of this shard's members to its own records.  Moves no weights."""
+        G = self.n_global
+        f = np.ascontiguousarray(fitness_global, dtype=np.float64).copy()
+        h = np.ascontiguousarray(hparams_global, dtype=np.float64).copy()
+        assert f.shape == (G,) and h.shape == (G, self.nh)
+        src, level = np.zeros(G, dtype=np.int32), np.zeros(G, dtype=np.int32)
+        n_levels = C.c_int32(0)
+        mask = None
+        if ready is not None:
+            mask = np.ascontiguousarray(np.asarray(ready, dtype=bool).astype(np.uint8))
+            assert mask.shape == (G,)
+        self._check(self.lib.pbt_exploit_explore_global(
+            self.handle, f.ctypes.data_as(C.POINTER(C.c_double)), h.ctypes.data_as(C.POINTER(C.c_double)),
+            mask.ctypes.data_as(C.POINTER(C.c_uint8)) if mask is not None else None,
+            src.ctypes.data_as(C.POINTER(C.c_int32)), level.ctypes.data_as(C.POINTER(C.c_int32)), C.byref(n_levels)))
+        return src, level, n_levels.value, f, h
+
+    def copy_members_level(self, level: int):
+        self._check(self.lib.pbt_copy_members_level(self.handle, int(level)))
+
+    def member_slabs(self, m: int):
+        """The arrays of local member m's copied record as uint8 views of the workspace (device memory, no copy)."""
+        ptrs, sizes, n = (C.c_void_p * 5)(), (C.c_size_t * 5)(), C.c_int32(0)
+        self._check(self.lib.pbt_member_slabs(self.handle, int(m), ptrs, sizes, C.byref(n)))
+        base = self.workspace.data_ptr()
+        return [self.workspace[ptrs[i] - base:ptrs[i] - base + sizes[i]] for i in range(n.value)]
 
     # ----- state access ---------------------------------------------------
     def get_state(self, m: int) -> Dict[str, np.ndarray]:

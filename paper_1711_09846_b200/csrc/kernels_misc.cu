@@ -12,12 +12,12 @@ namespace pbt {
 // philox(seed; m, idx >> 2, init stream, tensor_id).x[idx & 3].
 // ---------------------------------------------------------------------------
 __global__ void k_init_weights(float* __restrict__ w32, long long p_pad, long long w_off, long long count,
-                               int tensor_id, float bound, uint64_t seed) {
+                               int tensor_id, float bound, uint64_t seed, int member_base) {
   pdl_prologue();
   const int m = blockIdx.y;
   const long long blk = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (blk * 4 >= count) return;
-  const U4 r = philox4x32_10((uint32_t)m, (uint32_t)blk, kStreamInit, (uint32_t)tensor_id, seed);
+  const U4 r = philox4x32_10((uint32_t)(member_base + m), (uint32_t)blk, kStreamInit, (uint32_t)tensor_id, seed);
   float* dst = w32 + (long long)m * p_pad + w_off;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
@@ -30,11 +30,11 @@ __global__ void k_init_weights(float* __restrict__ w32, long long p_pad, long lo
 }
 
 cudaError_t launch_init_weights(float* w32, long long p_pad, int n_members, long long w_off, int fan_out,
-                                int fan_in, int tensor_id, float bound, uint64_t seed, cudaStream_t s) {
+                                int fan_in, int tensor_id, float bound, uint64_t seed, int member_base, cudaStream_t s) {
   const long long count = (long long)fan_out * fan_in;
   const long long blocks4 = (count + 3) / 4;
   dim3 grid((unsigned)((blocks4 + 255) / 256), n_members);
-  launch_with(grid, 256, 0, s)(k_init_weights, w32, p_pad, w_off, count, tensor_id, bound, seed);
+  launch_with(grid, 256, 0, s)(k_init_weights, w32, p_pad, w_off, count, tensor_id, bound, seed, member_base);
   return cudaGetLastError();
 }
 

@@ -63,6 +63,8 @@ struct pbt_handle {
   int* hist_n;       // [N]
   Counters* counters;
   long long* tm;     // [N] every member's own step count (Algorithm 1's t)
+  // sharded populations: the whole population's selection inputs and outputs (n_global entries each)
+  void* g_fit; void* g_H; int* g_src; int* g_level;
   int member_base;   // population index of the first member the pointers below refer to (0 unless a window is open)
   float* last_loss;  // [N][2]
   double* theta;     // toy: [N][nh]
@@ -162,6 +164,9 @@ int validate(const pbt_spec* s) {
   const int slots[5] = {s->slot_lr, s->slot_lr_d, s->slot_momentum, s->slot_beta1, s->slot_wd};
   for (int i = 0; i < 5; ++i)
     if (slots[i] < -1 || slots[i] >= s->nh) return fail(nullptr, PBT_ERR_INVALID_ARG, "hyperparameter slot out of range");
+  if (s->member_base < 0 || s->n_global < 0 || s->n_global > 1024 ||
+      (s->n_global == 0 && s->member_base != 0) || (s->n_global > 0 && s->member_base + s->n_members > s->n_global))
+    return fail(nullptr, PBT_ERR_INVALID_ARG, "member_base / n_global do not describe a shard of a population of at most 1024 members");
   if (s->model == PBT_TOY_QUADRATIC) {
     if (s->dtype != PBT_FP64_TOY) return fail(nullptr, PBT_ERR_UNSUPPORTED, "the toy model runs in fp64 only");
     if (s->nh < 1) return fail(nullptr, PBT_ERR_INVALID_ARG, "toy model needs nh >= 1");
@@ -219,7 +224,15 @@ size_t plan(pbt_handle* h, char* base) {
   const size_t N = h->N;
   h->counters = (Counters*)take(sizeof(Counters));
   h->tm = (long long*)take(N * sizeof(long long));
-  h->member_base = 0;
+  h->member_base = s.member_base;
+  h->g_fit = h->g_H = nullptr; h->g_src = h->g_level = nullptr;
+  if (s.n_global > 0) {
+    const size_t G = s.n_global;
+    h->g_fit = take(G * sizeof(double));
+    h->g_H = take(G * PBT_MAX_NH * sizeof(double));
+    h->g_src = (int*)take(G * sizeof(int));
+    h->g_level = (int*)take(G * sizeof(int));
+  }
   h->src = (int*)take(N * sizeof(int));
   h->level = (int*)take(N * sizeof(int));
   h->H = take(N * PBT_MAX_NH * sizeof(double));
@@ -908,7 +921,7 @@ int pbt_create(pbt_t** out, const pbt_spec* spec, const double* init_hparams, ui
       for (int l = 0; l < h->st[k].nl; ++l) {
         const Layer& L = h->st[k].L[l];
         const float bound = (float)sqrt(6.0 / (double)L.in);
-        CREATE_CU(launch_init_weights(h->W32, h->P_pad, h->N, L.w_off, L.out, L.in, k * PBT_MAX_LAYERS + l, bound, seed, h->stream));
+        CREATE_CU(launch_init_weights(h->W32, h->P_pad, h->N, L.w_off, L.out, L.in, k * PBT_MAX_LAYERS + l, bound, seed, h->member_base, h->stream));
       }
     if (h->is_bf16) CREATE_CU(launch_f32_to_bf16(h->W32, h->W16, (long long)h->N * h->P_pad, h->stream));
   }
@@ -1044,26 +1057,26 @@ int pbt_eval(pbt_t* p) {
 
 int pbt_exploit_explore(pbt_t* p) { return pbt_exploit_explore_ready(p, nullptr); }
 
-int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host) {
-  if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
-  set_serial_launches(p->spec.programmatic_launches == 0);
-  p->launches = 0;
+// the arguments of the selection / explore kernel for a population of n members whose records are the given arrays
+static void fill_select_args(pbt_t* p, SelectArgs* out, int n, const uint8_t* ready_host, void* H, void* fitness, int* src,
+                             int* level, int* n_cut_out) {
   const pbt_spec& s = p->spec;
-  SelectArgs a;
+  SelectArgs& a = *out;
   memset(&a, 0, sizeof(a));
-  for (int i = 0; i < p->N; ++i)
+  for (int i = 0; i < n; ++i)
     if (!ready_host || ready_host[i]) a.ready_bits[i >> 5] |= 1u << (i & 31);
-  a.n = p->N; a.nh = p->nh;
+  a.n = n; a.nh = p->nh;
   int n_cut = 0;
-  if (p->N >= 2) {
-    long long c = ((long long)p->N * s.trunc_num) / s.trunc_den;
+  if (n >= 2) {
+    long long c = ((long long)n * s.trunc_num) / s.trunc_den;
     if (c < 1) c = 1;
-    if (c > p->N / 2) c = p->N / 2;
+    if (c > n / 2) c = n / 2;
     n_cut = (int)c;
   }
   a.n_cut = n_cut;
+  *n_cut_out = n_cut;
   a.h_is_double = p->toy ? 1 : 0;
-  a.H = p->H; a.fitness = p->fitness; a.src = p->src; a.level = p->level; a.counters = p->counters; a.seed = p->seed;
+  a.H = H; a.fitness = fitness; a.src = src; a.level = level; a.counters = p->counters; a.seed = p->seed;
   a.rule = s.exploit_rule;
   a.hist = p->hist; a.hist_n = p->hist_n; a.alpha = s.ttest_alpha;
   a.explore_rule = s.explore_rule;
@@ -1080,6 +1093,34 @@ int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host) {
   a.perturb_mask = s.perturb_mask; a.flags = s.flags;
   a.factor_lo = s.factor_lo; a.factor_hi = s.factor_hi;
   for (int k = 0; k < PBT_MAX_NH; ++k) { a.clamp_lo[k] = s.clamp_lo[k]; a.clamp_hi[k] = s.clamp_hi[k]; }
+}
+
+// the member-major arrays a slab copy moves (weights, optimiser state, shadow, Adam's running products)
+static void fill_copy_arrays(pbt_t* p, CopyArgs* c) {
+  auto add = [&](void* base, long long stride, long long bytes) {
+    if (!base) return;
+    c->base[c->n_arrays] = (char*)base; c->stride_bytes[c->n_arrays] = stride; c->copy_bytes[c->n_arrays] = bytes;
+    c->n_arrays++;
+  };
+  if (p->toy) return;
+  const long long slab = p->P_pad * 4;
+  add(p->W32, slab, slab);
+  add(p->O1, slab, slab);
+  add(p->O2, slab, slab);
+  add(p->W16, p->P_pad * 2, p->P_pad * 2);
+  add(p->scalars, PBT_N_SCALARS * 4, PBT_N_SCALARS * 4);
+}
+
+int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host) {
+  if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  set_serial_launches(p->spec.programmatic_launches == 0);
+  p->launches = 0;
+  const pbt_spec& s = p->spec;
+  if (s.n_global > 0 && s.n_global != p->N)
+    return fail(p, PBT_ERR_STATE, "a shard of a larger population takes its ready points through pbt_exploit_explore_global");
+  SelectArgs a;
+  int n_cut = 0;
+  fill_select_args(p, &a, p->N, ready_host, p->H, p->fitness, p->src, p->level, &n_cut);
   LAUNCH(p, kSelect, launch_select_explore(a, p->stream));
   if (!(s.flags & PBT_COPY_WEIGHTS) || p->N < 2 || (s.exploit_rule == 0 && n_cut == 0)) return PBT_OK;
   // Truncation: donors are never recipients, one parallel copy pass.  Tournament, t-test: a donor may be a recipient
@@ -1089,19 +1130,7 @@ int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host) {
   memset(&c, 0, sizeof(c));
   c.n = p->N; c.src = p->src;
   c.level = s.exploit_rule != 0 ? p->level : nullptr;
-  auto add = [&](void* base, long long stride, long long bytes) {
-    if (!base) return;
-    c.base[c.n_arrays] = (char*)base; c.stride_bytes[c.n_arrays] = stride; c.copy_bytes[c.n_arrays] = bytes;
-    c.n_arrays++;
-  };
-  if (!p->toy) {
-    const long long slab = p->P_pad * 4;
-    add(p->W32, slab, slab);
-    add(p->O1, slab, slab);
-    add(p->O2, slab, slab);
-    add(p->W16, p->P_pad * 2, p->P_pad * 2);
-    add(p->scalars, PBT_N_SCALARS * 4, PBT_N_SCALARS * 4);
-  }
+  fill_copy_arrays(p, &c);
   if (p->toy) {
     // nh doubles per member: tiny, and not a multiple of 16 bytes in general
     if (s.exploit_rule != 0)
@@ -1113,6 +1142,103 @@ int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host) {
   } else {
     LAUNCH(p, kCopy, launch_slab_copy(c, p->stream));
   }
+  return PBT_OK;
+}
+
+int pbt_exploit_explore_global(pbt_t* p, double* fit_g, double* H_g, const uint8_t* ready_g, int32_t* src_out,
+                               int32_t* level_out, int32_t* n_levels_out) {
+  if (!p || !fit_g || !H_g || !src_out || !level_out || !n_levels_out) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  const pbt_spec& s = p->spec;
+  if (s.n_global <= 0) return fail(p, PBT_ERR_STATE, "the handle was not created as a shard (n_global = 0)");
+  if (s.exploit_rule == 2) return fail(p, PBT_ERR_UNSUPPORTED, "t-test selection is not available for sharded populations");
+  set_serial_launches(s.programmatic_launches == 0);
+  p->launches = 0;
+  const int G = s.n_global;
+  // the whole population's p and h, in the element type of the handle's own records
+  std::vector<double> Hd((size_t)G * PBT_MAX_NH, 0.0);
+  std::vector<float> Hf((size_t)G * PBT_MAX_NH, 0.f), ff(G);
+  for (int m = 0; m < G; ++m) {
+    ff[m] = (float)fit_g[m];
+    for (int k = 0; k < p->nh; ++k) {
+      Hd[(size_t)m * PBT_MAX_NH + k] = H_g[(size_t)m * p->nh + k];
+      Hf[(size_t)m * PBT_MAX_NH + k] = (float)H_g[(size_t)m * p->nh + k];
+    }
+  }
+  if (p->toy) {
+    CU(p, cudaMemcpyAsync(p->g_fit, fit_g, (size_t)G * 8, cudaMemcpyHostToDevice, p->stream));
+    CU(p, cudaMemcpyAsync(p->g_H, Hd.data(), Hd.size() * 8, cudaMemcpyHostToDevice, p->stream));
+  } else {
+    CU(p, cudaMemcpyAsync(p->g_fit, ff.data(), (size_t)G * 4, cudaMemcpyHostToDevice, p->stream));
+    CU(p, cudaMemcpyAsync(p->g_H, Hf.data(), Hf.size() * 4, cudaMemcpyHostToDevice, p->stream));
+  }
+  SelectArgs a;
+  int n_cut = 0;
+  fill_select_args(p, &a, G, ready_g, p->g_H, p->g_fit, p->g_src, p->g_level, &n_cut);
+  LAUNCH(p, kSelect, launch_select_explore(a, p->stream));
+  LAUNCH(p, kSelect, launch_localize_selection(p->g_src, p->g_level, p->g_H, p->g_fit, p->toy ? 1 : 0, s.member_base, p->N,
+                                               p->src, p->level, p->H, p->fitness, p->stream));
+  Counters cnt;
+  CU(p, cudaMemcpyAsync(&cnt, p->counters, sizeof(cnt), cudaMemcpyDeviceToHost, p->stream));
+  CU(p, cudaMemcpyAsync(src_out, p->g_src, (size_t)G * 4, cudaMemcpyDeviceToHost, p->stream));
+  CU(p, cudaMemcpyAsync(level_out, p->g_level, (size_t)G * 4, cudaMemcpyDeviceToHost, p->stream));
+  if (p->toy) {
+    CU(p, cudaMemcpyAsync(fit_g, p->g_fit, (size_t)G * 8, cudaMemcpyDeviceToHost, p->stream));
+    CU(p, cudaMemcpyAsync(Hd.data(), p->g_H, Hd.size() * 8, cudaMemcpyDeviceToHost, p->stream));
+  } else {
+    CU(p, cudaMemcpyAsync(ff.data(), p->g_fit, (size_t)G * 4, cudaMemcpyDeviceToHost, p->stream));
+    CU(p, cudaMemcpyAsync(Hf.data(), p->g_H, Hf.size() * 4, cudaMemcpyDeviceToHost, p->stream));
+  }
+  CU(p, cudaStreamSynchronize(p->stream));
+  if (cnt.status != 0) return fail(p, cnt.status, "a kernel reported status %d (site %d)", cnt.status, cnt.status_info);
+  for (int m = 0; m < G; ++m) {
+    if (!p->toy) fit_g[m] = ff[m];
+    for (int k = 0; k < p->nh; ++k)
+      H_g[(size_t)m * p->nh + k] = p->toy ? Hd[(size_t)m * PBT_MAX_NH + k] : (double)Hf[(size_t)m * PBT_MAX_NH + k];
+  }
+  const bool copies = (s.flags & PBT_COPY_WEIGHTS) && G >= 2 && !(s.exploit_rule == 0 && n_cut == 0);
+  if (!copies) {
+    // no weights move: report an empty copy map so that the caller's exchange has nothing to do
+    for (int m = 0; m < G; ++m) { src_out[m] = m; level_out[m] = 0; }
+    *n_levels_out = 0;
+    return PBT_OK;
+  }
+  *n_levels_out = (s.exploit_rule == 0 ? 0 : cnt.max_level) + 1;
+  return PBT_OK;
+}
+
+int pbt_copy_members_level(pbt_t* p, int level) {
+  if (!p) return fail(nullptr, PBT_ERR_INVALID_ARG, "handle is NULL");
+  if (level < 0) return fail(p, PBT_ERR_INVALID_ARG, "level must be >= 0");
+  if (!(p->spec.flags & PBT_COPY_WEIGHTS) || p->N < 2) return PBT_OK;
+  set_serial_launches(p->spec.programmatic_launches == 0);
+  p->launches = 0;
+  if (p->toy) {
+    LAUNCH(p, kCopy, launch_copy_small((char*)p->theta, (long long)p->nh * 8, p->src, p->N, p->level, level, p->stream));
+    return PBT_OK;
+  }
+  CopyArgs c;
+  memset(&c, 0, sizeof(c));
+  c.n = p->N; c.src = p->src; c.level = p->level; c.want_level = level;
+  fill_copy_arrays(p, &c);
+  LAUNCH(p, kCopy, launch_slab_copy(c, p->stream));
+  return PBT_OK;
+}
+
+int pbt_member_slabs(pbt_t* p, int member, void** ptrs, size_t* bytes, int32_t* count) {
+  if (!p || !ptrs || !bytes || !count) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  if (member < 0 || member >= p->N) return fail(p, PBT_ERR_INVALID_ARG, "member out of range");
+  int n = 0;
+  if (p->toy) {
+    ptrs[n] = p->theta + (size_t)member * p->nh; bytes[n++] = (size_t)p->nh * 8;
+  } else {
+    const size_t off = (size_t)member * p->P_pad;
+    ptrs[n] = p->W32 + off; bytes[n++] = (size_t)p->P_pad * 4;
+    ptrs[n] = p->O1 + off; bytes[n++] = (size_t)p->P_pad * 4;
+    if (p->O2) { ptrs[n] = p->O2 + off; bytes[n++] = (size_t)p->P_pad * 4; }
+    if (p->W16) { ptrs[n] = p->W16 + off; bytes[n++] = (size_t)p->P_pad * 2; }
+    ptrs[n] = p->scalars + (size_t)member * PBT_N_SCALARS; bytes[n++] = PBT_N_SCALARS * 4;
+  }
+  *count = n;
   return PBT_OK;
 }
 

@@ -248,6 +248,12 @@ struct CopyArgs {
   long long stride_bytes[5];
   long long copy_bytes[5];  // multiples of 16
 };
+// After a selection over the whole (sharded) population: rows [base, base + n_local) of the global hyperparameter
+// and fitness vectors become the shard's own, and the global copy map is translated: src_local[i] is the donor's
+// local index if the donor of member base + i lives in this shard, i otherwise (the record arrives from outside).
+cudaError_t launch_localize_selection(const int* src_global, const int* level_global, const void* H_global,
+                                      const void* fit_global, int is_double, int base, int n_local, int* src_local,
+                                      int* level_local, void* H_local, void* fit_local, cudaStream_t s);
 cudaError_t launch_slab_copy(const CopyArgs& a, cudaStream_t s);
 cudaError_t launch_copy_small(char* base, long long bytes, const int* src, int n, const int* level, int want_level,
                               cudaStream_t s);
@@ -261,7 +267,7 @@ cudaError_t launch_copy_small_levels(char* base, long long bytes, const int* src
 
 // misc kernels -------------------------------------------------------------
 cudaError_t launch_init_weights(float* w32, long long p_pad, int n_members, long long w_off, int fan_out,
-                                int fan_in, int tensor_id, float bound, uint64_t seed, cudaStream_t s);
+                                int fan_in, int tensor_id, float bound, uint64_t seed, int member_base, cudaStream_t s);
 cudaError_t launch_f32_to_bf16(const float* in, bf16* out, long long n, cudaStream_t s);
 // copy rows [off, off+rows) of a pool into dst + m*dst_stride_bytes (+ dst_offset_bytes) for every member;
 // off = 128 * ((word * n_win) >> 32), word = philox(seed; m, step, batch stream, block).x[word_index]
