@@ -273,24 +273,28 @@ __global__ void __launch_bounds__(512) k_gemm_colacc(GemmArgs g) {
 // The column-accumulate kernel for bf16 operands with the long dimension a multiple of 8: a thread owns 8
 // consecutive indices of the long dimension (one 16-byte load per batch row), 16 threads cover 128 of them, and the
 // block's 16 slices of K are combined in a fixed order, one short index at a time through 8 KB of shared memory.
-template <bool LONG_A, int ST>
+// LG = lane groups per block (LG * 8 indices of the long dimension), 256 / LG slices of K: 16 x 16 when that gives
+// enough blocks to fill the GPU, 8 x 32 (half as many indices per block, twice the blocks) for small populations.
+template <bool LONG_A, int ST, int LG>
 __global__ void __launch_bounds__(256) k_gemm_colacc_bf16x8(GemmArgs g) {
   pdl_prologue();
-  __shared__ float red[16][128 + 4];
-  const int member = blockIdx.y, lg = threadIdx.x & 15, ks = threadIdx.x >> 4;
+  constexpr int KS = 256 / LG, W = LG * 8;
+  __shared__ float red[KS][W + 4];
+  const int member = blockIdx.y, lg = threadIdx.x % LG, ks = threadIdx.x / LG;
   const int L = LONG_A ? g.M : g.N;
   const long long ldx = LONG_A ? g.lda : g.ldb, ldy = LONG_A ? g.ldb : g.lda;
   const bf16* __restrict__ X = reinterpret_cast<const bf16*>(LONG_A ? g.A : g.B) + member * (LONG_A ? g.strideA : g.strideB);
   const bf16* __restrict__ Y = reinterpret_cast<const bf16*>(LONG_A ? g.B : g.A) + member * (LONG_A ? g.strideB : g.strideA);
-  const int l0 = blockIdx.x * 128 + lg * 8;
+  const int l0 = blockIdx.x * W + lg * 8;
   float acc[8][ST];
 #pragma unroll
   for (int j = 0; j < 8; ++j)
 #pragma unroll
     for (int t = 0; t < ST; ++t) acc[j][t] = 0.f;
   if (l0 < L) {
-#pragma unroll 2
-    for (int k = ks; k < g.K; k += 16) {
+    // short widths leave registers for more loads in flight: a block's 16 slices of K are walked by 8 warps only
+#pragma unroll(ST <= 2 ? 8 : (ST <= 4 ? 4 : 2))
+    for (int k = ks; k < g.K; k += KS) {
       float x[8];
       unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(X + (long long)k * ldx + l0)), x);
       const bf16* yk = Y + (long long)k * ldy;
@@ -302,16 +306,16 @@ __global__ void __launch_bounds__(256) k_gemm_colacc_bf16x8(GemmArgs g) {
       }
     }
   }
-  const int l = blockIdx.x * 128 + threadIdx.x;
+  const int l = blockIdx.x * W + threadIdx.x;
 #pragma unroll
   for (int t = 0; t < ST; ++t) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) red[ks][lg * 8 + j] = acc[j][t];
     __syncthreads();
-    if (threadIdx.x < 128 && l < L) {
+    if (threadIdx.x < W && l < L) {
       float v = 0.f;
 #pragma unroll
-      for (int q = 0; q < 16; ++q) v += red[q][threadIdx.x];
+      for (int q = 0; q < KS; ++q) v += red[q][threadIdx.x];
       const int m = LONG_A ? l : t, n = LONG_A ? t : l;
       store_one(g, member, m, n, epilogue_one(g, member, m, n, v, 1));
     }
@@ -321,17 +325,18 @@ __global__ void __launch_bounds__(256) k_gemm_colacc_bf16x8(GemmArgs g) {
 
 template <bool LONG_A, int ST>
 static void launch_colacc_vec_n(const GemmArgs& g, int L, cudaStream_t s) {
-  launch_with(dim3((L + 127) / 128, g.batch), 256, 0, s)(k_gemm_colacc_bf16x8<LONG_A, ST>, g);
+  if ((long long)((L + 127) / 128) * g.batch >= 296)
+    launch_with(dim3((L + 127) / 128, g.batch), 256, 0, s)(k_gemm_colacc_bf16x8<LONG_A, ST, 16>, g);
+  else
+    launch_with(dim3((L + 63) / 64, g.batch), 256, 0, s)(k_gemm_colacc_bf16x8<LONG_A, ST, 8>, g);
 }
 template <bool LONG_A>
 static bool launch_colacc_vec(const GemmArgs& g, cudaStream_t s) {
   const int L = LONG_A ? g.M : g.N, S = LONG_A ? g.N : g.M;
   const long long ldx = LONG_A ? g.lda : g.ldb, sx = LONG_A ? g.strideA : g.strideB;
   const void* X = LONG_A ? g.A : g.B;
-  if (g.in_dtype != kBF16 || L % 8 != 0 || L < 128 || ldx % 8 != 0 || sx % 8 != 0 || ((uintptr_t)X & 15) || g.batch > 65535)
+  if (g.in_dtype != kBF16 || L % 8 != 0 || L < 64 || ldx % 8 != 0 || sx % 8 != 0 || ((uintptr_t)X & 15) || g.batch > 65535)
     return false;
-  // one block per 128 indices and problem: worth it only when that fills the GPU (the scalar kernel has 4x the blocks)
-  if ((long long)((L + 127) / 128) * g.batch < 200) return false;
   switch (S) {   // one instantiation per width: no predicated-off columns in the inner loop
     case 1: launch_colacc_vec_n<LONG_A, 1>(g, L, s); break;   case 2: launch_colacc_vec_n<LONG_A, 2>(g, L, s); break;
     case 3: launch_colacc_vec_n<LONG_A, 3>(g, L, s); break;   case 4: launch_colacc_vec_n<LONG_A, 4>(g, L, s); break;
@@ -446,6 +451,88 @@ __global__ void __launch_bounds__(256) k_gemm_smallk_bf16x8(GemmArgs g) {
   }
 }
 
+// The same product for K <= 4 (a critic's two-wide input layer, the data gradient of its one-wide output layer) with
+// the roles turned around: a thread keeps the weights and the bias of ITS 8 columns in registers and walks down the
+// rows, so that per output vector there is one small broadcast load of the row's K inputs, K x 8 multiply-adds,
+// the mask load and one 16-byte store, with four rows in flight.  A block covers all columns (up to 2048) and
+// kRowsPerLane rows per row lane.  Same multiply-add order per element as the kernels above.
+constexpr int kRowsPerLane = 16;
+template <bool B_MN, int KK>
+__global__ void __launch_bounds__(256) k_gemm_tinyk_bf16x8(GemmArgs g) {
+  pdl_prologue();
+  const int member = blockIdx.z;
+  const int groups = g.N >> 3;
+  const int tpr = groups < 256 ? groups : 256;          // threads across one row
+  const int lanes = 256 / tpr;                          // rows worked on at a time
+  const int cg = threadIdx.x % tpr, rl = threadIdx.x / tpr;
+  if (rl >= lanes) return;
+  const int n = (blockIdx.x * tpr + cg) << 3;
+  if (n >= g.N) return;
+  const bf16* __restrict__ A = reinterpret_cast<const bf16*>(g.A) + member * g.strideA;
+  const bf16* __restrict__ B = reinterpret_cast<const bf16*>(g.B) + member * g.strideB;
+  float b[KK][8], bias[8];
+#pragma unroll
+  for (int k = 0; k < KK; ++k) {
+    if (B_MN) {
+      unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(B + (long long)k * g.ldb + n)), b[k]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) b[k][j] = __bfloat162float(B[(long long)(n + j) * g.ldb + k]);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) bias[j] = g.bias ? g.bias[member * g.strideBias + n + j] : 0.f;
+  const bf16* mask = g.mask ? reinterpret_cast<const bf16*>(g.mask) + member * g.strideMask : nullptr;
+  bf16* C = reinterpret_cast<bf16*>(g.C) + member * g.strideC;
+  const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
+  const int m_begin = blockIdx.y * (lanes * kRowsPerLane) + rl;
+  const int m_end = min(g.M, (int)(blockIdx.y + 1) * (lanes * kRowsPerLane));
+#pragma unroll 4
+  for (int m = m_begin; m < m_end; m += lanes) {
+    float a[KK];
+#pragma unroll
+    for (int k = 0; k < KK; ++k) a[k] = __bfloat162float(A[(long long)m * g.lda + k]);
+    float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int k = 0; k < KK; ++k)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = fmaf(a[k], b[k][j], v[j]);
+    if (g.bias) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] += bias[j];
+    }
+    if (g.relu) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = fmaxf(v[j], 0.f);
+    }
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      __nv_bfloat162 t = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+      o[j] = *reinterpret_cast<uint32_t*>(&t);
+    }
+    if (mask) {
+      const uint4 mk = __ldg(reinterpret_cast<const uint4*>(mask + (long long)m * g.ldmask + n));
+      const uint32_t mu[4] = {mk.x, mk.y, mk.z, mk.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) o[j] &= __hgt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&mu[j]), zero2);
+    }
+    *reinterpret_cast<uint4*>(C + (long long)m * g.ldc + n) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+template <bool B_MN>
+static void launch_tinyk(const GemmArgs& g, cudaStream_t s) {
+  const int groups = g.N >> 3, tpr = groups < 256 ? groups : 256, lanes = 256 / tpr;
+  const dim3 grid((groups + tpr - 1) / tpr, (g.M + lanes * kRowsPerLane - 1) / (lanes * kRowsPerLane), g.batch);
+  switch (g.K) {
+    case 1: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 1>, g); break;
+    case 2: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 2>, g); break;
+    case 3: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 3>, g); break;
+    default: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 4>, g); break;
+  }
+}
+
 static bool smallk_vec_ok(const GemmArgs& g) {
   if (g.in_dtype != kBF16 || g.out_dtype != kBF16 || g.K < 1 || g.K > kSkinny || g.N % 8 != 0) return false;
   if (g.ldc % 8 || g.strideC % 8 || ((uintptr_t)g.C & 15)) return false;
@@ -477,6 +564,12 @@ static void launch_colacc(const GemmArgs& g, cudaStream_t s) {
 
 template <typename T>
 static bool launch_skinny(const GemmArgs& g, cudaStream_t s) {
+  if (smallk_vec_ok(g) && g.K <= 4 && !g.a_mn && g.N >= 8 &&
+      (long long)((g.M + kRowsPerLane - 1) / kRowsPerLane) <= 65535) {
+    if (g.b_mn) launch_tinyk<true>(g, s);
+    else launch_tinyk<false>(g, s);
+    return true;
+  }
   if (smallk_vec_ok(g)) {
     const int per_slab = kSmallKRows * (g.N / 8);
     const dim3 grid((per_slab + 255) / 256 > 8 ? 8 : (per_slab + 255) / 256, (g.M + kSmallKRows - 1) / kSmallKRows, g.batch);

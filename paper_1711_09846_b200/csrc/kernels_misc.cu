@@ -426,6 +426,80 @@ __global__ void __launch_bounds__(256) k_bias_grad_bf16x8(const bf16* __restrict
   }
 }
 
+// The same sums for populations whose layers are too narrow to fill the GPU with one block per 256 columns: a block
+// owns 64 columns, 8 threads x 16 bytes across and 32 row lanes down (a warp reads 4 rows x 128 contiguous bytes),
+// every thread keeps 8 loads in flight, and the 32 partial sums of a column are combined in a fixed order.
+__global__ void __launch_bounds__(256) k_bias_grad_bf16x8_tall(const bf16* __restrict__ dz, long long ld, long long stride,
+                                                               int rows, int cols, float* __restrict__ out,
+                                                               long long out_stride) {
+  pdl_prologue();
+  __shared__ float sh[32][64 + 1];
+  const int m = blockIdx.y, cl = threadIdx.x & 7, rl = threadIdx.x >> 3;
+  const int c0 = blockIdx.x * 64 + cl * 8;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (c0 < cols) {
+    const bf16* p = dz + m * stride + c0;
+#pragma unroll 8
+    for (int r = rl; r < rows; r += 32) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(p + (long long)r * ld));
+      const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        acc[2 * j] += __uint_as_float(u[j] << 16);
+        acc[2 * j + 1] += __uint_as_float(u[j] & 0xFFFF0000u);
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) sh[rl][cl * 8 + j] = acc[j];
+  __syncthreads();
+  const int c = blockIdx.x * 64 + threadIdx.x;
+  if (threadIdx.x < 64 && c < cols) {
+    float t = 0.f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) t += sh[j][threadIdx.x];
+    out[m * out_stride + c] = t;
+  }
+}
+
+// Column sums of a narrow matrix (one-, two- or ten-wide output layers): one block per member, thread t adds rows
+// t, t + 256, ..., then the 256 partial sums of a column are combined in a fixed order (warp shuffles, then warps).
+template <typename T>
+__global__ void __launch_bounds__(256) k_bias_grad_narrow(const T* __restrict__ dz, long long ld, long long stride, int rows,
+                                                          int cols, float* __restrict__ out, long long out_stride) {
+  pdl_prologue();
+  __shared__ float sh[8][16];
+  const int m = blockIdx.x, lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const T* p = dz + m * stride;
+  float acc[16];
+#pragma unroll
+  for (int c = 0; c < 16; ++c) acc[c] = 0.f;
+  for (int r = threadIdx.x; r < rows; r += 256) {
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+      if (c < cols) {
+        if constexpr (sizeof(T) == 2) acc[c] += __bfloat162float(p[(long long)r * ld + c]);
+        else acc[c] += p[(long long)r * ld + c];
+      }
+  }
+#pragma unroll
+  for (int c = 0; c < 16; ++c) {
+    if (c < cols) {
+      float v = acc[c];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) sh[w][c] = v;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < cols) {
+    float t = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) t += sh[j][threadIdx.x];
+    out[m * out_stride + threadIdx.x] = t;
+  }
+}
+
 cudaError_t launch_bias_grad(const void* dz, int dz_dtype, long long ld, long long stride, int rows, int cols,
                              float* out, long long out_stride, int n_members, cudaStream_t s) {
   // the wide kernel has one block per 256 columns and member: only when that fills the GPU twice over
@@ -433,6 +507,19 @@ cudaError_t launch_bias_grad(const void* dz, int dz_dtype, long long ld, long lo
       stride % 8 == 0 && ((uintptr_t)dz & 15) == 0) {
     dim3 grid((cols + 255) / 256, n_members);
     launch_with(grid, 256, 0, s)(k_bias_grad_bf16x8, (const bf16*)dz, ld, stride, rows, cols, out, out_stride);
+    return cudaGetLastError();
+  }
+  if (dz_dtype == kBF16 && cols % 8 == 0 && cols >= 64 && rows >= 64 && ld % 8 == 0 && stride % 8 == 0 &&
+      ((uintptr_t)dz & 15) == 0) {
+    dim3 grid((cols + 63) / 64, n_members);
+    launch_with(grid, 256, 0, s)(k_bias_grad_bf16x8_tall, (const bf16*)dz, ld, stride, rows, cols, out, out_stride);
+    return cudaGetLastError();
+  }
+  if (cols <= 16 && rows >= 256) {
+    if (dz_dtype == kBF16)
+      launch_with(n_members, 256, 0, s)(k_bias_grad_narrow<bf16>, (const bf16*)dz, ld, stride, rows, cols, out, out_stride);
+    else
+      launch_with(n_members, 256, 0, s)(k_bias_grad_narrow<float>, (const float*)dz, ld, stride, rows, cols, out, out_stride);
     return cudaGetLastError();
   }
   dim3 grid((cols + 31) / 32, n_members), block(32, 8);

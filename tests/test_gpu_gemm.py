@@ -99,7 +99,8 @@ def test_tensor_core_shared_operand(env):
                                    (3, 200, 300, 2), (515, 2, 1024, 2), (1, 520, 1031, 2), (300, 16, 40, 1), (16, 300, 40, 1),
                                    (70, 136, 2, 2), (33, 512, 1, 3), (64, 64, 4, 1), (40, 72, 3, 2), (1030, 512, 2, 2),
                                    (45, 264, 5, 2), (512, 10, 256, 2), (10, 1024, 256, 3), (256, 10, 1024, 2), (136, 1, 512, 2),
-                                   (8, 264, 72, 2), (2, 512, 1024, 2), (264, 16, 200, 1), (40, 1024, 10, 2)])
+                                   (8, 264, 72, 2), (2, 512, 1024, 2), (264, 16, 200, 1), (40, 1024, 10, 2),
+                                   (100, 2304, 2, 1), (1024, 512, 1, 2), (300, 8, 4, 2)])
 def test_alu_engine(env, dtype, a_mn, b_mn, shape):
     pkg, torch = env
     M, N, K, batch = shape
