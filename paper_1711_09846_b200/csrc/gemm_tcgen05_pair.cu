@@ -28,7 +28,8 @@ constexpr int kPEpiW = 8;         // epilogue warps per CTA
 constexpr int kPThreads = 64 + 32 * kPEpiW;
 constexpr int kPABytes = kBM * kBK * 2, kPBBytes = (kPN / 2) * kBK * 2, kPStageBytes = kPABytes + kPBBytes;
 constexpr int kPEpiOffset = kPStages * kPStageBytes;
-constexpr int kPEpiBytesPerWarp = 32 * kEpiPitch * 4;
+constexpr int kPEpiBytesPerWarp = 8192;   // two staging boxes of 32 rows x 128 bytes (the transposing path uses 4.5 KB of it)
+static_assert(kPEpiBytesPerWarp >= 32 * kEpiPitch * 4 && kPEpiOffset % 1024 == 0, "staging boxes are 1024-byte aligned");
 constexpr int kPBarOffset = kPEpiOffset + kPEpiW * kPEpiBytesPerWarp;
 constexpr int kPSmemTotal = kPBarOffset + 256 + 1024;
 static_assert(kPSmemTotal <= 232448, "shared memory budget of one CTA");
@@ -84,7 +85,8 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t cluster_addr) {
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
-k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmC, const TcParams p) {
   pdl_prologue();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -204,7 +206,9 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else {
     // ------------------------------ epilogue (both CTAs, own 128 rows) ------------------------------
     const int q = warp & 3, e = warp - 2, half = e >> 2;
-    float* buf = reinterpret_cast<float*>(smem + kPEpiOffset + e * kPEpiBytesPerWarp);
+    uint8_t* stage = smem + kPEpiOffset + e * kPEpiBytesPerWarp;
+    float* buf = reinterpret_cast<float*>(stage);
+    uint32_t boxes_used = 0;
     int it = 0;
     bool ok = true;
     const int esz = p.out_dtype == kBF16 ? 2 : 4;
@@ -217,12 +221,19 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int acc = it & 1;
       if (!mbar_wait(&tfull[acc], (it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      epilogue_tile<kPN, kPEpiW>(p, buf, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kPN), member, m0, n0, q,
-                                 half, lane, vec_ok);
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kPN);
+      if (p.c_tma && m0 + kBM <= p.M && n0 + kPN <= p.N && (p.out_dtype == kBF16 || !p.mask)) {
+        epilogue_tile_tma<kPN, kPEpiW>(p, &tmC, stage, tacc, member, m0, n0, q, half, lane, boxes_used);
+      } else {
+        if (lane == 0) tma_store_wait_all();   // the transposing path reuses the staging memory
+        __syncwarp();
+        epilogue_tile<kPN, kPEpiW>(p, buf, tacc, member, m0, n0, q, half, lane, vec_ok);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty[acc]), 0));
     }
+    if (lane == 0) tma_store_wait_all();     // the bulk stores have read the staging boxes and reached memory
     if (!ok && lane == 0) {
       *abort_flag = 1;
       atomicCAS(&p.counters->status, 0, PBT_ERR_TIMEOUT);
@@ -268,13 +279,24 @@ cudaError_t launch_gemm_tc_pair(const GemmArgs& g, Counters* counters, cudaStrea
   if (!g.b_mn) ok = make_map(&tmB, g.B, g.K, b_rows, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kPN / 2);
   else ok = make_map(&tmB, g.B, g.N, b_rows, g.ldb, p.b_batched ? g.batch : 1, g.strideB, kBK);
   if (!ok) return cudaErrorInvalidValue;
+  // C as a tensor map (boxes of 32 rows x 128 bytes, 128-byte swizzle) when its layout allows bulk stores
+  CUtensorMap tmC;
+  memset(&tmC, 0, sizeof(tmC));
+  {
+    const int esz = g.out_dtype == kBF16 ? 2 : 4;
+    const bool mask_ok = !g.mask || ((((uintptr_t)g.mask) & 15) == 0 && g.ldmask % 8 == 0 && g.strideMask % 8 == 0);
+    const bool bias_ok = !g.bias || ((((uintptr_t)g.bias) & 15) == 0 && g.strideBias % 4 == 0);
+    if (mask_ok && bias_ok && (((uintptr_t)g.C) & 15) == 0 && (g.ldc * esz) % 16 == 0 && (g.strideC * esz) % 16 == 0 &&
+        make_map(&tmC, g.C, g.N, g.M, g.ldc, g.batch, g.strideC, 32, esz, 128 / esz, 128))
+      p.c_tma = 1;
+  }
   static DeviceSetup setup;
   int sms = 0;
   cudaError_t e = device_setup(&setup, k_gemm_tc_pair, kPSmemTotal, &sms);
   if (e != cudaSuccess) return e;
   int pairs = sms / 2;
   if (pairs > p.num_tiles) pairs = p.num_tiles;
-  launch_with(2 * pairs, kPThreads, kPSmemTotal, s)(k_gemm_tc_pair, tmA, tmB, p);
+  launch_with(2 * pairs, kPThreads, kPSmemTotal, s)(k_gemm_tc_pair, tmA, tmB, tmC, p);
   return cudaGetLastError();
 }
 

@@ -18,6 +18,7 @@ struct TcParams {
   void* C; long long ldc, strideC; int out_dtype;
   const float* bias; long long strideBias; int relu;
   const bf16* mask; long long ldmask, strideMask;
+  int c_tma;             // the kernel was given a tensor map of C: interior tiles leave through bulk tensor stores
   Counters* counters;
   const int* a_rowoff;   // per-problem first row of the A / B operand inside a shared matrix (null: batched operand)
   const int* b_rowoff;
@@ -193,6 +194,109 @@ __device__ __forceinline__ void epilogue_tile(const TcParams& p, float* buf, uin
       }
     }
 }
+}
+
+// Interior tiles when a tensor map of C is available.  A thread's TMEM lane is a row of the tile, so after
+// tcgen05.ld a thread holds 32 consecutive columns of ITS row: bias / ReLU / conversion / mask are applied in
+// registers and the row segment goes, with the 128-byte swizzle of the tensor map (16-byte chunk index XOR row & 7,
+// which also makes the warp's 16-byte shared-memory stores conflict-free), into a staging box of 32 rows x 128 bytes;
+// one lane then issues a bulk tensor store of the box.  No transpose through shared memory and no per-thread global
+// stores.  `stage` is this warp's 8 KB (two boxes, 1024-byte aligned): a box is rewritten only after the store that
+// read it two boxes ago has finished reading.  bf16 output: a box is 64 columns (two 32-column chunks); fp32: 32.
+template <int BN, int NEPIW>
+__device__ __forceinline__ void epilogue_tile_tma(const TcParams& p, const CUtensorMap* tmC, uint8_t* stage, uint32_t tacc,
+                                                  int member, int m0, int n0, int q, int half, int lane,
+                                                  uint32_t& boxes_used) {
+  constexpr int kCols = BN / (NEPIW / 4);   // columns of the tile this warp drains
+  constexpr int kChunks = kCols / 32;
+  const int cbase = half * kCols;
+  const float* bias = p.bias ? p.bias + member * p.strideBias + n0 + cbase : nullptr;
+  const long long row = m0 + q * 32 + lane;
+  const uint32_t sw = (uint32_t)(lane & 7);
+  uint32_t r[32];
+  tmem_ld32(tacc + cbase, r);
+  if (p.out_dtype == kBF16) {
+    const bf16* mrow = p.mask ? p.mask + member * p.strideMask + row * p.ldmask + n0 + cbase : nullptr;
+    const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f);
+#pragma unroll 1
+    for (int c = 0; c < kChunks; ++c) {
+      uint4 mk[4];
+      if (mrow) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) mk[j] = __ldg(reinterpret_cast<const uint4*>(mrow + c * 32) + j);
+      }
+      uint8_t* box = stage + (boxes_used & 1u) * 4096u;
+      if ((c & 1) == 0) {
+        if (lane == 0) tma_store_wait_read_but_one();
+        __syncwarp();
+      }
+      tmem_ld_wait();
+      uint32_t o[16];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float x0 = __uint_as_float(r[4 * j]), x1 = __uint_as_float(r[4 * j + 1]);
+        float x2 = __uint_as_float(r[4 * j + 2]), x3 = __uint_as_float(r[4 * j + 3]);
+        if (bias) {
+          const float4 bv = __ldg(reinterpret_cast<const float4*>(bias + c * 32) + j);   // same address in every lane
+          x0 += bv.x; x1 += bv.y; x2 += bv.z; x3 += bv.w;
+        }
+        if (p.relu) { x0 = fmaxf(x0, 0.f); x1 = fmaxf(x1, 0.f); x2 = fmaxf(x2, 0.f); x3 = fmaxf(x3, 0.f); }
+        __nv_bfloat162 t0 = __floats2bfloat162_rn(x0, x1), t1 = __floats2bfloat162_rn(x2, x3);
+        o[2 * j] = *reinterpret_cast<uint32_t*>(&t0);
+        o[2 * j + 1] = *reinterpret_cast<uint32_t*>(&t1);
+      }
+      if (c + 1 < kChunks) tmem_ld32(tacc + cbase + (c + 1) * 32, r);
+      if (mrow) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          o[4 * j] &= __hgt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&mk[j].x), zero2);
+          o[4 * j + 1] &= __hgt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&mk[j].y), zero2);
+          o[4 * j + 2] &= __hgt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&mk[j].z), zero2);
+          o[4 * j + 3] &= __hgt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&mk[j].w), zero2);
+        }
+      }
+      const uint32_t hh = (uint32_t)(c & 1) * 4u;
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        *reinterpret_cast<uint4*>(box + lane * 128 + (((hh + j) ^ sw) << 4)) = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+      if (c & 1) {
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_3d(tmC, box, n0 + cbase + (c - 1) * 32, m0 + q * 32, member);
+          tma_store_commit();
+        }
+        ++boxes_used;
+      }
+    }
+  } else {
+#pragma unroll 1
+    for (int c = 0; c < kChunks; ++c) {
+      uint8_t* box = stage + (boxes_used & 1u) * 4096u;
+      if (lane == 0) tma_store_wait_read_but_one();
+      __syncwarp();
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                               __uint_as_float(r[4 * j + 3]));
+        if (bias) {
+          const float4 bv = __ldg(reinterpret_cast<const float4*>(bias + c * 32) + j);
+          v.x += bv.x; v.y += bv.y; v.z += bv.z; v.w += bv.w;
+        }
+        if (p.relu) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f); }
+        *reinterpret_cast<float4*>(box + lane * 128 + ((((uint32_t)j) ^ sw) << 4)) = v;
+      }
+      if (c + 1 < kChunks) tmem_ld32(tacc + cbase + (c + 1) * 32, r);
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        tma_store_3d(tmC, box, n0 + cbase + c * 32, m0 + q * 32, member);
+        tma_store_commit();
+      }
+      ++boxes_used;
+    }
+  }
 }
 
 }  // namespace tc
