@@ -799,14 +799,6 @@ class Population:
             A[dst] = [x.copy() for x in rows]
         self.scalars[dst] = scalars
 
-    def _copy_member(self, dst, src):
-        if self.toy:
-            self.theta[dst] = self.theta[src]
-            return
-        for A in (self.W, self.b, self.o1W, self.o1b, self.o2W, self.o2b):
-            A[dst] = [x.copy() for x in A[src]]
-        self.scalars[dst] = self.scalars[src]
-
     def best(self) -> int:
         """Member with the highest p; the lowest index wins ties (Algorithm 1, return)."""
         return rank_members(self.fitness)[0]

@@ -445,6 +445,14 @@ class Population:
         out.update(scalars=sc, hparams=hp[:self.nh], fitness=fit.value, step=step.value, round=rnd.value)
         return out
 
+    def step_count(self, m: int = 0) -> int:
+        """Member m's own step count t (Algorithm 1's t); reads one counter, not the member's record."""
+        step = C.c_int64(0)
+        v = PbtStateView()
+        v.step = C.pointer(step)
+        self._check(self.lib.pbt_get_state(self.handle, int(m), C.byref(v)))
+        return step.value
+
     def set_state(self, m: int, w=None, opt1=None, opt2=None, scalars=None, hparams=None, fitness=None,
                   step=None, round=None):
         dt = np.float64 if self.toy else np.float32
@@ -638,7 +646,7 @@ class Population:
         reads."""
         cfg = self.cfg
         total = cfg.total_steps if total_steps is None else total_steps
-        done = int(self.get_state(0)["step"])
+        done = self.step_count(0)
         offsets = tuple(getattr(cfg, "ready_offsets", ())) or (0,) * cfg.n_members
         iv = cfg.ready_interval
         while done < total:
