@@ -173,36 +173,49 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& w, float* f) {
 // The row-dot kernel for bf16 operands that are both K-major with K a multiple of 8: a lane takes 8 consecutive k
 // per trip with one 16-byte load per operand row.  The scalar form above is bound by instruction issue (address
 // arithmetic, conversion and one multiply-add per 2-byte load); this one issues about a third as many.
-template <int NT>
+// A warp works on RPW rows at a time, so that every 16-byte load of a B row serves RPW rows of A and RPW + NT loads
+// are in flight per trip; the sum of a row is formed in the same order whatever RPW is.
+template <int NT, int RPW>
 __global__ void __launch_bounds__(256) k_gemm_rowdot_bf16x8(GemmArgs g) {
   pdl_prologue();
   const int member = blockIdx.y, lane = threadIdx.x & 31;
-  const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (m >= g.M) return;
-  const bf16* __restrict__ A = reinterpret_cast<const bf16*>(g.A) + member * g.strideA + (long long)m * g.lda;
+  const int m0 = (blockIdx.x * 8 + (threadIdx.x >> 5)) * RPW;
+  if (m0 >= g.M) return;
+  const bf16* __restrict__ A = reinterpret_cast<const bf16*>(g.A) + member * g.strideA;
   const bf16* __restrict__ B = reinterpret_cast<const bf16*>(g.B) + member * g.strideB;
-  float acc[NT];
+  float acc[RPW][NT];
 #pragma unroll
-  for (int n = 0; n < NT; ++n) acc[n] = 0.f;
+  for (int r = 0; r < RPW; ++r)
+#pragma unroll
+    for (int n = 0; n < NT; ++n) acc[r][n] = 0.f;
 #pragma unroll 2
   for (int k = lane * 8; k < g.K; k += 256) {
-    float a[8];
-    unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(A + k)), a);
+    float a[RPW][8];
+#pragma unroll
+    for (int r = 0; r < RPW; ++r) {
+      const int m = m0 + r < g.M ? m0 + r : g.M - 1;      // rows past the end repeat the last row and are not stored
+      unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(A + (long long)m * g.lda + k)), a[r]);
+    }
     const bf16* bk = B + k;
 #pragma unroll
     for (int n = 0; n < NT; ++n) {
       float b[8];
       unpack_bf16x8(__ldg(reinterpret_cast<const uint4*>(bk + (long long)n * g.ldb)), b);
 #pragma unroll
-      for (int j = 0; j < 8; ++j) acc[n] = fmaf(a[j], b[j], acc[n]);
+      for (int r = 0; r < RPW; ++r)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[r][n] = fmaf(a[r][j], b[j], acc[r][n]);
     }
   }
 #pragma unroll
-  for (int n = 0; n < NT; ++n) {
-    float v = acc[n];
+  for (int r = 0; r < RPW; ++r) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    if (lane == n) store_one(g, member, m, n, epilogue_one(g, member, m, n, v, 1));
+    for (int n = 0; n < NT; ++n) {
+      float v = acc[r][n];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == n && m0 + r < g.M) store_one(g, member, m0 + r, n, epilogue_one(g, member, m0 + r, n, v, 1));
+    }
   }
 }
 
@@ -214,7 +227,11 @@ static bool rowdot_vec_ok(const GemmArgs& g) {
 // one instantiation per width: no predicated-off columns in the inner loop
 template <int NT>
 static void launch_rowdot_vec_n(const GemmArgs& g, cudaStream_t s) {
-  launch_with(dim3((g.M + 7) / 8, g.batch), 256, 0, s)(k_gemm_rowdot_bf16x8<NT>, g);
+  constexpr int RPW = NT <= 4 ? 4 : 2;
+  if (g.M >= 8 * RPW)
+    launch_with(dim3((g.M + 8 * RPW - 1) / (8 * RPW), g.batch), 256, 0, s)(k_gemm_rowdot_bf16x8<NT, RPW>, g);
+  else
+    launch_with(dim3((g.M + 7) / 8, g.batch), 256, 0, s)(k_gemm_rowdot_bf16x8<NT, 1>, g);
 }
 static void launch_rowdot_vec(const GemmArgs& g, cudaStream_t s) {
   switch (g.N) {
@@ -451,12 +468,14 @@ __global__ void __launch_bounds__(256) k_gemm_smallk_bf16x8(GemmArgs g) {
   }
 }
 
-// The same product for K <= 4 (a critic's two-wide input layer, the data gradient of its one-wide output layer) with
+// The same product for K <= 10 (a critic's two-wide input layer, the data gradient of a one-, two- or ten-wide
+// output layer) with
 // the roles turned around: a thread keeps the weights and the bias of ITS 8 columns in registers and walks down the
 // rows, so that per output vector there is one small broadcast load of the row's K inputs, K x 8 multiply-adds,
 // the mask load and one 16-byte store, with four rows in flight.  A block covers all columns (up to 2048) and
 // kRowsPerLane rows per row lane.  Same multiply-add order per element as the kernels above.
 constexpr int kRowsPerLane = 16;
+constexpr int kTinyK = 10;   // K up to which a thread keeps its 8 columns' weights in registers
 template <bool B_MN, int KK>
 __global__ void __launch_bounds__(256) k_gemm_tinyk_bf16x8(GemmArgs g) {
   pdl_prologue();
@@ -529,7 +548,13 @@ static void launch_tinyk(const GemmArgs& g, cudaStream_t s) {
     case 1: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 1>, g); break;
     case 2: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 2>, g); break;
     case 3: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 3>, g); break;
-    default: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 4>, g); break;
+    case 4: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 4>, g); break;
+    case 5: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 5>, g); break;
+    case 6: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 6>, g); break;
+    case 7: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 7>, g); break;
+    case 8: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 8>, g); break;
+    case 9: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 9>, g); break;
+    default: launch_with(grid, 256, 0, s)(k_gemm_tinyk_bf16x8<B_MN, 10>, g); break;
   }
 }
 
@@ -564,7 +589,7 @@ static void launch_colacc(const GemmArgs& g, cudaStream_t s) {
 
 template <typename T>
 static bool launch_skinny(const GemmArgs& g, cudaStream_t s) {
-  if (smallk_vec_ok(g) && g.K <= 4 && !g.a_mn && g.N >= 8 &&
+  if (smallk_vec_ok(g) && g.K <= kTinyK && !g.a_mn && g.N >= 8 &&
       (long long)((g.M + kRowsPerLane - 1) / kRowsPerLane) <= 65535) {
     if (g.b_mn) launch_tinyk<true>(g, s);
     else launch_tinyk<false>(g, s);
