@@ -30,7 +30,7 @@ def _tiny_cfg(n, dtype=C.FP32, **kw):
 def _inject_histories(gpu, cpu, rng, n, rnd):
     """Random histories: member means spread so that some pairs differ significantly and some do not."""
     for m in range(n):
-        cnt = int(rng.integers(0, 11)) if rnd == 1 else 10          # round 1: ragged counts incl. 0 and 1
+        cnt = int(rng.integers(0, 11)) if rnd == 1 else 10          # second ready point: ragged counts incl. 0 and 1
         mu, sd = rng.normal(0.0, 0.5), abs(rng.normal(0.3, 0.2)) + 1e-3
         vals = rng.normal(mu, sd, cnt).astype(np.float32)
         if rnd == 2 and m % 7 == 3 and cnt:
