@@ -252,6 +252,16 @@ bool gemm_tc_pair_supported(const GemmArgs& g) {
   return gemm_tc_supported(g) && g.M >= 256 && g.N >= 256;
 }
 
+// Whether the pair kernel is the faster of the two tensor-core kernels for this problem.  Few tiles AND a short
+// contraction (under four waves of pairs, under 12 k-blocks): the single-CTA kernel's shorter pipeline fills and
+// drains faster (24 GAN pairs, 1024 x 512 x 512 per member: 23 -> 20 us per launch); longer contractions amortise the
+// pair's set-up even on two waves (32 members of 256 x 1024 x 1024).
+bool gemm_tc_pair_preferred(const GemmArgs& g) {
+  if (!gemm_tc_pair_supported(g)) return false;
+  const long long tiles = (long long)((g.M + 255) / 256) * ((g.N + 255) / 256) * g.batch;
+  return tiles >= 296 || g.K >= 768;
+}
+
 cudaError_t launch_gemm_tc_pair(const GemmArgs& g, Counters* counters, cudaStream_t s) {
   if (g.adam) return cudaErrorInvalidValue;
   TcParams p;

@@ -426,7 +426,7 @@ struct LaunchScope {
 int gemm(pbt_handle* h, const GemmArgs& g) {
   if (g.adam) {
     LAUNCH(h, kFused, launch_wgrad_adam(g, h->counters, h->stream));
-  } else if (gemm_tc_pair_supported(g)) {
+  } else if (gemm_tc_pair_preferred(g)) {
     LAUNCH(h, kGemm, launch_gemm_tc_pair(g, h->counters, h->stream));
   } else if (gemm_tc_supported(g)) {
     LAUNCH(h, kGemm, launch_gemm_tc(g, h->counters, h->stream));
@@ -1578,7 +1578,7 @@ int pbt_grouped_gemm(const pbt_gemm_desc* d, void* stream) {
   g.mask = d->mask; g.ldmask = d->ldmask; g.strideMask = d->strideMask;
   const bool tc = gemm_tc_supported(g), pair = gemm_tc_pair_supported(g);
   cudaError_t e;
-  if (d->engine == 3 || (d->engine == 0 && pair && d->status_device)) {
+  if (d->engine == 3 || (d->engine == 0 && pair && gemm_tc_pair_preferred(g) && d->status_device)) {
     if (!pair) return fail(nullptr, PBT_ERR_UNSUPPORTED, "shape / alignment does not qualify for the CTA-pair tensor-core kernel");
     if (!d->status_device) return fail(nullptr, PBT_ERR_INVALID_ARG, "status_device is required by the tensor-core kernels");
     e = launch_gemm_tc_pair(g, (Counters*)d->status_device, (cudaStream_t)stream);

@@ -146,6 +146,7 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s
 cudaError_t launch_selftest_bounded_wait(Counters* counters, uint32_t limit, cudaStream_t s);
 // CTA-pair variant (256 x 256 tiles shared by two CTAs of a cluster) for shapes with M, N >= 256
 bool gemm_tc_pair_supported(const GemmArgs& g);
+bool gemm_tc_pair_preferred(const GemmArgs& g);   // the faster of the two tensor-core kernels for this problem?
 cudaError_t launch_gemm_tc_pair(const GemmArgs& g, Counters* counters, cudaStream_t s);
 // weight gradient with the Adam update applied in the same kernel (g.adam must be set; tensor-core shapes only)
 cudaError_t launch_wgrad_adam(const GemmArgs& g, Counters* counters, cudaStream_t s);
