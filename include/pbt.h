@@ -302,12 +302,21 @@ int pbt_exploit_explore_ready(pbt_t* p, const uint8_t* ready_host);
  * carried out, the local ones by pbt_copy_members_level(p, L), the ones that cross shards by sending the donor's
  * slabs (pbt_member_slabs) into the recipient's slabs on the other device (peer copy or send / receive; the data
  * lands in the recipient's own memory before any kernel reads it).  Within a pass no recipient is anybody's donor.
- * Truncation selection and the binary tournament; PBT_ERR_UNSUPPORTED for t-test selection (the score histories are
- * not exchanged).  Synchronises the stream (it returns data to the host).
+ * All three exploit rules; for t-test selection the whole population's score histories have to be given first
+ * (pbt_set_global_history, else PBT_ERR_STATE), and the rows of this shard's members, with the histories that
+ * moved with a copy, are written back into the shard's own history.  Synchronises the stream (it returns data to
+ * the host).
  */
 int pbt_exploit_explore_global(pbt_t* p, double* fitness_global_host, double* hparams_global_host,
                                const uint8_t* ready_global_host, int32_t* src_global_out_host,
                                int32_t* level_global_out_host, int32_t* n_levels_out_host);
+
+/*
+ * T-test selection on a sharded population: the score histories of ALL members (each shard's pbt_get_history,
+ * all-gathered), hist [n_global][PBT_HISTORY] doubles oldest first, count [n_global] int32; consumed by the next
+ * pbt_exploit_explore_global.  Both host.
+ */
+int pbt_set_global_history(pbt_t* p, const double* hist_global_host, const int32_t* count_global_host);
 
 /* The local slab copies of one pass of the copy map left by pbt_exploit_explore_global.  Only enqueues. */
 int pbt_copy_members_level(pbt_t* p, int level);

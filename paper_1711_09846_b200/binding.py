@@ -77,7 +77,8 @@ class PbtGemmDesc(C.Structure):
 
 EXPORTS = [
     "pbt_query_workspace", "pbt_param_count", "pbt_create", "pbt_destroy", "pbt_step", "pbt_step_subset", "pbt_eval",
-    "pbt_exploit_explore", "pbt_exploit_explore_ready", "pbt_exploit_explore_global", "pbt_copy_members_level",
+    "pbt_exploit_explore", "pbt_exploit_explore_ready", "pbt_exploit_explore_global", "pbt_set_global_history",
+    "pbt_copy_members_level",
     "pbt_member_slabs", "pbt_get_state", "pbt_set_state", "pbt_get_fitness", "pbt_set_fitness",
     "pbt_get_history", "pbt_set_history",
     "pbt_get_hparams", "pbt_set_hparams", "pbt_get_copy_map", "pbt_get_best", "pbt_get_last_loss",
@@ -115,6 +116,7 @@ def load_library() -> C.CDLL:
     lib.pbt_exploit_explore_ready.argtypes = [vp, C.POINTER(C.c_uint8)]
     lib.pbt_exploit_explore_global.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_uint8),
                                                C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.pbt_set_global_history.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int32)]
     lib.pbt_copy_members_level.argtypes = [vp, C.c_int]
     lib.pbt_member_slabs.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(C.c_size_t), C.POINTER(C.c_int32)]
     lib.pbt_get_state.argtypes = [vp, C.c_int, C.POINTER(PbtStateView)]
@@ -413,6 +415,14 @@ class Population:
             mask.ctypes.data_as(C.POINTER(C.c_uint8)) if mask is not None else None,
             src.ctypes.data_as(C.POINTER(C.c_int32)), level.ctypes.data_as(C.POINTER(C.c_int32)), C.byref(n_levels)))
         return src, level, n_levels.value, f, h
+
+    def set_global_history(self, hist_global, count_global):
+        """The whole population's score histories for the next exploit_explore_global (t-test selection)."""
+        h = np.ascontiguousarray(hist_global, dtype=np.float64)
+        c = np.ascontiguousarray(count_global, dtype=np.int32)
+        assert h.shape == (self.n_global, PBT_HISTORY) and c.shape == (self.n_global,)
+        self._check(self.lib.pbt_set_global_history(self.handle, h.ctypes.data_as(C.POINTER(C.c_double)),
+                                                    c.ctypes.data_as(C.POINTER(C.c_int32))))
 
     def copy_members_level(self, level: int):
         self._check(self.lib.pbt_copy_members_level(self.handle, int(level)))

@@ -65,6 +65,7 @@ struct pbt_handle {
   long long* tm;     // [N] every member's own step count (Algorithm 1's t)
   // sharded populations: the whole population's selection inputs and outputs (n_global entries each)
   void* g_fit; void* g_H; int* g_src; int* g_level;
+  void* g_hist; int* g_hist_n; bool g_hist_set;   // t-test selection: the whole population's score histories
   int member_base;   // population index of the first member the pointers below refer to (0 unless a window is open)
   float* last_loss;  // [N][2]
   double* theta;     // toy: [N][nh]
@@ -226,12 +227,15 @@ size_t plan(pbt_handle* h, char* base) {
   h->tm = (long long*)take(N * sizeof(long long));
   h->member_base = s.member_base;
   h->g_fit = h->g_H = nullptr; h->g_src = h->g_level = nullptr;
+  h->g_hist = nullptr; h->g_hist_n = nullptr;
   if (s.n_global > 0) {
     const size_t G = s.n_global;
     h->g_fit = take(G * sizeof(double));
     h->g_H = take(G * PBT_MAX_NH * sizeof(double));
     h->g_src = (int*)take(G * sizeof(int));
     h->g_level = (int*)take(G * sizeof(int));
+    h->g_hist = take(G * PBT_HISTORY * sizeof(double));
+    h->g_hist_n = (int*)take(G * sizeof(int));
   }
   h->src = (int*)take(N * sizeof(int));
   h->level = (int*)take(N * sizeof(int));
@@ -1150,7 +1154,8 @@ int pbt_exploit_explore_global(pbt_t* p, double* fit_g, double* H_g, const uint8
   if (!p || !fit_g || !H_g || !src_out || !level_out || !n_levels_out) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
   const pbt_spec& s = p->spec;
   if (s.n_global <= 0) return fail(p, PBT_ERR_STATE, "the handle was not created as a shard (n_global = 0)");
-  if (s.exploit_rule == 2) return fail(p, PBT_ERR_UNSUPPORTED, "t-test selection is not available for sharded populations");
+  if (s.exploit_rule == 2 && !p->g_hist_set)
+    return fail(p, PBT_ERR_STATE, "t-test selection needs the whole population's score histories: call pbt_set_global_history first");
   set_serial_launches(s.programmatic_launches == 0);
   p->launches = 0;
   const int G = s.n_global;
@@ -1174,9 +1179,18 @@ int pbt_exploit_explore_global(pbt_t* p, double* fit_g, double* H_g, const uint8
   SelectArgs a;
   int n_cut = 0;
   fill_select_args(p, &a, G, ready_g, p->g_H, p->g_fit, p->g_src, p->g_level, &n_cut);
+  if (s.exploit_rule == 2) { a.hist = p->g_hist; a.hist_n = p->g_hist_n; }
   LAUNCH(p, kSelect, launch_select_explore(a, p->stream));
   LAUNCH(p, kSelect, launch_localize_selection(p->g_src, p->g_level, p->g_H, p->g_fit, p->toy ? 1 : 0, s.member_base, p->N,
                                                p->src, p->level, p->H, p->fitness, p->stream));
+  if (s.exploit_rule == 2) {
+    // a copy moved the donor's score history with it (inside the global arrays): take this shard's rows back
+    const size_t esz = p->toy ? 8 : 4;
+    CU(p, cudaMemcpyAsync(p->hist, (const char*)p->g_hist + (size_t)s.member_base * PBT_HISTORY * esz,
+                          (size_t)p->N * PBT_HISTORY * esz, cudaMemcpyDeviceToDevice, p->stream));
+    CU(p, cudaMemcpyAsync(p->hist_n, p->g_hist_n + s.member_base, (size_t)p->N * 4, cudaMemcpyDeviceToDevice, p->stream));
+    p->g_hist_set = false;
+  }
   Counters cnt;
   CU(p, cudaMemcpyAsync(&cnt, p->counters, sizeof(cnt), cudaMemcpyDeviceToHost, p->stream));
   CU(p, cudaMemcpyAsync(src_out, p->g_src, (size_t)G * 4, cudaMemcpyDeviceToHost, p->stream));
@@ -1203,6 +1217,24 @@ int pbt_exploit_explore_global(pbt_t* p, double* fit_g, double* H_g, const uint8
     return PBT_OK;
   }
   *n_levels_out = (s.exploit_rule == 0 ? 0 : cnt.max_level) + 1;
+  return PBT_OK;
+}
+
+int pbt_set_global_history(pbt_t* p, const double* hist, const int32_t* count) {
+  if (!p || !hist || !count) return fail(p, PBT_ERR_INVALID_ARG, "NULL argument");
+  const pbt_spec& s = p->spec;
+  if (s.n_global <= 0) return fail(p, PBT_ERR_STATE, "the handle was not created as a shard (n_global = 0)");
+  const int G = s.n_global;
+  for (int m = 0; m < G; ++m)
+    if (count[m] < 0 || count[m] > PBT_HISTORY) return fail(p, PBT_ERR_INVALID_ARG, "history count out of range");
+  const size_t n = (size_t)G * PBT_HISTORY;
+  std::vector<float> hf(n);
+  for (size_t i = 0; i < n; ++i) hf[i] = (float)hist[i];
+  if (p->toy) CU(p, cudaMemcpyAsync(p->g_hist, hist, n * 8, cudaMemcpyHostToDevice, p->stream));
+  else CU(p, cudaMemcpyAsync(p->g_hist, hf.data(), n * 4, cudaMemcpyHostToDevice, p->stream));
+  CU(p, cudaMemcpyAsync(p->g_hist_n, count, (size_t)G * 4, cudaMemcpyHostToDevice, p->stream));
+  CU(p, cudaStreamSynchronize(p->stream));
+  p->g_hist_set = true;
   return PBT_OK;
 }
 

@@ -161,10 +161,13 @@ class ShardedPopulation:
     def slabs_of(self, member: int):
         return self.local.member_slabs(member - self.first)
 
-    def decide(self, fitness_all, hparams_all, ready=None) -> CopyPlan:
+    def decide(self, fitness_all, hparams_all, ready=None, history_all=None) -> CopyPlan:
         """Selection and explore for the whole population on this shard (every shard gets the same answer); the
-        rows of this shard's members are applied to its own records.  Returns the copy plan."""
+        rows of this shard's members are applied to its own records.  history_all = (scores [N][10], counts [N]) of
+        the whole population, needed by t-test selection.  Returns the copy plan."""
         n = self.cfg.n_members
+        if history_all is not None:
+            self.local.set_global_history(np.asarray(history_all[0]).reshape(n, -1), np.asarray(history_all[1]).reshape(n))
         src, level, n_levels, _, _ = self.local.exploit_explore_global(
             np.asarray(fitness_all, dtype=np.float64).reshape(n), np.asarray(hparams_all, dtype=np.float64).reshape(n, -1), ready)
         self.last_src = src
@@ -177,7 +180,12 @@ class ShardedPopulation:
         import torch
         f = self.transport.all_gather(self, torch.from_numpy(self.local.fitness()))
         h = self.transport.all_gather(self, torch.from_numpy(self.local.hparams()))
-        plan = self.decide(f.numpy(), h.numpy(), ready)
+        hist = None
+        if getattr(self.cfg, "exploit", "truncation") == "ttest":
+            hs, hc = self.local.history()
+            hist = (self.transport.all_gather(self, torch.from_numpy(hs)).numpy(),
+                    self.transport.all_gather(self, torch.from_numpy(hc)).numpy())
+        plan = self.decide(f.numpy(), h.numpy(), ready, hist)
         for lv in range(plan.n_levels):
             self.local.copy_members_level(lv)            # local copies of this pass (enqueued on the shard's stream)
             self.transport.exchange(self, plan, lv)      # records that cross shards land in the recipients' slabs
@@ -220,7 +228,11 @@ def ready_point_in_process(shards: Sequence[ShardedPopulation], ready=None) -> n
     import torch
     f = np.concatenate([s.local.fitness() for s in shards])
     h = np.concatenate([s.local.hparams() for s in shards], axis=0)
-    plans = [s.decide(f, h, ready) for s in shards]
+    hist = None
+    if getattr(shards[0].cfg, "exploit", "truncation") == "ttest":
+        parts = [s.local.history() for s in shards]
+        hist = (np.concatenate([p[0] for p in parts], axis=0), np.concatenate([p[1] for p in parts]))
+    plans = [s.decide(f, h, ready, hist) for s in shards]
     assert all(np.array_equal(s.last_src, shards[0].last_src) for s in shards), "the shards disagree on the copy map"
     n, world = shards[0].cfg.n_members, len(shards)
     for lv in range(max(p.n_levels for p in plans)):

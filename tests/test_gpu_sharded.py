@@ -23,7 +23,8 @@ def pkg():
 
 @pytest.mark.parametrize("name,n,world,rule", [("c2_mini", 10, 2, "truncation"), ("c3_mini", 11, 3, "truncation"),
                                                ("c3_mini", 12, 2, "tournament"), ("c5_mid", 6, 2, "truncation"),
-                                               ("c1", 9, 3, "tournament"), ("c4_mini_wgan", 7, 2, "truncation")])
+                                               ("c1", 9, 3, "tournament"), ("c4_mini_wgan", 7, 2, "truncation"),
+                                               ("c2_mini", 9, 2, "ttest"), ("c3_mini", 10, 3, "ttest")])
 def test_sharded_run_equals_the_unsharded_run_bit_for_bit(pkg, name, n, world, rule):
     from paper_1711_09846_b200 import sharding as S
     cfg = get_config(name).replace(n_members=n, exploit=rule, ready_interval=2, trunc_num=2, trunc_den=5)
@@ -36,7 +37,7 @@ def test_sharded_run_equals_the_unsharded_run_bit_for_bit(pkg, name, n, world, r
     whole = pkg.Population(cfg, inp)
     shards = [S.ShardedPopulation(pkg, cfg, inp, r, world, transport=object()) for r in range(world)]
     crossed = 0
-    for rnd in range(3):
+    for rnd in range(5 if rule == "ttest" else 3):
         whole.step(cfg.ready_interval)
         whole.eval()
         for s in shards:
@@ -50,6 +51,11 @@ def test_sharded_run_equals_the_unsharded_run_bit_for_bit(pkg, name, n, world, r
         crossed += shards[0].last_plan.crossing()
         assert np.array_equal(whole.hparams(), np.concatenate([s.local.hparams() for s in shards], axis=0))
         assert np.array_equal(whole.fitness(), np.concatenate([s.local.fitness() for s in shards]), equal_nan=True)
+        if rule == "ttest":
+            hw, cw = whole.history()
+            parts = [s.local.history() for s in shards]
+            assert np.array_equal(cw, np.concatenate([p[1] for p in parts]))
+            assert np.array_equal(hw, np.concatenate([p[0] for p in parts], axis=0))
         for m in range(n):
             r = S.owner_of(m, world, n)
             a, b = whole.get_state(m), shards[r].local.get_state(m - shards[r].first)
@@ -62,7 +68,7 @@ def test_sharded_run_equals_the_unsharded_run_bit_for_bit(pkg, name, n, world, r
         s.close()
 
 
-def test_a_shard_refuses_the_unsharded_ready_point_and_t_test_selection(pkg):
+def test_a_shard_refuses_the_unsharded_ready_point_and_t_test_selection_without_histories(pkg):
     from paper_1711_09846_b200 import sharding as S
     cfg = get_config("c2_mini").replace(n_members=6)
     inp = make_inputs(cfg)
@@ -72,7 +78,7 @@ def test_a_shard_refuses_the_unsharded_ready_point_and_t_test_selection(pkg):
     assert e.value.code == 6
     s.close()
     t = S.ShardedPopulation(pkg, cfg.replace(exploit="ttest"), inp, 1, 2, transport=object())
-    with pytest.raises(pkg.PbtError) as e:
+    with pytest.raises(pkg.PbtError) as e:                 # t-test selection wants the whole population's histories first
         t.decide(np.zeros(6), np.asarray(inp.init_hparams))
-    assert e.value.code == 2
+    assert e.value.code == 6
     t.close()
