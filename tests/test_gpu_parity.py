@@ -656,6 +656,45 @@ def test_prefetched_steps_after_pool_steps_match_the_oracle(pkg):
     gpu.close()
 
 
+def test_degenerate_populations_and_empty_calls(pkg):
+    """step(0) and an all-inactive subset step change nothing; a population of one steps like member 0 of a larger
+    one and its ready point is a no-op; a fitness vector of NaNs and one of equal values select by index alone."""
+    cfg = get_config("c3_mini")
+    inp = make_inputs(cfg)
+    gpu = pkg.Population(cfg, inp)
+    before = [gpu.get_state(m) for m in range(cfg.n_members)]
+    gpu.step(0)
+    gpu.step_subset(np.zeros(cfg.n_members, dtype=bool), 3)
+    for m in range(cfg.n_members):
+        now = gpu.get_state(m)
+        assert now["step"] == 0
+        for key in ("w", "opt1", "opt2", "scalars"):
+            assert np.array_equal(now[key], before[m][key])
+    cpu = O.Population(cfg, inp)
+    for f in (np.full(cfg.n_members, np.nan), np.full(cfg.n_members, 0.25)):
+        cpu.fitness[:] = f
+        gpu.set_fitness(f)
+        gpu.exploit_explore()
+        src = cpu.exploit_explore()
+        assert np.array_equal(gpu.copy_map(), src)
+        assert (src != np.arange(cfg.n_members)).sum() == O.n_cut_of(cfg.n_members, cfg.trunc_num, cfg.trunc_den)
+        assert np.array_equal(gpu.hparams(), cpu.H.astype(np.float64))
+    gpu.close()
+    one = cfg.replace(n_members=1)
+    inp1 = make_inputs(one)
+    solo, many = pkg.Population(one, inp1), pkg.Population(cfg, inp)
+    many.set_hparams(np.tile(np.asarray(inp1.init_hparams, dtype=np.float64), (cfg.n_members, 1)))
+    solo.step(2)
+    many.step(2)
+    for key in ("w", "opt1", "opt2"):
+        assert np.array_equal(solo.get_state(0)[key], many.get_state(0)[key])
+    solo.eval()
+    solo.exploit_explore()
+    assert list(solo.copy_map()) == [0] and solo.get_state(0)["round"] == 1
+    solo.close()
+    many.close()
+
+
 def test_invalid_arguments_are_reported_not_fatal(pkg):
     cfg = get_config("c2_mini")
     inp = make_inputs(cfg)
