@@ -8,8 +8,10 @@ of every case carries the stated bar (1e-5 in fp32, 2e-2 in bf16); later ones ca
 workload, a few times the observed drift: training with ReLU units and sign-like optimiser steps amplifies a
 rounding difference (a unit that is active on one side only, a near-zero gradient whose sign differs), and the
 oracle run against a copy of itself whose initial weights were moved by one fp32 ulp drifts apart at the same rate.
-What the ready point consumes, the fitness vector, is held to the per-step bar at every ready point, and the
-decisions taken on it are checked bit for bit against the oracle's selection and explore functions.
+What the ready point consumes, the fitness vector, is held to the per-step bar at every ready point of the fp32 and
+the large bf16 population (1e-3 / 2e-2), to 5e-2 for the 50-step intervals of the 32 classifiers and to 0.2 for the
+GAN pairs (the last column of CASES), and the decisions taken on the GPU's fitness vector are checked bit for bit
+against the oracle's selection and explore functions.
 
 Full-size cases run the whole population on the GPU and a sample of members on the oracle (members are independent
 between ready points); after the ready point every sampled member starts the next interval from identical state on
