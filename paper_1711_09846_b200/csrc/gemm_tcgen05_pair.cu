@@ -222,16 +222,15 @@ k_gemm_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!mbar_wait(&tfull[acc], (it >> 1) & 1, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kPN);
+      const uint32_t handback = map_to_cta(smem_u32(&tempty[acc]), 0);
       if (p.c_tma && m0 + kBM <= p.M && n0 + kPN <= p.N && (p.out_dtype == kBF16 || !p.mask)) {
-        epilogue_tile_tma<kPN, kPEpiW>(p, &tmC, stage, tacc, member, m0, n0, q, half, lane, boxes_used);
+        epilogue_tile_tma<kPN, kPEpiW>(p, &tmC, stage, tacc, member, m0, n0, q, half, lane, handback, boxes_used);
       } else {
         if (lane == 0) tma_store_wait_all();   // the transposing path reuses the staging memory
         __syncwarp();
         epilogue_tile<kPN, kPEpiW>(p, buf, tacc, member, m0, n0, q, half, lane, vec_ok);
+        release_accumulator(handback, lane);
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty[acc]), 0));
     }
     if (lane == 0) tma_store_wait_all();     // the bulk stores have read the staging boxes and reached memory
     if (!ok && lane == 0) {
