@@ -373,6 +373,7 @@ def main():
     ap.add_argument("--no-workloads", action="store_true", help="skip the compact figures of the other benchmark populations")
     ap.add_argument("--fuse-adam", type=int, default=-1, help="1/0: apply Adam inside the weight-gradient GEMM (default: the library's choice)")
     ap.add_argument("--graph", type=int, default=-1, help="1: time CUDA-graph replays and profile in a second pass; 0: profile the timed region; -1: by step length")
+    ap.add_argument("--backward-streams", type=int, default=0, help="0: the library's choice; 1: one stream; 2: weight and bias gradients beside the data gradient on a second stream")
     ap.add_argument("--members", type=int, default=0, help="override the population size (profiling a small case)")
     ap.add_argument("--pool-rows", type=int, default=0, help="override the training-pool size (default: the workload's)")
     args = ap.parse_args()
@@ -407,6 +408,7 @@ def main():
     import paper_1711_09846_b200 as pkg
     inp = make_inputs(cfg)
     kw = {} if args.fuse_adam < 0 else {"fuse_adam": bool(args.fuse_adam)}
+    kw["backward_streams"] = args.backward_streams
     pop = pkg.Population(cfg, inp, device=f"cuda:{local}", **kw)
     interval = cfg.ready_interval
 

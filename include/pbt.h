@@ -138,6 +138,15 @@ typedef struct pbt_spec {
                         until the predecessor's results are visible (same dependences, bit-identical results).  On a
                         B200 this was not faster than replaying the captured step in stream order.  The setting of
                         the handle used last applies to the process. */
+  int32_t backward_streams; /* Back-propagation of one layer is three independent launches that all read the layer's
+                        delta: the data gradient (which the next layer waits for), the weight gradient and the bias
+                        gradient.  0 (default) or 2: the bias gradient, and the weight gradient unless its Adam update
+                        is fused into it (that launch must follow the data gradient, which reads the old weights),
+                        are enqueued on a second stream owned by the handle, forked from and joined to the handle's
+                        stream inside each layer, so they run beside the data gradient; the replayed step graph
+                        captures them as parallel branches.  1: everything in the handle's stream.  Same kernels on
+                        the same inputs either way: results are bit-identical.  On the legacy default stream (NULL)
+                        the setting is ignored and one stream is used. */
   int32_t member_base;  /* this handle holds members [member_base, member_base + n_members) of a larger population that
                            is sharded over several handles (one per GPU).  Everything that is drawn per member (initial
                            weights, training rows, interpolation coefficients, donors, explore draws) is keyed by the

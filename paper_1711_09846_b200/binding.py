@@ -38,7 +38,7 @@ class PbtSpec(C.Structure):
         ("slot_lr", C.c_int32), ("slot_lr_d", C.c_int32), ("slot_momentum", C.c_int32),
         ("slot_beta1", C.c_int32), ("slot_wd", C.c_int32),
         ("perturb_mask", C.c_uint32), ("flags", C.c_uint32),
-        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("programmatic_launches", C.c_int32), ("member_base", C.c_int32), ("n_global", C.c_int32), ("exploit_rule", C.c_int32),
+        ("trunc_num", C.c_int32), ("trunc_den", C.c_int32), ("keep_grad", C.c_int32), ("fuse_adam", C.c_int32), ("programmatic_launches", C.c_int32), ("backward_streams", C.c_int32), ("member_base", C.c_int32), ("n_global", C.c_int32), ("exploit_rule", C.c_int32),
         ("explore_rule", C.c_int32), ("prior_kind", C.c_int32 * PBT_MAX_NH),
         ("const_lr", C.c_double), ("const_momentum", C.c_double), ("const_beta1", C.c_double),
         ("const_beta2", C.c_double), ("const_eps", C.c_double), ("const_wd", C.c_double),
@@ -154,7 +154,8 @@ class PbtError(RuntimeError):
         self.code = code
 
 
-def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True, programmatic_launches: bool = False) -> PbtSpec:
+def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True, programmatic_launches: bool = False,
+                     backward_streams: int = 0) -> PbtSpec:
     """Translate a declarative population description (see workloads.configs.PBTConfig) into pbt_spec."""
     s = PbtSpec()
     s.n_members = cfg.n_members
@@ -183,6 +184,7 @@ def spec_from_config(cfg, keep_grad: bool = False, fuse_adam: bool = True, progr
     s.trunc_num, s.trunc_den = cfg.trunc_num, cfg.trunc_den
     s.keep_grad = 1 if keep_grad else 0
     s.programmatic_launches = 1 if programmatic_launches else 0
+    s.backward_streams = int(backward_streams)
     s.exploit_rule = {"truncation": 0, "tournament": 1, "ttest": 2}[getattr(cfg, "exploit", "truncation")]
     s.explore_rule = {"perturb": 0, "resample": 1}[getattr(cfg, "explore", "perturb")]
     s.ttest_alpha = getattr(cfg, "ttest_alpha", 0.05)
@@ -276,7 +278,7 @@ class Population:
 
     def __init__(self, cfg, inputs, seed: Optional[int] = None, device: str = "cuda:0", keep_grad: bool = False,
                  fuse_adam: bool = True, guard_bytes: int = 0, programmatic_launches: bool = False,
-                 member_base: int = 0, n_global: int = 0):
+                 member_base: int = 0, n_global: int = 0, backward_streams: int = 0):
         """cfg.n_members members on `device`.  member_base / n_global: this population is the shard
         [member_base, member_base + cfg.n_members) of a population of n_global members (see sharding.py);
         inputs.init_hparams then holds the rows of the whole population."""
@@ -288,7 +290,7 @@ class Population:
         self.cfg = cfg
         self.device = torch.device(device)
         self.seed = int(cfg.seed if seed is None else seed)
-        self.spec = spec_from_config(cfg, keep_grad, fuse_adam, programmatic_launches)
+        self.spec = spec_from_config(cfg, keep_grad, fuse_adam, programmatic_launches, backward_streams)
         self.member_base, self.n_global = int(member_base), int(n_global)
         self.spec.member_base, self.spec.n_global = self.member_base, self.n_global
         self.N, self.nh = cfg.n_members, cfg.nh

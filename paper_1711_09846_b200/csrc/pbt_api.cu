@@ -43,6 +43,10 @@ struct pbt_handle {
   pbt_spec spec;
   pbt_data data;
   cudaStream_t stream;
+  // Launches go to `ls`: the handle's stream, except while a backward pass has forked work to `side` (a second
+  // stream the handle owns; every fork is joined back before the pass returns).  side == nullptr: never fork.
+  cudaStream_t ls, side;
+  cudaEvent_t ev_fork, ev_join;
   uint64_t seed;
   int N, ns, nh;
   bool toy, gan, is_bf16;
@@ -165,6 +169,8 @@ int validate(const pbt_spec* s) {
   const int slots[5] = {s->slot_lr, s->slot_lr_d, s->slot_momentum, s->slot_beta1, s->slot_wd};
   for (int i = 0; i < 5; ++i)
     if (slots[i] < -1 || slots[i] >= s->nh) return fail(nullptr, PBT_ERR_INVALID_ARG, "hyperparameter slot out of range");
+  if (s->backward_streams < 0 || s->backward_streams > 2)
+    return fail(nullptr, PBT_ERR_INVALID_ARG, "backward_streams must be 0 (automatic), 1 or 2");
   if (s->member_base < 0 || s->n_global < 0 || s->n_global > 1024 ||
       (s->n_global == 0 && s->member_base != 0) || (s->n_global > 0 && s->member_base + s->n_members > s->n_global))
     return fail(nullptr, PBT_ERR_INVALID_ARG, "member_base / n_global do not describe a shard of a population of at most 1024 members");
@@ -406,12 +412,12 @@ struct LaunchScope {
     if (h->profiling) {
       a = get_event(h);
       b = get_event(h);
-      cudaEventRecord(a, h->stream);
+      cudaEventRecord(a, h->ls);
     }
   }
   ~LaunchScope() {
     if (h->profiling) {
-      cudaEventRecord(b, h->stream);
+      cudaEventRecord(b, h->ls);
       h->prof.push_back(ProfRec{cls, a, b});
     }
   }
@@ -429,17 +435,37 @@ struct LaunchScope {
 
 int gemm(pbt_handle* h, const GemmArgs& g) {
   if (g.adam) {
-    LAUNCH(h, kFused, launch_wgrad_adam(g, h->counters, h->stream));
+    LAUNCH(h, kFused, launch_wgrad_adam(g, h->counters, h->ls));
   } else if (gemm_tc_pair_preferred(g)) {
-    LAUNCH(h, kGemm, launch_gemm_tc_pair(g, h->counters, h->stream));
+    LAUNCH(h, kGemm, launch_gemm_tc_pair(g, h->counters, h->ls));
   } else if (gemm_tc_supported(g)) {
-    LAUNCH(h, kGemm, launch_gemm_tc(g, h->counters, h->stream));
+    LAUNCH(h, kGemm, launch_gemm_tc(g, h->counters, h->ls));
   } else {
     if (g.a_rowoff || g.b_rowoff) return fail(h, PBT_ERR_UNSUPPORTED, "row-window operands need a tensor-core shape");
-    LAUNCH(h, kGemm, launch_gemm_simt(g, h->stream));
+    LAUNCH(h, kGemm, launch_gemm_simt(g, h->ls));
   }
   return PBT_OK;
 }
+
+// Work enqueued between fork_side() and the matching join_side() may be sent to the side stream by wrapping it in
+// a SideScope: it then depends on everything in the handle's stream up to the fork, and everything enqueued in
+// the handle's stream after the join depends on it.  In a stream capture the two become parallel branches of the
+// graph.  The side stream is in order, so the work of successive forks never overlaps itself.
+bool fork_side(pbt_handle* h) {
+  if (!h->side) return false;
+  cudaEventRecord(h->ev_fork, h->stream);
+  cudaStreamWaitEvent(h->side, h->ev_fork, 0);
+  return true;
+}
+void join_side(pbt_handle* h) {
+  cudaEventRecord(h->ev_join, h->side);
+  cudaStreamWaitEvent(h->stream, h->ev_join, 0);
+}
+struct SideScope {
+  pbt_handle* h;
+  SideScope(pbt_handle* h_, bool on) : h(h_) { if (on) h->ls = h->side; }
+  ~SideScope() { h->ls = h->stream; }
+};
 
 const void* weights(const pbt_handle* h, long long off) {
   return h->is_bf16 ? (const void*)(h->W16 + off) : (const void*)(h->W32 + off);
@@ -507,7 +533,10 @@ int dgrad(pbt_handle* h, int k, int l, int rows, const void* dz, long long dz_st
 // (the caller must have finished every read of the layer's old weights); fused[l] records it.
 int wgrad_layer(pbt_handle* h, int k, int l, int rows, int bias_rows, const void* dz, long long dz_stride,
                 const void* in, long long in_stride, const OptArgs& opt, bool* fused, const int* in_rowoff = nullptr,
-                long long in_rows_total = 0) {
+                long long in_rows_total = 0, bool forked = false, bool gemm_on_side = true) {
+  // forked: the caller has forked the side stream where dz was complete; the bias gradient goes there, and so
+  // does an unfused weight gradient if gemm_on_side (a fused one stays in the handle's stream, behind the data
+  // gradient that reads the old weights)
   const pbt_spec& s = h->spec;
   const Layer& L = h->st[k].L[l];
   GemmArgs g;
@@ -525,9 +554,14 @@ int wgrad_layer(pbt_handle* h, int k, int l, int rows, int bias_rows, const void
     if (!s.keep_grad) g.C = nullptr;
     fused[l] = true;
   }
-  int rc = gemm(h, g);
+  int rc;
+  {
+    SideScope side(h, forked && gemm_on_side && !g.adam);
+    rc = gemm(h, g);
+  }
   if (rc) return rc;
-  LAUNCH(h, kLoss, launch_bias_grad(dz, h->cdt, L.out, dz_stride, bias_rows, L.out, h->G + L.b_off, h->P_pad, h->N, h->stream));
+  SideScope side(h, forked);
+  LAUNCH(h, kLoss, launch_bias_grad(dz, h->cdt, L.out, dz_stride, bias_rows, L.out, h->G + L.b_off, h->P_pad, h->N, h->ls));
   return PBT_OK;
 }
 
@@ -582,6 +616,9 @@ int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride
   for (int l = st.nl - 1; l >= 0; --l) {
     const void* dz = h->dz[*cur];
     bool wrote_dgrad = false;
+    // dz is complete here: what else reads it may run beside the data gradient; it is joined before the next
+    // layer's data gradient overwrites dz
+    const bool forked = need_wgrad && fork_side(h);
     if (l > 0 || need_input_grad) {
       int rc = dgrad(h, k, l, rows, dz, dzs, h->dz[1 - *cur], dzs, h->cdt, l > 0 ? h->act[k][l] : nullptr,
                      l > 0 ? act_stride(h, k, l) : 0);
@@ -591,7 +628,8 @@ int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride
     if (need_wgrad) {
       int rc = wgrad_layer(h, k, l, rows, rows, dz, dzs, l == 0 ? in : h->act[k][l],
                            l == 0 ? in_stride : act_stride(h, k, l), opt, fused, l == 0 ? in_rowoff : nullptr,
-                           in_rows_total);
+                           in_rows_total, forked, wrote_dgrad);
+      if (forked) join_side(h);
       if (rc) return rc;
     }
     if (wrote_dgrad) *cur = 1 - *cur;
@@ -763,10 +801,15 @@ int step_wgan(pbt_handle* h) {
     OptArgs opt;
     fill_opt_args(h, &opt, s.slot_lr_d, 2);
     bool fused[PBT_MAX_LAYERS] = {false};
+    // every layer's deltas are complete: the weight and bias gradients of all layers are independent launches
+    const bool forked = fork_side(h);
     for (int l = D.nl - 1; l >= 0; --l) {
-      rc = wgrad_layer(h, 1, l, 3 * B, 2 * B, h->gp_dz[l], 3ll * B * D.L[l].out, h->act[1][l], act_stride(h, 1, l), opt, fused);
-      if (rc) return rc;
+      rc = wgrad_layer(h, 1, l, 3 * B, 2 * B, h->gp_dz[l], 3ll * B * D.L[l].out, h->act[1][l], act_stride(h, 1, l), opt, fused,
+                       nullptr, 0, forked, (l & 1) != 0);
+      if (rc) break;
     }
+    if (forked) join_side(h);
+    if (rc) return rc;
     rc = finish_optimizer(h, 1, fused, opt);
     if (rc) return rc;
   }
@@ -875,6 +918,8 @@ int pbt_create(pbt_t** out, const pbt_spec* spec, const double* init_hparams, ui
   h->spec = *spec;
   if (data) h->data = *data;
   h->stream = (cudaStream_t)stream;
+  h->ls = h->stream;
+  h->side = nullptr;
   h->seed = seed;
   h->step_graph = nullptr;
   const size_t need = plan(h, nullptr);
@@ -929,6 +974,13 @@ int pbt_create(pbt_t** out, const pbt_spec* spec, const double* init_hparams, ui
       }
     if (h->is_bf16) CREATE_CU(launch_f32_to_bf16(h->W32, h->W16, (long long)h->N * h->P_pad, h->stream));
   }
+  {
+    if (spec->backward_streams != 1 && h->stream != nullptr && !h->toy) {
+      CREATE_CU(cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking));
+      CREATE_CU(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
+      CREATE_CU(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
+    }
+  }
 #undef CREATE_CU
   h->err[0] = 0;
   h->host_loss.assign((size_t)h->N * 2, 0.f);
@@ -944,6 +996,12 @@ int pbt_destroy(pbt_t* p) {
     cudaEventDestroy(p->ev_copied);
     cudaEventDestroy(p->ev_release);
     cudaStreamDestroy(p->copy_stream);
+  }
+  if (p->side) {
+    cudaStreamSynchronize(p->side);
+    cudaEventDestroy(p->ev_fork);
+    cudaEventDestroy(p->ev_join);
+    cudaStreamDestroy(p->side);
   }
   for (auto& r : p->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
   for (auto e : p->event_pool) cudaEventDestroy(e);

@@ -450,6 +450,37 @@ def test_step_eval_exploit_parity(pkg, name):
     gpu.close()
 
 
+@pytest.mark.parametrize("name", ["c2_mini", "c2_mini_rms", "c3_mini", "c3_mid", "c5_mid", "c4_mini", "c4_mid", "c4_mini_wgan",
+                                  "c4_mid_wgan", "c4_mini_wgan_fp32"])
+@pytest.mark.parametrize("fuse", [True, False])
+def test_backward_on_two_streams_is_bit_identical(pkg, name, fuse):
+    """A layer's weight and bias gradients beside its data gradient on a second stream (captured into the replayed
+    step as parallel branches): the same kernels on the same inputs, so every tensor, the gradients included,
+    and the fitness must equal the single-stream run bit for bit; plain (not replayed) steps and own-pace steps of
+    a subset too."""
+    cfg = get_config(name)
+    inp = make_inputs(cfg)
+    pops = [pkg.Population(cfg, inp, keep_grad=True, fuse_adam=fuse, backward_streams=k) for k in (1, 2)]
+    active = np.zeros(cfg.n_members, dtype=np.uint8)
+    active[1:cfg.n_members - 1] = 1
+    for pop in pops:
+        pop.step(3)                          # replayed graph
+        pop.step_subset(active, 1)           # plain launches on a member window
+        pop.eval()
+        pop.exploit_explore()
+        pop.step(2)
+        pop.eval()
+    a, b = pops
+    assert np.array_equal(a.fitness(), b.fitness())
+    for m in range(cfg.n_members):
+        sa, sb = a.get_state(m), b.get_state(m)
+        assert sa["step"] == sb["step"]
+        for key in ("w", "opt1", "opt2", "scalars", "grad"):
+            assert np.array_equal(sa[key], sb[key]), (name, m, key)
+    for pop in pops:
+        pop.close()
+
+
 @pytest.mark.parametrize("name", ["c3_mid", "c5_mid", "c4_mid", "c5_mini", "c4_mid_wgan"])
 def test_fused_update_is_the_same_with_and_without_stored_gradients(pkg, name):
     """The benchmarked configuration never writes the weight gradient of tensor-core layers to HBM.
