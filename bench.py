@@ -533,7 +533,8 @@ def main():
                    "optimizer": cfg.optimizer, "ready_interval": interval, "parallelism": "replicas only" if world > 1 else "1 gpu",
                    "timed_region": f"{args.steps} lockstep steps + 1 ready point (pbt_eval, pbt_exploit_explore); "
                                    f"median of {args.repeats} repeats",
-                   "timing": "CUDA-graph replay; per-kernel times from an extra profiled pass" if two_pass else "per-launch events in the last repeat",
+                   "timing": ("CUDA-graph replay; per-kernel times from an extra profiled pass" if two_pass else "per-launch events in the last repeat")
+                             + "; profiled launches run one at a time, while unprofiled steps run bias gradients beside data gradients on a second stream, so class times can add up to slightly more than the step",
                    "l2": "inputs larger than L2: population state %.1f GB" % (pop.workspace_bytes / 1e9)},
         "repeats": args.repeats, "ms_per_step_spread": [x / args.steps for x in total_spread],
         "train_ms_per_step": train_ms, "train_ms_per_step_spread": train_spread, "ready_point_ms": ready_ms,

@@ -407,7 +407,9 @@ int pbt_get_launch_count(const pbt_t* p, int64_t* count);
  * since pbt_profile_begin: "gemm", "wgrad_adam" (weight gradient with the Adam update fused in),
  * "optimizer" (the separate update pass), "loss", "copy", "select", "other".
  * Profiling brackets each launch with events on the handle's stream and
- * therefore slows the step down; it is off unless begun.
+ * therefore slows the step down; it is off unless begun.  While it is on, steps are not replayed from the
+ * captured graph and the backward pass stays in one stream (pbt_spec.backward_streams), so that every launch is
+ * timed alone: the class times of a step can then add up to a little more than an unprofiled step takes.
  */
 int pbt_profile_begin(pbt_t* p);
 int pbt_profile_end(pbt_t* p);

@@ -247,7 +247,18 @@ cudaError_t launch_gemm_tc(const GemmArgs& g, Counters* counters, cudaStream_t s
   p.bias = g.bias; p.strideBias = g.strideBias; p.relu = g.relu;
   p.mask = reinterpret_cast<const bf16*>(g.mask); p.ldmask = g.ldmask; p.strideMask = g.strideMask;
   p.counters = counters;
-  const int BN = g.N >= 256 ? 256 : 128;
+  int BN = g.N >= 256 ? 256 : 128;
+  if (BN == 256) {
+    // Few tiles: 128-wide tiles when the 256-wide ones would leave most of the last wave idle (a wave of half tiles
+    // costs a little over half a wave of full ones).  512 x 512 x 512 for 24 members: 192 wide tiles are 2 waves on
+    // 148 SMs, 384 narrow ones 3 half-waves.
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long long wide = (long long)p.tiles_m * ((g.N + 255) / 256) * g.batch;
+    const long long narrow = (long long)p.tiles_m * ((g.N + 127) / 128) * g.batch;
+    if (1.15 * (double)((narrow + sms - 1) / sms) < 2.0 * (double)((wide + sms - 1) / sms)) BN = 128;
+  }
   CUtensorMap tmA, tmB;
   bool ok;
   // K-major operand: rows = M (or N), cols = K.  MN-major operand: rows = K, cols = M (or N), boxes of 64 x 64.

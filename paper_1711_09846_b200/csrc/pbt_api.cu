@@ -452,7 +452,7 @@ int gemm(pbt_handle* h, const GemmArgs& g) {
 // the handle's stream after the join depends on it.  In a stream capture the two become parallel branches of the
 // graph.  The side stream is in order, so the work of successive forks never overlaps itself.
 bool fork_side(pbt_handle* h) {
-  if (!h->side) return false;
+  if (!h->side || h->profiling) return false;   // per-launch timing wants every launch alone on the GPU
   cudaEventRecord(h->ev_fork, h->stream);
   cudaStreamWaitEvent(h->side, h->ev_fork, 0);
   return true;
@@ -533,7 +533,7 @@ int dgrad(pbt_handle* h, int k, int l, int rows, const void* dz, long long dz_st
 // (the caller must have finished every read of the layer's old weights); fused[l] records it.
 int wgrad_layer(pbt_handle* h, int k, int l, int rows, int bias_rows, const void* dz, long long dz_stride,
                 const void* in, long long in_stride, const OptArgs& opt, bool* fused, const int* in_rowoff = nullptr,
-                long long in_rows_total = 0, bool forked = false, bool gemm_on_side = true) {
+                long long in_rows_total = 0, bool forked = false, bool gemm_on_side = true, bool* bias_done = nullptr) {
   // forked: the caller has forked the side stream where dz was complete; the bias gradient goes there, and so
   // does an unfused weight gradient if gemm_on_side (a fused one stays in the handle's stream, behind the data
   // gradient that reads the old weights)
@@ -554,20 +554,30 @@ int wgrad_layer(pbt_handle* h, int k, int l, int rows, int bias_rows, const void
     if (!s.keep_grad) g.C = nullptr;
     fused[l] = true;
   }
-  int rc;
   {
     SideScope side(h, forked && gemm_on_side && !g.adam);
-    rc = gemm(h, g);
+    int rc = gemm(h, g);
+    if (rc) return rc;
   }
-  if (rc) return rc;
   SideScope side(h, forked);
   LAUNCH(h, kLoss, launch_bias_grad(dz, h->cdt, L.out, dz_stride, bias_rows, L.out, h->G + L.b_off, h->P_pad, h->N, h->ls));
+  if (forked && bias_done && g.adam) {
+    // the layer's weights are updated by the fused launch: its bias vector is the whole of what is left, nothing
+    // in the backward pass reads it, and its gradient is complete in this stream: update it here, off the
+    // critical path, instead of in a launch of its own after the pass
+    const Stack& st = h->st[k];
+    OptArgs a = opt;
+    a.begin = L.b_off;
+    a.count = (l + 1 < st.nl ? st.L[l + 1].w_off : st.begin + st.count) - L.b_off;
+    LAUNCH(h, kOpt, launch_adam(a, h->ls));
+    bias_done[l] = true;
+  }
   return PBT_OK;
 }
 
 // element-wise optimiser over what the fused epilogues did not cover (biases, skinny layers, SGD-momentum,
 // RMSProp); adjacent slab ranges are merged into one launch
-int finish_optimizer(pbt_handle* h, int k, const bool* fused, const OptArgs& opt) {
+int finish_optimizer(pbt_handle* h, int k, const bool* fused, const OptArgs& opt, const bool* bias_done = nullptr) {
   const pbt_spec& s = h->spec;
   const Stack& st = h->st[k];
   long long rb = -1, re = -1;
@@ -592,6 +602,11 @@ int finish_optimizer(pbt_handle* h, int k, const bool* fused, const OptArgs& opt
       int rc = flush();
       if (rc) return rc;
     }
+    if (bias_done && bias_done[l]) {
+      int rc = flush();
+      if (rc) return rc;
+      continue;
+    }
     if (rb < 0) rb = L.b_off;
     re = b_end;
   }
@@ -612,7 +627,7 @@ int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride
   const long long dzs = dz_stride(h);
   OptArgs opt;
   fill_opt_args(h, &opt, slot_lr, scalar_base);
-  bool fused[PBT_MAX_LAYERS] = {false};
+  bool fused[PBT_MAX_LAYERS] = {false}, bias_done[PBT_MAX_LAYERS] = {false};
   for (int l = st.nl - 1; l >= 0; --l) {
     const void* dz = h->dz[*cur];
     bool wrote_dgrad = false;
@@ -628,14 +643,14 @@ int backward(pbt_handle* h, int k, int rows, const void* in, long long in_stride
     if (need_wgrad) {
       int rc = wgrad_layer(h, k, l, rows, rows, dz, dzs, l == 0 ? in : h->act[k][l],
                            l == 0 ? in_stride : act_stride(h, k, l), opt, fused, l == 0 ? in_rowoff : nullptr,
-                           in_rows_total, forked, wrote_dgrad);
+                           in_rows_total, forked, wrote_dgrad, bias_done);
       if (forked) join_side(h);
       if (rc) return rc;
     }
     if (wrote_dgrad) *cur = 1 - *cur;
   }
   if (!need_wgrad) return PBT_OK;
-  return finish_optimizer(h, k, fused, opt);
+  return finish_optimizer(h, k, fused, opt, bias_done);
 }
 
 int loss_and_dz(pbt_handle* h, int k, int rows, int n_real, const void* target, long long target_stride,
@@ -800,17 +815,17 @@ int step_wgan(pbt_handle* h) {
     }
     OptArgs opt;
     fill_opt_args(h, &opt, s.slot_lr_d, 2);
-    bool fused[PBT_MAX_LAYERS] = {false};
+    bool fused[PBT_MAX_LAYERS] = {false}, bias_done[PBT_MAX_LAYERS] = {false};
     // every layer's deltas are complete: the weight and bias gradients of all layers are independent launches
     const bool forked = fork_side(h);
     for (int l = D.nl - 1; l >= 0; --l) {
       rc = wgrad_layer(h, 1, l, 3 * B, 2 * B, h->gp_dz[l], 3ll * B * D.L[l].out, h->act[1][l], act_stride(h, 1, l), opt, fused,
-                       nullptr, 0, forked, (l & 1) != 0);
+                       nullptr, 0, forked, (l & 1) != 0, bias_done);
       if (rc) break;
     }
     if (forked) join_side(h);
     if (rc) return rc;
-    rc = finish_optimizer(h, 1, fused, opt);
+    rc = finish_optimizer(h, 1, fused, opt, bias_done);
     if (rc) return rc;
   }
   // generator update
