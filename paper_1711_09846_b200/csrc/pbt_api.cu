@@ -47,6 +47,7 @@ struct pbt_handle {
   // stream the handle owns; every fork is joined back before the pass returns).  side == nullptr: never fork.
   cudaStream_t ls, side;
   cudaEvent_t ev_fork, ev_join;
+  bool side_pending;   // side-stream work not yet joined
   uint64_t seed;
   int N, ns, nh;
   bool toy, gan, is_bf16;
@@ -455,11 +456,13 @@ bool fork_side(pbt_handle* h) {
   if (!h->side || h->profiling) return false;   // per-launch timing wants every launch alone on the GPU
   cudaEventRecord(h->ev_fork, h->stream);
   cudaStreamWaitEvent(h->side, h->ev_fork, 0);
+  h->side_pending = true;
   return true;
 }
 void join_side(pbt_handle* h) {
   cudaEventRecord(h->ev_join, h->side);
   cudaStreamWaitEvent(h->stream, h->ev_join, 0);
+  h->side_pending = false;
 }
 struct SideScope {
   pbt_handle* h;
@@ -667,7 +670,11 @@ int loss_and_dz(pbt_handle* h, int k, int rows, int n_real, const void* target, 
   a.dz = want_dz ? h->dz[dz_buf] : nullptr; a.dz_dtype = h->cdt; a.ld_dz = a.cols; a.stride_dz = dz_stride(h);
   a.row_loss = h->row_loss;
   LAUNCH(h, kLoss, launch_loss_rows(a, h->stream));
-  LAUNCH(h, kLoss, launch_reduce_rows(h->row_loss, rows, h->N, scale, out, 0, out_stride, h->stream));
+  // With deltas wanted, a backward pass follows that waits for the deltas only: the reduction of the row losses to
+  // the member's loss runs beside it (joined with the pass's first join, at the latest when the step ends; the
+  // next writer of row_loss is a later loss kernel in the handle's stream, behind that join).
+  SideScope side(h, want_dz && fork_side(h));
+  LAUNCH(h, kLoss, launch_reduce_rows(h->row_loss, rows, h->N, scale, out, 0, out_stride, h->ls));
   return PBT_OK;
 }
 
@@ -697,9 +704,15 @@ int step_mlp(pbt_handle* h) {
                                         in * h->esz, s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, clock(h), h->stream));
   const size_t trb = target_row_bytes(h);
   const size_t tsz = s.loss == PBT_LOSS_CE_SOFT ? h->esz : 4;
-  LAUNCH(h, kCopy, launch_gather_window((char*)h->ybatch, h->ybatch_stride * tsz, 0, (const char*)h->data.y_pool, (int)trb,
-                                        s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, clock(h), h->stream));
+  // the targets are needed by the loss only: their gather runs beside the forward pass
+  const bool forked = fork_side(h);
+  {
+    SideScope side(h, forked);
+    LAUNCH(h, kCopy, launch_gather_window((char*)h->ybatch, h->ybatch_stride * tsz, 0, (const char*)h->data.y_pool, (int)trb,
+                                          s.batch, s.pool_rows, h->N, 0, 0, h->seed, h->counters, clock(h), h->ls));
+  }
   int rc = forward(h, 0, s.batch, h->act[0][0], act_stride(h, 0, 0));
+  if (forked) join_side(h);
   if (rc) return rc;
   rc = loss_and_dz(h, 0, s.batch, s.batch, h->ybatch, h->ybatch_stride, true, 0, 1.0f / s.batch, h->last_loss, 2);
   if (rc) return rc;
@@ -716,12 +729,17 @@ int step_gan(pbt_handle* h) {
   int rc;
   for (int j = 0; j <= s.gan_d_steps; ++j) {
     const bool d_phase = j < s.gan_d_steps;
-    if (d_phase)
+    // the real rows are needed by the discriminator only: their gather runs beside the generator's forward pass
+    const bool forked = d_phase && fork_side(h);
+    if (d_phase) {
+      SideScope side(h, forked);
       LAUNCH(h, kCopy, launch_gather_window((char*)h->act[1][0], d_in_stride * h->esz, 0, (const char*)h->data.x_pool,
-                                            xdim * h->esz, B, s.pool_rows, h->N, j, 0, h->seed, h->counters, clock(h), h->stream));
+                                            xdim * h->esz, B, s.pool_rows, h->N, j, 0, h->seed, h->counters, clock(h), h->ls));
+    }
     LAUNCH(h, kCopy, launch_gather_window((char*)h->act[0][0], act_stride(h, 0, 0) * h->esz, 0, (const char*)h->data.z_pool,
                                           zdim * h->esz, B, s.pool_rows, h->N, j, 1, h->seed, h->counters, clock(h), h->stream));
     rc = forward(h, 0, B, h->act[0][0], act_stride(h, 0, 0));
+    if (forked) join_side(h);
     if (rc) return rc;
     // generated samples become discriminator input rows (after the real rows in a discriminator update)
     char* fake_dst = (char*)h->act[1][0] + (d_phase ? (size_t)B * xdim * h->esz : 0);
@@ -859,6 +877,7 @@ int one_step(pbt_handle* h) {
     rc = step_mlp(h);
     if (rc) return rc;
   }
+  if (h->side_pending) join_side(h);
   LAUNCH(h, kOther, launch_advance_step(h->counters, h->tm, h->N, h->stream));
   h->supplied_next = false;
   return PBT_OK;
@@ -935,6 +954,7 @@ int pbt_create(pbt_t** out, const pbt_spec* spec, const double* init_hparams, ui
   h->stream = (cudaStream_t)stream;
   h->ls = h->stream;
   h->side = nullptr;
+  h->side_pending = false;
   h->seed = seed;
   h->step_graph = nullptr;
   const size_t need = plan(h, nullptr);
