@@ -100,7 +100,8 @@ def test_tensor_core_shared_operand(env):
                                    (70, 136, 2, 2), (33, 512, 1, 3), (64, 64, 4, 1), (40, 72, 3, 2), (1030, 512, 2, 2),
                                    (45, 264, 5, 2), (512, 10, 256, 2), (10, 1024, 256, 3), (256, 10, 1024, 2), (136, 1, 512, 2),
                                    (8, 264, 72, 2), (2, 512, 1024, 2), (264, 16, 200, 1), (40, 1024, 10, 2),
-                                   (100, 2304, 2, 1), (1024, 512, 1, 2), (300, 8, 4, 2)])
+                                   (100, 2304, 2, 1), (1024, 512, 1, 2), (300, 8, 4, 2),
+                                   (128, 512, 256, 3), (512, 256, 128, 2), (192, 128, 48, 2)])   # all tiles interior
 def test_alu_engine(env, dtype, a_mn, b_mn, shape):
     pkg, torch = env
     M, N, K, batch = shape
