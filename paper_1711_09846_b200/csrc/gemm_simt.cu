@@ -112,9 +112,9 @@ __global__ void __launch_bounds__(256) k_gemm_simt(GemmArgs g) {
   }
 }
 
-// The same tile, K order and multiply-add order (bit-identical results) for GEMMs whose tiles are all interior
-// (M, N multiples of 64, K of 16) with 4-element-aligned operands: every thread moves ONE 4-element vector of each
-// operand per K slice through pointers that advance by a constant, and writes its 4 x 4 outputs as four vectors.
+// The same K order and multiply-add order (bit-identical results) for GEMMs whose tiles are all interior
+// (M, N multiples of 64, K of 16) with 4-element-aligned operands: every thread moves one or two 4-element vectors
+// of each operand per K slice through pointers that advance by a constant, and writes its outputs as vectors.
 // In the general kernel above the per-element index arithmetic and bounds checks of the slice loads were 46 % of
 // the instructions issued, and issue was the limit (FMA pipe 43-46 % busy on the 128 x 512 x 512 layers of the
 // fp32 population).
@@ -130,34 +130,52 @@ __device__ __forceinline__ float4 ld4<bf16>(const bf16* p) {
   return make_float4(a.x, a.y, b.x, b.y);
 }
 
-template <typename T, bool A_MN, bool B_MN>
+template <typename T, bool A_MN, bool B_MN, int TMV>
 __global__ void __launch_bounds__(256) k_gemm_simt_interior(GemmArgs g) {
+  // TMV = 4: 64 x 64 tile, 4 x 4 outputs per thread.  TMV = 8: 128 x 64 tile, 8 x 4 outputs per thread (fewer
+  // shared-memory reads per multiply-add; for GEMMs with enough 128-row tiles to go round).
+  constexpr int BMV = 16 * TMV, AV = TMV / 4;   // tile rows; vectors of A a thread moves per K slice
   pdl_prologue();
-  __shared__ __align__(16) float As[2][BK][BM + 4];
+  __shared__ __align__(16) float As[2][BK][BMV + 4];
   __shared__ __align__(16) float Bs[2][BK][BN + 4];
   const int member = blockIdx.z;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int m0 = blockIdx.y * BMV, n0 = blockIdx.x * BN;
   const int tid = threadIdx.x;
-  const int tx = tid & 15, ty = tid >> 4;
-  // K-major operand: the slice is 64 rows x 16 k, a thread takes row tid / 4, k (tid % 4) * 4 .. + 3.
-  // MN-major operand: the slice is 16 k x 64 columns, a thread takes k tid / 16, columns (tid % 16) * 4 .. + 3.
+  // a warp covers 8 x 4 threads, so that its shared-memory reads per k are one 128-byte row segment of B and 64 (128)
+  // bytes of A: two (three) wavefronts
+  const int lane = tid & 31, warp = tid >> 5;
+  const int tx = (lane & 7) + 8 * (warp & 1), ty = (lane >> 3) + 4 * (warp >> 1);
+  // K-major operand: the slice is rows x 16 k, a thread takes row tid / 4 (+ 64), k (tid % 4) * 4 .. + 3.
+  // MN-major operand: the slice is 16 k x columns, a thread takes columns (tid % (columns / 4)) * 4 .. + 3 of
+  // k = tid / (columns / 4) (+ 8 when the slice has 128 columns).
+  constexpr int AVW = BMV / 4;   // vectors per k row of an MN-major A slice
   const T* pa = reinterpret_cast<const T*>(g.A) + member * g.strideA +
-                (A_MN ? (long long)(tid >> 4) * g.lda + m0 + (tid & 15) * 4 : (long long)(m0 + (tid >> 2)) * g.lda + (tid & 3) * 4);
+                (A_MN ? (long long)(tid / AVW) * g.lda + m0 + (tid % AVW) * 4 : (long long)(m0 + (tid >> 2)) * g.lda + (tid & 3) * 4);
   const T* pb = reinterpret_cast<const T*>(g.B) + member * g.strideB +
                 (B_MN ? (long long)(tid >> 4) * g.ldb + n0 + (tid & 15) * 4 : (long long)(n0 + (tid >> 2)) * g.ldb + (tid & 3) * 4);
   const long long step_a = A_MN ? (long long)BK * g.lda : BK, step_b = B_MN ? (long long)BK * g.ldb : BK;
-  float acc[TM][TN];
+  const long long second_a = A_MN ? (long long)(256 / AVW) * g.lda : 64ll * g.lda;   // the thread's second vector of A
+  float acc[TMV][TN];
 #pragma unroll
-  for (int i = 0; i < TM; ++i)
+  for (int i = 0; i < TMV; ++i)
 #pragma unroll
     for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
-  float4 ra, rb;
+  float4 ra[AV], rb;
+  auto load_slab = [&]() {
+#pragma unroll
+    for (int v = 0; v < AV; ++v) ra[v] = ld4<T>(pa + v * second_a);
+    rb = ld4<T>(pb);
+    pa += step_a; pb += step_b;
+  };
   auto store_slab = [&](int buf) {
-    if (A_MN) {
-      *reinterpret_cast<float4*>(&As[buf][tid >> 4][(tid & 15) * 4]) = ra;
-    } else {
-      const int kq = (tid & 3) * 4, mm = tid >> 2;
-      As[buf][kq][mm] = ra.x; As[buf][kq + 1][mm] = ra.y; As[buf][kq + 2][mm] = ra.z; As[buf][kq + 3][mm] = ra.w;
+#pragma unroll
+    for (int v = 0; v < AV; ++v) {
+      if (A_MN) {
+        *reinterpret_cast<float4*>(&As[buf][tid / AVW + v * (256 / AVW)][(tid % AVW) * 4]) = ra[v];
+      } else {
+        const int kq = (tid & 3) * 4, mm = (tid >> 2) + 64 * v;
+        As[buf][kq][mm] = ra[v].x; As[buf][kq + 1][mm] = ra[v].y; As[buf][kq + 2][mm] = ra[v].z; As[buf][kq + 3][mm] = ra[v].w;
+      }
     }
     if (B_MN) {
       *reinterpret_cast<float4*>(&Bs[buf][tid >> 4][(tid & 15) * 4]) = rb;
@@ -166,25 +184,25 @@ __global__ void __launch_bounds__(256) k_gemm_simt_interior(GemmArgs g) {
       Bs[buf][kq][nn] = rb.x; Bs[buf][kq + 1][nn] = rb.y; Bs[buf][kq + 2][nn] = rb.z; Bs[buf][kq + 3][nn] = rb.w;
     }
   };
-  ra = ld4<T>(pa); rb = ld4<T>(pb);
-  pa += step_a; pb += step_b;
+  load_slab();
   store_slab(0);
   __syncthreads();
   int buf = 0;
   for (int k0 = 0; k0 < g.K; k0 += BK, buf ^= 1) {
     const bool more = k0 + BK < g.K;
-    if (more) {
-      ra = ld4<T>(pa); rb = ld4<T>(pb);
-      pa += step_a; pb += step_b;
-    }
+    if (more) load_slab();
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
-      const float4 a4 = *reinterpret_cast<const float4*>(&As[buf][kk][ty * TM]);
+      float a[TMV];
+#pragma unroll
+      for (int v = 0; v < AV; ++v) {
+        const float4 a4 = *reinterpret_cast<const float4*>(&As[buf][kk][ty * TMV + 4 * v]);
+        a[4 * v] = a4.x; a[4 * v + 1] = a4.y; a[4 * v + 2] = a4.z; a[4 * v + 3] = a4.w;
+      }
       const float4 b4 = *reinterpret_cast<const float4*>(&Bs[buf][kk][tx * TN]);
-      const float a[TM] = {a4.x, a4.y, a4.z, a4.w};
       const float b[TN] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
-      for (int i = 0; i < TM; ++i)
+      for (int i = 0; i < TMV; ++i)
 #pragma unroll
         for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
     }
@@ -197,8 +215,8 @@ __global__ void __launch_bounds__(256) k_gemm_simt_interior(GemmArgs g) {
   if (g.bias) bv = __ldg(reinterpret_cast<const float4*>(g.bias + member * g.strideBias + gn));
   const T* mask = g.mask ? reinterpret_cast<const T*>(g.mask) + member * g.strideMask : nullptr;
 #pragma unroll
-  for (int i = 0; i < TM; ++i) {
-    const int gm = m0 + ty * TM + i;
+  for (int i = 0; i < TMV; ++i) {
+    const int gm = m0 + ty * TMV + i;
     float4 v = make_float4(acc[i][0] + bv.x, acc[i][1] + bv.y, acc[i][2] + bv.z, acc[i][3] + bv.w);
     if (!g.bias) v = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
     if (g.relu) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f); }
@@ -749,10 +767,24 @@ template <typename T>
 static cudaError_t launch_t(const GemmArgs& g, cudaStream_t s) {
   dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.batch);
   if (simt_interior_ok<T>(g)) {
-    if (!g.a_mn && !g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, false, false>, g);
-    else if (!g.a_mn && g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, false, true>, g);
-    else if (g.a_mn && g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, true, true>, g);
-    else launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, true, false>, g);
+    // 128 x 64 tiles when they still go round the SMs (both tiles add in the same order: the choice, which depends on
+    // the number of members, does not change a bit of the result)
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const bool tall = g.M % 128 == 0 && (long long)(g.M / 128) * grid.x * g.batch * 5 >= (long long)sms * 4;
+    if (tall) {
+      grid.y = g.M / 128;
+      if (!g.a_mn && !g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, false, false, 8>, g);
+      else if (!g.a_mn && g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, false, true, 8>, g);
+      else if (g.a_mn && g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, true, true, 8>, g);
+      else launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, true, false, 8>, g);
+      return cudaGetLastError();
+    }
+    if (!g.a_mn && !g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, false, false, 4>, g);
+    else if (!g.a_mn && g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, false, true, 4>, g);
+    else if (g.a_mn && g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, true, true, 4>, g);
+    else launch_with(grid, 256, 0, s)(k_gemm_simt_interior<T, true, false, 4>, g);
     return cudaGetLastError();
   }
   if (!g.a_mn && !g.b_mn) launch_with(grid, 256, 0, s)(k_gemm_simt<T, false, false>, g);

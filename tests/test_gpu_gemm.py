@@ -101,7 +101,8 @@ def test_tensor_core_shared_operand(env):
                                    (45, 264, 5, 2), (512, 10, 256, 2), (10, 1024, 256, 3), (256, 10, 1024, 2), (136, 1, 512, 2),
                                    (8, 264, 72, 2), (2, 512, 1024, 2), (264, 16, 200, 1), (40, 1024, 10, 2),
                                    (100, 2304, 2, 1), (1024, 512, 1, 2), (300, 8, 4, 2),
-                                   (128, 512, 256, 3), (512, 256, 128, 2), (192, 128, 48, 2)])   # all tiles interior
+                                   (128, 512, 256, 3), (512, 256, 128, 2), (192, 128, 48, 2),    # all tiles interior
+                                   (256, 512, 64, 8), (128, 1024, 32, 8)])                      # ... and enough of them for 128-row tiles
 def test_alu_engine(env, dtype, a_mn, b_mn, shape):
     pkg, torch = env
     M, N, K, batch = shape
