@@ -227,7 +227,11 @@ cudaError_t launch_selftest_bounded_wait(Counters* counters, uint32_t limit, cud
 
 bool gemm_tc_supported(const GemmArgs& g) {
   if (g.in_dtype != kBF16) return false;
-  if (g.M < 128 || g.N < 128 || g.K < 64 || g.batch < 1) return false;  // every TMA box fits inside its tensor
+  if (g.M < 128 || g.K < 64 || g.batch < 1) return false;
+  // Narrow outputs (a ten-wide logit layer): a 128-column tile whose B rows past N are out-of-range rows of the
+  // tensor map and arrive as zeros, like the last tile of any ragged N.  Worth it when the ALU row-dot kernel would
+  // be bound by unpacking and multiplying (5 or more columns) and the operand is long enough to stream.
+  if (g.N < 128 && (g.N < 5 || g.a_mn || g.b_mn || g.K < 256)) return false;
   if (g.lda % 8 || g.ldb % 8) return false;
   if (g.batch > 1 && ((g.strideA != 0 && g.strideA % 8) || (g.strideB != 0 && g.strideB % 8))) return false;
   if (((uintptr_t)g.A & 15) || ((uintptr_t)g.B & 15)) return false;

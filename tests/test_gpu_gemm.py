@@ -110,6 +110,17 @@ def test_alu_engine(env, dtype, a_mn, b_mn, shape):
         _run(pkg, torch, M, N, K, batch, a_mn, b_mn, engine=1, epilogue=ep, out_bf16=ob, dtype=dtype, seed=11)
 
 
+@pytest.mark.parametrize("shape", [(256, 10, 1024, 3), (2048, 10, 1024, 2), (200, 16, 264, 2), (128, 5, 256, 1), (512, 72, 512, 2)])
+@pytest.mark.parametrize("epilogue,out_bf16", [("bias", False), ("bias_relu", True), ("none", False)])
+def test_tensor_core_narrow_outputs(env, shape, epilogue, out_bf16):
+    """Fewer than 128 output columns (a ten-wide logit layer): the B rows past N are out-of-range rows of the
+    tensor map and arrive as zeros."""
+    pkg, torch = env
+    M, N, K, batch = shape
+    _run(pkg, torch, M, N, K, batch, False, False, engine=2, epilogue=epilogue, out_bf16=out_bf16, seed=23)
+    _run(pkg, torch, M, N, K, batch, False, False, engine=0, epilogue=epilogue, out_bf16=out_bf16, seed=24)
+
+
 def test_unsupported_shapes_are_refused_by_the_tensor_engine(env):
     pkg, torch = env
     A = torch.zeros(1, 16, 16, device="cuda", dtype=torch.bfloat16)
